@@ -1,0 +1,91 @@
+"""The pins have teeth: plausible mistakes planted in a COPY of the oracle source make them fail.
+
+Each mutation is a one-token edit of ``oracle/circ_oracle.c`` compiled to a temporary library
+(CPU only); the original file and library are never touched.
+"""
+import ctypes
+import subprocess
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+SRC = Path(__file__).resolve().parent.parent / "oracle" / "circ_oracle.c"
+_dp = ctypes.POINTER(ctypes.c_double)
+
+MUTATIONS = {
+    "swapped_shift_direction": ("convention == 0 ? r - c : c - r", "convention == 0 ? c - r : r - c"),
+    "dropped_column_blocks": ("for (int j = 0; j < q; ++j) {\n                    const double* wij",
+                              "for (int j = 0; j < 1; ++j) {\n                    const double* wij"),
+    "wrong_block_stride": ("w + ((size_t)i * q + j) * k;\n                    const double* xj",
+                           "w + ((size_t)j * p + i) * k;\n                    const double* xj"),
+    "flipped_tap": ("int hi = ho + ti - pad;", "int hi = ho - ti + pad;"),
+    "transposed_taps": ("((((size_t)ti * r + tj) * p + ib) * q + jb) * k", "((((size_t)tj * r + ti) * p + ib) * q + jb) * k"),
+    "relu_on_wrong_side": ("if (relu && acc < 0.0) acc = 0.0;\n                y[", "if (relu && acc > 0.0) acc = 0.0;\n                y["),
+}
+
+
+def _build(tmp_path, name):
+    old, new = MUTATIONS[name]
+    text = SRC.read_text()
+    assert text.count(old) >= 1, f"mutation anchor for {name} not found"
+    out = tmp_path / f"{name}.c"
+    out.write_text(text.replace(old, new, 1))
+    lib = tmp_path / f"{name}.so"
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(lib), str(out), "-lm"], check=True)
+    return ctypes.CDLL(str(lib))
+
+
+def _fc(lib, w, x, bias=None, relu=False, conv=0):
+    p, q, k = w.shape
+    x = np.ascontiguousarray(np.atleast_2d(x), dtype=np.float64)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    y = np.empty((x.shape[0], p * k))
+    lib.circ_oracle_fc(p * k, q * k, k, conv, w.ctypes.data_as(_dp), x.ctypes.data_as(_dp),
+                       None if bias is None else bias.ctypes.data_as(_dp), int(relu), ctypes.c_long(x.shape[0]),
+                       y.ctypes.data_as(_dp))
+    return y
+
+
+def _conv(lib, w, x, pad):
+    r, _, p, q, k = w.shape
+    N, H, W, C = x.shape
+    y = np.empty((N, H + 2 * pad - r + 1, W + 2 * pad - r + 1, p * k))
+    lib.circ_oracle_conv(p * k, C, r, pad, k, 0, w.ctypes.data_as(_dp), x.ctypes.data_as(_dp), None, 0, N, H, W,
+                         y.ctypes.data_as(_dp))
+    return y
+
+
+def _pins_hold(lib) -> bool:
+    """A reduced copy of the pins: hand cases, a 2x3-block library product, ReLU sign, one conv tap."""
+    import scipy.linalg
+    rng = np.random.default_rng(5)
+    ok = True
+    ok &= np.array_equal(_fc(lib, np.array([1., 2, 3, 4]).reshape(1, 1, 4), np.array([1., 2, 3, 4]))[0], [26, 28, 26, 20])
+    ok &= np.array_equal(_fc(lib, np.array([1., 2, 3, 4]).reshape(1, 2, 2), np.array([1., 0, 0, 1]))[0], [5, 5])
+    w = rng.standard_normal((2, 3, 4))
+    x = rng.standard_normal((2, 12))
+    dense = np.block([[scipy.linalg.circulant(w[i, j]) for j in range(3)] for i in range(2)])
+    ok &= np.allclose(_fc(lib, w, x), x @ dense.T, atol=1e-12)
+    ok &= np.allclose(_fc(lib, w, x, relu=True), np.maximum(x @ dense.T, 0), atol=1e-12)
+    wc = np.zeros((3, 3, 1, 1, 1))
+    wc[0, 2] = 1.0
+    xc = rng.standard_normal((1, 5, 6, 1))
+    ok &= np.array_equal(_conv(lib, wc, xc, 0)[0, :, :, 0], xc[0, 0:3, 2:6, 0])
+    wc = np.zeros((3, 3, 1, 1, 1))
+    wc[2, 1] = 1.0
+    ok &= np.array_equal(_conv(lib, wc, xc, 0)[0, :, :, 0], xc[0, 2:5, 1:5, 0])
+    return bool(ok)
+
+
+def test_unmutated_copy_passes(tmp_path):
+    text = SRC.read_text()
+    (tmp_path / "plain.c").write_text(text)
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(tmp_path / "plain.so"), str(tmp_path / "plain.c"), "-lm"],
+                   check=True)
+    assert _pins_hold(ctypes.CDLL(str(tmp_path / "plain.so")))
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_planted_mistake_is_caught(tmp_path, name):
+    assert not _pins_hold(_build(tmp_path, name)), f"pins did not notice mutation {name}"

@@ -1,0 +1,209 @@
+"""Pins for the CPU oracle: everything here ties ``oracle/`` to something other than itself.
+
+Sources of truth used: hand-computed fixtures (tests/golden), the closed-form
+eigenvalues of a circulant matrix, library routines (numpy FFT, numpy matmul,
+scipy.linalg.circulant, torch float64 conv2d) and algebraic invariants of the
+layer definition (Eq. 1, Eq. 3, Eq. 6, Eq. 7 and the convolution theorem of
+Sec. 3.1).  None of these tests touches the CUDA library.
+"""
+import numpy as np
+import pytest
+import scipy.linalg
+
+import oracle
+
+RNG = np.random.default_rng(1708_08917)
+
+
+def _parse_fields(line):
+    return [np.array(f.split(), dtype=np.float64) for f in line.split("|")]
+
+
+def _hand_cases(golden_dir):
+    out = []
+    for line in (golden_dir / "hand_cases.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        conv, dims, w, x, y = _parse_fields(line)
+        m, n, k = (int(v) for v in dims)
+        out.append((int(conv[0]), m, n, k, w.reshape(m // k, n // k, k), x, y))
+    return out
+
+
+def test_hand_cases(golden_dir):
+    cases = _hand_cases(golden_dir)
+    assert len(cases) >= 15
+    for conv, m, n, k, w, x, y in cases:
+        got = oracle.fc(w, x, convention=conv)[0]
+        assert np.array_equal(got, y), (conv, m, n, k, got, y)
+
+
+def test_fig1_parameter_count():
+    # Fig. 1: an 18-entry 6x3 matrix is represented by two 3x3 circulant blocks = 6 stored parameters.
+    w = np.arange(1, 7, dtype=np.float64).reshape(2, 1, 3)
+    dense = oracle.expand_matrix(w)
+    assert dense.shape == (6, 3) and w.size == 6 and dense.size == 18
+    assert len(np.unique(dense)) == 6
+    for blk in (dense[:3], dense[3:]):
+        for r in range(1, 3):                       # each row is the previous one rotated right (Eq. 7)
+            assert np.array_equal(blk[r], np.roll(blk[r - 1], 1))
+
+
+def test_eigenvalues_closed_form(golden_dir):
+    for line in (golden_dir / "eigenvalues.txt").read_text().splitlines():
+        if not line.strip() or line.startswith("#"):
+            continue
+        kk, w, lre, lim = _parse_fields(line)
+        k = int(kk[0])
+        lam = lre + 1j * lim
+        dre, dim = oracle.dft(w)
+        np.testing.assert_allclose(dre + 1j * dim, lam, atol=1e-12)
+        t = np.arange(k)
+        for conv in (0, 1):
+            dense = oracle.expand_block(w, conv)
+            for f in range(k):
+                v = np.exp(2j * np.pi * f * t / k)
+                expect = lam[f] if conv == 0 else np.conj(lam[f])
+                np.testing.assert_allclose(dense @ v, expect * v, atol=1e-12)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 5, 8, 16, 64])
+def test_eigenvalues_random(k):
+    w = RNG.standard_normal(k)
+    lam = np.fft.fft(w)
+    t = np.arange(k)
+    dense = oracle.expand_block(w, 0)
+    for f in range(k):
+        v = np.exp(2j * np.pi * f * t / k)
+        np.testing.assert_allclose(dense @ v, lam[f] * v, atol=1e-10)
+    dre, dim = oracle.dft(w)
+    np.testing.assert_allclose(dre + 1j * dim, lam, atol=1e-10)
+
+
+@pytest.mark.parametrize("k", [2, 3, 4, 8, 16, 128])
+def test_single_block_convolution_theorem(k):
+    # Sec. 3.1: W_ij x_j = IFFT(FFT(w_ij) o FFT(x_j)); numpy's FFT is the independent routine.
+    w = RNG.standard_normal(k)
+    x = RNG.standard_normal(k)
+    via_fft = np.fft.ifft(np.fft.fft(w) * np.fft.fft(x)).real
+    np.testing.assert_allclose(oracle.fc(w.reshape(1, 1, k), x)[0], via_fft, atol=1e-12)
+    corr = np.fft.ifft(np.conj(np.fft.fft(w)) * np.fft.fft(x)).real      # the other convention = correlation
+    np.testing.assert_allclose(oracle.fc(w.reshape(1, 1, k), x, convention=1)[0], corr, atol=1e-12)
+    # the oracle's own naive DFT agrees with the library one, forward and inverse
+    fr, fi = oracle.dft(x)
+    np.testing.assert_allclose(fr + 1j * fi, np.fft.fft(x), atol=1e-10)
+    br, bi = oracle.dft(fr, fi, sign=+1)
+    np.testing.assert_allclose(br / k, x, atol=1e-10)
+    np.testing.assert_allclose(bi / k, 0, atol=1e-10)
+
+
+@pytest.mark.parametrize("p,q,k,batch", [(1, 1, 4, 1), (2, 3, 4, 2), (3, 2, 8, 3), (2, 2, 3, 2), (3, 1, 5, 1),
+                                         (1, 3, 1, 2), (4, 5, 16, 3)])
+def test_against_library_circulant_and_matmul(p, q, k, batch):
+    # scipy.linalg.circulant(c)[r][s] = c[(r-s) mod k]: first COLUMN c -- exactly convention 0;
+    # its transpose has first ROW c -- convention 1.
+    w = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((batch, q * k))
+    bias = RNG.standard_normal(p * k)
+    for conv in (0, 1):
+        dense = np.block([[scipy.linalg.circulant(w[i, j]) if conv == 0 else scipy.linalg.circulant(w[i, j]).T
+                           for j in range(q)] for i in range(p)])
+        np.testing.assert_array_equal(oracle.expand_matrix(w, conv), dense)
+        np.testing.assert_allclose(oracle.fc(w, x, convention=conv), x @ dense.T, atol=1e-12)
+        np.testing.assert_allclose(oracle.fc(w, x, bias=bias, relu=True, convention=conv),
+                                   np.maximum(x @ dense.T + bias, 0.0), atol=1e-12)
+
+
+def test_block_size_one_is_dense():
+    # "no compression if the block size is 1": k=1 is an ordinary dense layer with W = [w_ij].
+    p, q = 5, 7
+    w = RNG.standard_normal((p, q, 1))
+    x = RNG.standard_normal((3, q))
+    np.testing.assert_allclose(oracle.fc(w, x), x @ w[:, :, 0].T, atol=1e-13)
+    np.testing.assert_allclose(oracle.fc(w, x, convention=1), x @ w[:, :, 0].T, atol=1e-13)
+
+
+def test_invariants():
+    p, q, k, batch = 3, 4, 8, 2
+    w = RNG.standard_normal((p, q, k))
+    w2 = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((batch, q * k))
+    x2 = RNG.standard_normal((batch, q * k))
+    for conv in (0, 1):
+        y = oracle.fc(w, x, convention=conv)
+        # linearity in x and in w
+        np.testing.assert_allclose(oracle.fc(w, 2 * x - 3 * x2, convention=conv),
+                                   2 * y - 3 * oracle.fc(w, x2, convention=conv), atol=1e-11)
+        np.testing.assert_allclose(oracle.fc(w + w2, x, convention=conv), y + oracle.fc(w2, x, convention=conv),
+                                   atol=1e-11)
+        # rotating every input block by s rotates every output block by s
+        for s in (1, 3):
+            xs = np.roll(x.reshape(batch, q, k), s, axis=2).reshape(batch, q * k)
+            ys = oracle.fc(w, xs, convention=conv).reshape(batch, p, k)
+            np.testing.assert_allclose(ys, np.roll(y.reshape(batch, p, k), s, axis=2), atol=1e-12)
+        # DC identity: sum_r a_i[r] = sum_j (sum_t w_ij[t]) (sum_c x_j[c])
+        dc = np.einsum("ij,bj->bi", w.sum(axis=2), x.reshape(batch, q, k).sum(axis=2))
+        np.testing.assert_allclose(y.reshape(batch, p, k).sum(axis=2), dc, atol=1e-11)
+    # the two conventions differ unless the block is symmetric
+    assert not np.allclose(oracle.fc(w, x, convention=0), oracle.fc(w, x, convention=1))
+    # convention 1 with w equals convention 0 with the index-reversed vector
+    wr = np.roll(w[:, :, ::-1], 1, axis=2)
+    np.testing.assert_allclose(oracle.fc(w, x, convention=1), oracle.fc(wr, x, convention=0), atol=1e-12)
+
+
+def _dense_filters(w, k, conv):
+    r, _, p, q, _ = w.shape
+    F = np.empty((p * k, q * k, r, r))
+    for ti in range(r):
+        for tj in range(r):
+            F[:, :, ti, tj] = np.block([[scipy.linalg.circulant(w[ti, tj, i, j]) if conv == 0
+                                         else scipy.linalg.circulant(w[ti, tj, i, j]).T
+                                         for j in range(q)] for i in range(p)])
+    return F
+
+
+@pytest.mark.parametrize("r,pad,p,q,k,N,H,W", [(3, 1, 2, 2, 4, 2, 5, 6), (3, 0, 1, 2, 4, 1, 4, 4), (1, 0, 2, 3, 2, 2, 3, 3),
+                                               (5, 2, 2, 1, 3, 1, 6, 5), (2, 0, 1, 1, 8, 1, 4, 3)])
+def test_conv_against_torch_float64(r, pad, p, q, k, N, H, W):
+    # Eq. 6 is a cross-correlation (no flip) over space, summed over input channels: that is what
+    # torch.nn.functional.conv2d computes once the filters are expanded to dense form.
+    import torch
+    w = RNG.standard_normal((r, r, p, q, k))
+    x = RNG.standard_normal((N, H, W, q * k))
+    bias = RNG.standard_normal(p * k)
+    for conv in (0, 1):
+        F = _dense_filters(w, k, conv)
+        ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2), torch.from_numpy(F),
+                                         bias=torch.from_numpy(bias), padding=pad).permute(0, 2, 3, 1).numpy()
+        got = oracle.conv(w, x, pad, bias=bias, convention=conv)
+        assert got.shape == (N, H + 2 * pad - r + 1, W + 2 * pad - r + 1, p * k)
+        np.testing.assert_allclose(got, ref, atol=1e-11)
+        np.testing.assert_allclose(oracle.conv(w, x, pad, bias=bias, relu=True, convention=conv),
+                                   np.maximum(ref, 0), atol=1e-11)
+        pix = [(0, 0, 0), (N - 1, got.shape[1] - 1, got.shape[2] - 1), (0, got.shape[1] // 2, got.shape[2] - 1)]
+        sampled = oracle.conv_pixels(w, x, pad, pix, bias=bias, convention=conv)
+        for t, (a, b, c) in enumerate(pix):
+            np.testing.assert_allclose(sampled[t], ref[a, b, c], atol=1e-11)
+
+
+def test_conv_valid_extent_and_tap_orientation():
+    # Eq. 6: output extent (W-r+1) x (H-r+1); tap (i,j) multiplies X(x+i-1, y+j-1): a single 1 at tap
+    # (0,2) of a 3x3 filter (k=1, one channel) copies the input shifted by (0, +2).
+    w = np.zeros((3, 3, 1, 1, 1))
+    w[0, 2] = 1.0
+    x = RNG.standard_normal((1, 5, 6, 1))
+    y = oracle.conv(w, x, pad=0)
+    assert y.shape == (1, 3, 4, 1)
+    np.testing.assert_array_equal(y[0, :, :, 0], x[0, 0:3, 2:6, 0])
+
+
+def test_conv_1x1_equals_fc():
+    p, q, k = 2, 3, 4
+    w = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((2, 3, 3, q * k))
+    y = oracle.conv(w.reshape(1, 1, p, q, k), x, pad=0)
+    np.testing.assert_allclose(y.reshape(-1, p * k), oracle.fc(w, x.reshape(-1, q * k)), atol=1e-13)
+
+
+def test_threads_reported():
+    assert oracle.threads() >= 1
