@@ -1,0 +1,155 @@
+/*
+ * circ.h -- C ABI of the block-circulant layer library (CUDA, sm_100a).
+ *
+ * A layer's m x n weight matrix is cut into p x q square blocks of size k
+ * (p = m / k, q = n / k); every block is circulant and is stored as one
+ * length-k defining vector w_ij (Sec. 3.1, Eq. 3).  The forward pass is
+ *
+ *     y_i = psi( IFFT( sum_j FFT(w_ij) o FFT(x_j) ) + theta_i )        (Algorithm 1 + Eq. 1)
+ *
+ * with the weight spectra computed once at create time, one forward transform
+ * per input block, accumulation in the frequency domain, and one inverse
+ * transform per output block with bias and ReLU fused.  Convolution layers use
+ * the same structure along the channel pair at every filter tap (Sec. 3.2,
+ * Eq. 6 and Eq. 7).
+ *
+ * General rules
+ *   - All functions are extern "C"; no exception crosses the boundary.
+ *   - Functions returning int return CIRC_OK (0) or a negative CIRC_ERR_* code;
+ *     create functions return NULL on error.  circ_last_error() gives a
+ *     thread-local message for the most recent failure.
+ *   - There is no CPU fallback: every call that computes needs a CUDA device.
+ *   - A handle belongs to the device that was current when it was created.
+ *   - Calls on one handle must not run concurrently (the handle owns one
+ *     workspace); different handles are independent.
+ */
+#ifndef CIRC_H_
+#define CIRC_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CIRC_API __attribute__((visibility("default")))
+#else
+#define CIRC_API
+#endif
+
+typedef struct circ_layer* circ_handle; /* opaque, owned by the library */
+
+enum {
+    CIRC_OK = 0,
+    CIRC_ERR_ARG = -1,            /* NULL / misaligned pointer, bad enum value, wrong handle kind */
+    CIRC_ERR_SHAPE = -2,          /* k not a power of two in [4,256], k does not divide m or n, batch < 1 ... */
+    CIRC_ERR_ALLOC = -3,          /* device or host allocation failed */
+    CIRC_ERR_CUDA = -4,           /* a CUDA runtime call or a kernel launch failed */
+    CIRC_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up */
+    CIRC_ERR_UNSUPPORTED = -6     /* valid request that this build cannot serve */
+};
+
+enum { CIRC_F32 = 0, CIRC_BF16 = 1 };
+
+/* Kernel variants (circ_set_variant). */
+enum {
+    CIRC_VARIANT_AUTO = 0,   /* chosen from (p, q, k, batch) */
+    CIRC_VARIANT_FUSED = 1,  /* one launch: transform x, stream the spectra, accumulate, inverse transform */
+    CIRC_VARIANT_STAGED = 2, /* three launches: transforms, per-frequency contraction on fp32 FMA pipes */
+    CIRC_VARIANT_TENSOR = 3  /* three launches, per-frequency contraction on the tensor cores */
+};
+
+/*
+ * circ_fc_create -- build a fully-connected block-circulant layer (Sec. 3.1).
+ *   m, n : output / input widths; k : block size, a power of two in [4, 256]
+ *          that divides both (the paper defines p = m / k, q = n / k and has no
+ *          remainder rule; pad on the caller's side).
+ *   w    : float32 defining vectors, layout [p][q][k]: w[(i*q + j)*k + t] is
+ *          element t of w_ij.  HOST or DEVICE pointer (detected); read during
+ *          the call, the caller keeps ownership.
+ * Circulant convention 0 (default): W_ij[r][c] = w_ij[(r - c) mod k], i.e.
+ * a_i = sum_j w_ij (*) x_j (circular convolution), which is what Algorithm 1's
+ * FFT product computes.  See circ_set_convention for the other reading.
+ * Computes the weight spectra FFT(w_ij) (the quantity the paper keeps in RAM,
+ * Sec. 4.2) on the current device and synchronises before returning.
+ * Defaults: no bias, identity activation, float32 x and y.
+ * Returns NULL on error (CIRC_ERR_SHAPE / ARG / ALLOC / CUDA in circ_last_code()).
+ */
+CIRC_API circ_handle circ_fc_create(int m, int n, int k, const float* w);
+
+/*
+ * circ_fc_forward -- y = psi(W x + theta) for a batch (Eq. 1, Algorithm 1).
+ *   x : DEVICE pointer, [batch][n] row-major contiguous, float32 or bfloat16 (circ_set_io_dtype)
+ *   y : DEVICE pointer, [batch][m] row-major contiguous; must not alias x
+ *   both 16-byte aligned, owned by the caller
+ *   stream : a cudaStream_t passed as void* (NULL = legacy default stream)
+ * Only enqueues work on `stream`; never synchronises.  After circ_reserve(h, B)
+ * a forward with batch <= B allocates nothing; otherwise the workspace grows
+ * (cudaMalloc) before the launch.
+ */
+CIRC_API int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stream);
+
+/*
+ * circ_conv_create -- build an r x r, stride-1 block-circulant convolution (Sec. 3.2).
+ *   c_out, c_in : output / input channels (P and C of Eq. 6); k divides both
+ *   r : filter size (1..7); pad : zero padding on each side (0..r-1)
+ *   w : float32 [r][r][p][q][k], p = c_out / k, q = c_in / k: at every tap (i, j)
+ *       the channel pair is a p x q grid of circulant blocks (Eq. 7), same
+ *       convention as the FC layer.  HOST or DEVICE pointer.
+ * Defaults: no bias, identity, bfloat16 x and y (change with circ_set_io_dtype).
+ */
+CIRC_API circ_handle circ_conv_create(int c_out, int c_in, int r, int pad, int k, const float* w);
+
+/*
+ * circ_conv_forward -- Eq. 6 with zero padding (cross-correlation, no filter flip):
+ *   y[n][h][w][P] = psi( theta + sum_{i,j<r} sum_c F(i,j,c,P) x[n][h+i-pad][w+j-pad][c] ),  out-of-image x = 0
+ *   x : DEVICE pointer, channel-last [N][H][W][c_in]
+ *   y : DEVICE pointer, channel-last [N][H + 2 pad - r + 1][W + 2 pad - r + 1][c_out]
+ * Same stream / allocation / alignment rules as circ_fc_forward.
+ */
+CIRC_API int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W, void* stream);
+
+/* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
+CIRC_API void circ_destroy(circ_handle h);
+
+/* circ_set_bias -- theta of Eq. 1: float32, length m (c_out); HOST or DEVICE pointer, copied.
+ * NULL removes the bias. */
+CIRC_API int circ_set_bias(circ_handle h, const float* bias);
+
+/* circ_set_activation -- psi of Eq. 1: 0 = identity, 1 = ReLU max(0, v). */
+CIRC_API int circ_set_activation(circ_handle h, int relu);
+
+/* circ_set_io_dtype -- element types of x and y in device memory (CIRC_F32 / CIRC_BF16).
+ * Arithmetic is float32 inside; bfloat16 outputs are rounded to nearest even.  With bfloat16
+ * inputs the tensor-core contraction takes single bfloat16 operands (float32 accumulate);
+ * with float32 inputs it takes split (high + low) bfloat16 operands. */
+CIRC_API int circ_set_io_dtype(circ_handle h, int x_dtype, int y_dtype);
+
+/* circ_set_convention -- 0: W_ij[r][c] = w_ij[(r-c) mod k] (default, Algorithm 1);
+ * 1: W_ij[r][c] = w_ij[(c-r) mod k] (w_ij read literally as the first row with a column
+ * vector x).  Recomputes the spectra from the retained copy of w; synchronises. */
+CIRC_API int circ_set_convention(circ_handle h, int convention);
+
+/* circ_set_variant -- force a kernel variant (CIRC_VARIANT_*); AUTO restores the planner. */
+CIRC_API int circ_set_variant(circ_handle h, int variant);
+
+/* circ_reserve -- size the workspace for forwards up to `max_batch` samples (FC) or pixels
+ * N*H*W (CONV), so that later forwards allocate nothing. */
+CIRC_API int circ_reserve(circ_handle h, long max_batch);
+
+/* circ_workspace_bytes -- bytes of device workspace currently held by the handle. */
+CIRC_API long circ_workspace_bytes(circ_handle h);
+
+/* circ_last_variant -- the CIRC_VARIANT_* the most recent forward on this handle used. */
+CIRC_API int circ_last_variant(circ_handle h);
+
+/* circ_launch_count -- kernels this library has launched in this process so far. */
+CIRC_API long circ_launch_count(void);
+
+/* circ_last_error / circ_last_code -- message and code of the calling thread's latest failure. */
+CIRC_API const char* circ_last_error(void);
+CIRC_API int circ_last_code(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CIRC_H_ */

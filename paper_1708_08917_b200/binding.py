@@ -1,0 +1,176 @@
+"""ctypes binding of ``libcirc.so``: the same names as ``include/circ.h``, argument marshalling only.
+
+Every step of the forward pass runs inside the CUDA library; nothing here computes.  torch (or any
+other owner of device memory) is used by callers for allocation and streams only: tensors are
+passed as raw device pointers, streams as ``cudaStream_t`` integers.  If the library has not been
+built, or cannot be loaded, importing a function from here raises -- there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+LIB_PATH = _HERE / "libcirc.so"
+
+CIRC_OK = 0
+CIRC_ERR_ARG, CIRC_ERR_SHAPE, CIRC_ERR_ALLOC, CIRC_ERR_CUDA, CIRC_ERR_DEVICE_TIMEOUT, CIRC_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
+CIRC_F32, CIRC_BF16 = 0, 1
+CIRC_VARIANT_AUTO, CIRC_VARIANT_FUSED, CIRC_VARIANT_STAGED, CIRC_VARIANT_TENSOR = 0, 1, 2, 3
+
+# name -> (restype, argtypes); mirrors include/circ.h one to one
+_vp, _ci, _cl = ctypes.c_void_p, ctypes.c_int, ctypes.c_long
+SIGNATURES = {
+    "circ_fc_create": (_vp, [_ci, _ci, _ci, _vp]),
+    "circ_fc_forward": (_ci, [_vp, _vp, _vp, _ci, _vp]),
+    "circ_conv_create": (_vp, [_ci, _ci, _ci, _ci, _ci, _vp]),
+    "circ_conv_forward": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
+    "circ_destroy": (None, [_vp]),
+    "circ_set_bias": (_ci, [_vp, _vp]),
+    "circ_set_activation": (_ci, [_vp, _ci]),
+    "circ_set_io_dtype": (_ci, [_vp, _ci, _ci]),
+    "circ_set_convention": (_ci, [_vp, _ci]),
+    "circ_set_variant": (_ci, [_vp, _ci]),
+    "circ_reserve": (_ci, [_vp, _cl]),
+    "circ_workspace_bytes": (_cl, [_vp]),
+    "circ_last_variant": (_ci, [_vp]),
+    "circ_launch_count": (_cl, []),
+    "circ_last_error": (ctypes.c_char_p, []),
+    "circ_last_code": (_ci, []),
+}
+
+_lib = None
+
+
+class CircError(RuntimeError):
+    """A libcirc call failed; ``code`` is the CIRC_ERR_* value."""
+
+    def __init__(self, code: int, message: str):
+        super().__init__(f"libcirc error {code}: {message}")
+        self.code = code
+
+
+def load() -> ctypes.CDLL:
+    """Load ``libcirc.so`` (built by ``paper_1708_08917_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1708_08917_b200.build` "
+                              "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _ptr(a) -> int | None:
+    """Raw address of a torch tensor, a numpy array, an int, or None."""
+    if a is None:
+        return None
+    if isinstance(a, int):
+        return a
+    if isinstance(a, np.ndarray):
+        assert a.flags["C_CONTIGUOUS"]
+        return a.ctypes.data
+    assert a.is_contiguous()
+    return a.data_ptr()
+
+
+def _stream(stream) -> int | None:
+    if stream is None or isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(rc: int) -> None:
+    if rc != CIRC_OK:
+        raise CircError(rc, circ_last_error())
+
+
+def _weights(w):
+    if isinstance(w, np.ndarray):
+        w = np.ascontiguousarray(w, dtype=np.float32)
+    return w
+
+
+def circ_last_error() -> str:
+    return load().circ_last_error().decode()
+
+
+def circ_last_code() -> int:
+    return load().circ_last_code()
+
+
+def circ_fc_create(m: int, n: int, k: int, w) -> int:
+    """``w``: float32 ``[p][q][k]`` defining vectors (numpy array on the host or a device tensor)."""
+    w = _weights(w)
+    h = load().circ_fc_create(m, n, k, _ptr(w))
+    if not h:
+        raise CircError(circ_last_code(), circ_last_error())
+    return h
+
+
+def circ_conv_create(c_out: int, c_in: int, r: int, pad: int, k: int, w) -> int:
+    """``w``: float32 ``[r][r][p][q][k]``."""
+    w = _weights(w)
+    h = load().circ_conv_create(c_out, c_in, r, pad, k, _ptr(w))
+    if not h:
+        raise CircError(circ_last_code(), circ_last_error())
+    return h
+
+
+def circ_fc_forward(h: int, x, y, batch: int, stream=None) -> None:
+    """Enqueue ``y[batch][m] = psi(W x + theta)``; ``x``, ``y`` are device tensors or raw device addresses."""
+    _check(load().circ_fc_forward(h, _ptr(x), _ptr(y), batch, _stream(stream)))
+
+
+def circ_conv_forward(h: int, x, y, N: int, H: int, W: int, stream=None) -> None:
+    """Enqueue the channel-last convolution ``x[N][H][W][C] -> y[N][Ho][Wo][P]``."""
+    _check(load().circ_conv_forward(h, _ptr(x), _ptr(y), N, H, W, _stream(stream)))
+
+
+def circ_destroy(h: int | None) -> None:
+    load().circ_destroy(h)
+
+
+def circ_set_bias(h: int, bias) -> None:
+    if isinstance(bias, np.ndarray):
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+    _check(load().circ_set_bias(h, _ptr(bias)))
+
+
+def circ_set_activation(h: int, relu: int) -> None:
+    _check(load().circ_set_activation(h, int(relu)))
+
+
+def circ_set_io_dtype(h: int, x_dtype: int, y_dtype: int) -> None:
+    _check(load().circ_set_io_dtype(h, x_dtype, y_dtype))
+
+
+def circ_set_convention(h: int, convention: int) -> None:
+    _check(load().circ_set_convention(h, convention))
+
+
+def circ_set_variant(h: int, variant: int) -> None:
+    _check(load().circ_set_variant(h, variant))
+
+
+def circ_reserve(h: int, max_batch: int) -> None:
+    _check(load().circ_reserve(h, max_batch))
+
+
+def circ_workspace_bytes(h: int) -> int:
+    return load().circ_workspace_bytes(h)
+
+
+def circ_last_variant(h: int) -> int:
+    return load().circ_last_variant(h)
+
+
+def circ_launch_count() -> int:
+    return load().circ_launch_count()

@@ -1,0 +1,367 @@
+// The C ABI (include/circ.h): argument checking, the layer object, workspace, variant choice.
+#include <atomic>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "circ_common.cuh"
+
+namespace circ {
+
+static thread_local char g_err[512] = "";
+static thread_local int g_code = CIRC_OK;
+static std::atomic<long> g_launches{0};
+
+void set_error(int code, const char* fmt, ...) {
+    g_code = code;
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    if (getenv("CIRC_LOG")) fprintf(stderr, "[circ] error %d: %s\n", code, g_err);
+}
+void count_launches(long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+static bool pow2_in_range(int k) { return k >= 4 && k <= 256 && (k & (k - 1)) == 0; }
+
+// Copy `count` floats from a host or device pointer into fresh device memory.
+static int to_device(const float* src, size_t count, float** out) {
+    float* d = nullptr;
+    if (cudaMalloc(&d, count * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        set_error(CIRC_ERR_ALLOC, "cudaMalloc of %zu bytes failed", count * sizeof(float));
+        return CIRC_ERR_ALLOC;
+    }
+    // cudaMemcpyDefault resolves host / device / managed sources under unified addressing.
+    cudaError_t e = cudaMemcpy(d, src, count * sizeof(float), cudaMemcpyDefault);
+    if (e != cudaSuccess) {
+        cudaFree(d);
+        set_error(CIRC_ERR_CUDA, "copy of %zu floats failed: %s", count, cudaGetErrorString(e));
+        return CIRC_ERR_CUDA;
+    }
+    *out = d;
+    return CIRC_OK;
+}
+
+static void free_layer(Layer* L) {
+    if (!L) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    if (prev != L->device) cudaSetDevice(L->device);
+    cudaFree(L->w_dev);
+    cudaFree(L->bias_dev);
+    cudaFree(L->tw256);
+    cudaFree(L->w_stream);
+    cudaFree(L->a_f32);
+    cudaFree(L->a_bf16);
+    cudaFree(L->ws);
+    cudaFree(L->dev_status);
+    if (prev != L->device && prev >= 0) cudaSetDevice(prev);
+    delete L;
+}
+
+static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const float* w) {
+    if (!w) {
+        set_error(CIRC_ERR_ARG, "w is NULL");
+        return nullptr;
+    }
+    if (!pow2_in_range(k)) {
+        set_error(CIRC_ERR_SHAPE, "block size k=%d must be a power of two in [4, 256]", k);
+        return nullptr;
+    }
+    if (m <= 0 || n <= 0 || m % k || n % k) {
+        set_error(CIRC_ERR_SHAPE, "k=%d must divide m=%d and n=%d (pad on the caller's side)", k, m, n);
+        return nullptr;
+    }
+    Layer* L = new (std::nothrow) Layer();
+    if (!L) {
+        set_error(CIRC_ERR_ALLOC, "host allocation failed");
+        return nullptr;
+    }
+    memset(L, 0, sizeof(*L));
+    L->kind = kind;
+    L->m = m;
+    L->n = n;
+    L->geo = Geometry{m / k, n / k, k, taps, r, pad};
+    L->x_dtype = L->y_dtype = (kind == 1 ? CIRC_BF16 : CIRC_F32);
+    L->variant = CIRC_VARIANT_AUTO;
+    if (cudaGetDevice(&L->device) != cudaSuccess) {
+        set_error(CIRC_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
+        delete L;
+        return nullptr;
+    }
+    const size_t wcount = (size_t)taps * (m / k) * (n / k) * k;
+    if (to_device(w, wcount, &L->w_dev) != CIRC_OK) {
+        free_layer(L);
+        return nullptr;
+    }
+    // master twiddle table exp(-2 pi i n / 256) in double precision
+    float2 host_tw[256];
+    for (int i = 0; i < 256; ++i) {
+        const double ang = -2.0 * M_PI * (double)i / 256.0;
+        host_tw[i] = make_float2((float)cos(ang), (float)sin(ang));
+    }
+    host_tw[0] = make_float2(1.f, 0.f);
+    host_tw[64] = make_float2(0.f, -1.f);
+    host_tw[128] = make_float2(-1.f, 0.f);
+    host_tw[192] = make_float2(0.f, 1.f);
+    const size_t a_real = (size_t)taps * (m / k) * (n / k);
+    L->a_elems = 2 * a_real + (size_t)(k / 2 - 1) * 4 * a_real;
+    bool ok = cudaMalloc(&L->tw256, sizeof(host_tw)) == cudaSuccess &&
+              cudaMalloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
+              cudaMalloc(&L->dev_status, sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        set_error(CIRC_ERR_ALLOC, "device allocation of the weight spectra failed");
+        free_layer(L);
+        return nullptr;
+    }
+    if (cudaMemcpy(L->tw256, host_tw, sizeof(host_tw), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(L->dev_status, 0, sizeof(int)) != cudaSuccess || launch_precompute(L, 0) != CIRC_OK ||
+        cudaDeviceSynchronize() != cudaSuccess) {
+        set_error(CIRC_ERR_CUDA, "spectrum precompute failed: %s", cudaGetErrorString(cudaGetLastError()));
+        free_layer(L);
+        return nullptr;
+    }
+    return L;
+}
+
+static size_t workspace_need(const Layer* L, const Extent& e) {
+    const size_t xin = (size_t)2 * e.Bh * L->geo.q * L->geo.k;   // floats: all problems of X
+    const size_t yout = (size_t)2 * e.Bho * L->geo.p * L->geo.k; // floats: all problems of Y
+    return (xin + yout) * sizeof(float) + 512;
+}
+
+static int ensure_workspace(Layer* L, size_t need) {
+    if (L->ws_bytes >= need) return CIRC_OK;
+    if (L->ws) cudaFree(L->ws);  // implicit synchronisation: earlier forwards have finished with it
+    L->ws = nullptr;
+    L->ws_bytes = 0;
+    if (cudaMalloc(&L->ws, need) != cudaSuccess) {
+        cudaGetLastError();
+        set_error(CIRC_ERR_ALLOC, "workspace allocation of %zu bytes failed", need);
+        return CIRC_ERR_ALLOC;
+    }
+    L->ws_bytes = need;
+    return CIRC_OK;
+}
+
+static Extent fc_extent(int batch) {
+    Extent e;
+    e.B = e.Bo = batch;
+    e.Bh = e.Bho = (batch + 1) / 2;
+    e.H = e.Ho = 1;
+    e.W = e.Wo = batch;
+    e.Nh = e.Bh;
+    return e;
+}
+
+static Extent conv_extent(const Layer* L, int N, int H, int W) {
+    Extent e;
+    e.H = H;
+    e.W = W;
+    e.Ho = H + 2 * L->geo.pad - L->geo.r + 1;
+    e.Wo = W + 2 * L->geo.pad - L->geo.r + 1;
+    e.Nh = (N + 1) / 2;
+    e.B = N * H * W;
+    e.Bh = e.Nh * H * W;
+    e.Bo = N * e.Ho * e.Wo;
+    e.Bho = e.Nh * e.Ho * e.Wo;
+    return e;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_io(const Layer* L, const void* x, const void* y) {
+    if (!L) {
+        set_error(CIRC_ERR_ARG, "handle is NULL");
+        return CIRC_ERR_ARG;
+    }
+    if (!x || !y || x == y) {
+        set_error(CIRC_ERR_ARG, "x and y must be distinct non-NULL device pointers");
+        return CIRC_ERR_ARG;
+    }
+    if (!aligned16(x) || !aligned16(y)) {
+        set_error(CIRC_ERR_ARG, "x and y must be 16-byte aligned");
+        return CIRC_ERR_ARG;
+    }
+    return CIRC_OK;
+}
+
+static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream) {
+    int rc = ensure_workspace(L, workspace_need(L, e));
+    if (rc != CIRC_OK) return rc;
+    float* xop = static_cast<float*>(L->ws);
+    float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
+    if ((rc = launch_input_fft(L, x, xop, e, stream)) != CIRC_OK) return rc;
+    if ((rc = launch_contract_fma(L, xop, yop, e, stream)) != CIRC_OK) return rc;
+    if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
+    L->last_variant = CIRC_VARIANT_STAGED;
+    return CIRC_OK;
+}
+
+}  // namespace circ
+
+using namespace circ;
+
+extern "C" {
+
+circ_handle circ_fc_create(int m, int n, int k, const float* w) {
+    return reinterpret_cast<circ_handle>(make_layer(0, m, n, k, 1, 1, 0, w));
+}
+
+circ_handle circ_conv_create(int c_out, int c_in, int r, int pad, int k, const float* w) {
+    if (r < 1 || r > 7 || pad < 0 || pad >= (r > 1 ? r : 2)) {
+        set_error(CIRC_ERR_SHAPE, "filter size r=%d must be in [1,7] and pad=%d in [0,r-1]", r, pad);
+        return nullptr;
+    }
+    return reinterpret_cast<circ_handle>(make_layer(1, c_out, c_in, k, r * r, r, pad, w));
+}
+
+void circ_destroy(circ_handle h) { free_layer(reinterpret_cast<Layer*>(h)); }
+
+int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    int rc = check_io(L, x, y);
+    if (rc != CIRC_OK) return rc;
+    if (L->kind != 0) {
+        set_error(CIRC_ERR_ARG, "circ_fc_forward called on a convolution handle");
+        return CIRC_ERR_ARG;
+    }
+    if (batch < 1) {
+        set_error(CIRC_ERR_SHAPE, "batch=%d must be >= 1", batch);
+        return CIRC_ERR_SHAPE;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int variant = L->variant;
+    if (variant == CIRC_VARIANT_AUTO) variant = fused_fc_supported(L, batch) && batch <= 8 ? CIRC_VARIANT_FUSED : CIRC_VARIANT_STAGED;
+    if (variant == CIRC_VARIANT_FUSED) {
+        if (!fused_fc_supported(L, batch)) {
+            set_error(CIRC_ERR_UNSUPPORTED, "the fused kernel does not serve batch=%d for this layer", batch);
+            return CIRC_ERR_UNSUPPORTED;
+        }
+        rc = launch_fused_fc(L, x, y, batch, s);
+        if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
+        return rc;
+    }
+    if (variant == CIRC_VARIANT_TENSOR) {
+        set_error(CIRC_ERR_UNSUPPORTED, "tensor-core contraction not available in this build");
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    return run_staged(L, x, y, fc_extent(batch), s);
+}
+
+int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    int rc = check_io(L, x, y);
+    if (rc != CIRC_OK) return rc;
+    if (L->kind != 1) {
+        set_error(CIRC_ERR_ARG, "circ_conv_forward called on a fully-connected handle");
+        return CIRC_ERR_ARG;
+    }
+    if (N < 1 || H < 1 || W < 1 || H + 2 * L->geo.pad < L->geo.r || W + 2 * L->geo.pad < L->geo.r) {
+        set_error(CIRC_ERR_SHAPE, "bad image extent N=%d H=%d W=%d for r=%d pad=%d", N, H, W, L->geo.r, L->geo.pad);
+        return CIRC_ERR_SHAPE;
+    }
+    if ((long)N * H * W > (1L << 30)) {
+        set_error(CIRC_ERR_SHAPE, "N*H*W too large");
+        return CIRC_ERR_SHAPE;
+    }
+    if (L->variant == CIRC_VARIANT_FUSED || L->variant == CIRC_VARIANT_TENSOR) {
+        set_error(CIRC_ERR_UNSUPPORTED, "variant %d not available for convolutions in this build", L->variant);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    return run_staged(L, x, y, conv_extent(L, N, H, W), static_cast<cudaStream_t>(stream));
+}
+
+int circ_set_bias(circ_handle h, const float* bias) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L) {
+        set_error(CIRC_ERR_ARG, "handle is NULL");
+        return CIRC_ERR_ARG;
+    }
+    CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+    cudaFree(L->bias_dev);
+    L->bias_dev = nullptr;
+    if (!bias) return CIRC_OK;
+    return to_device(bias, (size_t)L->m, &L->bias_dev);
+}
+
+int circ_set_activation(circ_handle h, int relu) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (relu != 0 && relu != 1)) {
+        set_error(CIRC_ERR_ARG, "bad handle or activation code %d", relu);
+        return CIRC_ERR_ARG;
+    }
+    L->relu = relu;
+    return CIRC_OK;
+}
+
+int circ_set_io_dtype(circ_handle h, int x_dtype, int y_dtype) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (x_dtype != CIRC_F32 && x_dtype != CIRC_BF16) || (y_dtype != CIRC_F32 && y_dtype != CIRC_BF16)) {
+        set_error(CIRC_ERR_ARG, "bad handle or dtype codes (%d, %d)", x_dtype, y_dtype);
+        return CIRC_ERR_ARG;
+    }
+    L->x_dtype = x_dtype;
+    L->y_dtype = y_dtype;
+    return CIRC_OK;
+}
+
+int circ_set_convention(circ_handle h, int convention) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (convention != 0 && convention != 1)) {
+        set_error(CIRC_ERR_ARG, "bad handle or convention %d", convention);
+        return CIRC_ERR_ARG;
+    }
+    if (convention == L->convention) return CIRC_OK;
+    CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+    L->convention = convention;
+    int rc = launch_precompute(L, 0);
+    if (rc != CIRC_OK) return rc;
+    CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int circ_set_variant(circ_handle h, int variant) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || variant < CIRC_VARIANT_AUTO || variant > CIRC_VARIANT_TENSOR) {
+        set_error(CIRC_ERR_ARG, "bad handle or variant %d", variant);
+        return CIRC_ERR_ARG;
+    }
+    L->variant = variant;
+    return CIRC_OK;
+}
+
+int circ_reserve(circ_handle h, long max_batch) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || max_batch < 1 || max_batch > (1L << 30)) {
+        set_error(CIRC_ERR_ARG, "bad handle or max_batch %ld", max_batch);
+        return CIRC_ERR_ARG;
+    }
+    // Bound for both layer kinds: pairs <= ceil(max_batch / 2) + one image's worth of slack is
+    // covered by sizing for max_batch pairs on each side.
+    Extent e;
+    e.Bh = e.Bho = (int)max_batch;
+    return ensure_workspace(L, workspace_need(L, e));
+}
+
+long circ_workspace_bytes(circ_handle h) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    return L ? (long)L->ws_bytes : 0;
+}
+
+int circ_last_variant(circ_handle h) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    return L ? L->last_variant : 0;
+}
+
+long circ_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+const char* circ_last_error(void) { return g_err; }
+int circ_last_code(void) { return g_code; }
+
+}  // extern "C"

@@ -1,0 +1,126 @@
+// Shared declarations of the block-circulant layer library: the layer object, the
+// layouts of the stored spectra and of the frequency-domain operands, and error plumbing.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/circ.h"
+
+namespace circ {
+
+// ---------------------------------------------------------------------------------------------
+// Frequency-domain layouts.
+//
+// Two real signals share one complex transform (see circ_fft.cuh).  Sample (or pixel) b < Bh is the
+// real part of pair b, sample Bh + b its imaginary part (Bh = "half": number of pairs).  The size-K
+// complex spectrum Z[f] of a pair is multiplied by the weight spectrum What[f], with
+// What[K - f] = conj(What[f]) because w is real.  Bins f and K - f therefore share one weight
+// matrix, and the per-frequency contraction  Yhat[f] (p x cols) = What[f] (p x q) . Z[f] (q x cols)
+// is organised as K/2 + 1 real "problems":
+//
+//   problem 0 : bin 0          real    M = p,  Kd = q    column c      <- Re Z[0]  of pair c
+//   problem 1 : bin K/2        real                      column Bh+c   <- Im Z[..] of pair c
+//   problem g+1, 0 < g < K/2 : complex, embedded as a real product
+//        [Yr]   [Wr -Wi] [Zr]      M = 2p, Kd = 2q       column c      <- ( Re Z[g],    Im Z[g]   )
+//        [Yi] = [Wi  Wr] [Zi]                            column Bh+c   <- ( Re Z[K-g], -Im Z[K-g] )
+//   (the second column group is the conjugate of bin K-g, so that it multiplies What[g] too).
+//
+// Every problem has 2*Bh columns.  Operands are "K-major": X[col][kk], A[row][kk]; results are
+// Y[col][row].  Convolutions concatenate the taps along the contraction index:
+// kk = tap * Kd + (kk within tap), and the column of tap (di, dj) is the input pixel shifted by it.
+// ---------------------------------------------------------------------------------------------
+
+struct Geometry {
+    int p, q, k;      // block grid and block size
+    int taps;         // 1 for FC, r*r for CONV
+    int r, pad;       // CONV filter size and zero padding (r = 1, pad = 0 for FC)
+};
+
+__host__ __device__ inline int problem_of_bin(int g, int k) { return g == 0 ? 0 : (g == k / 2 ? 1 : g + 1); }
+__host__ __device__ inline int num_problems(int k) { return k / 2 + 1; }
+__host__ __device__ inline bool problem_is_real(int prob) { return prob < 2; }
+
+// Offset (in elements) of problem `prob` inside an operand whose real problems have `real_sz`
+// elements each and whose complex problems have `cplx_sz` elements each.
+__host__ __device__ inline size_t problem_offset(int prob, size_t real_sz, size_t cplx_sz) {
+    return prob < 2 ? (size_t)prob * real_sz : 2 * real_sz + (size_t)(prob - 2) * cplx_sz;
+}
+
+// Spatial description of a forward call.  FC: images = 1, H = 1, W = batch (pixels = samples).
+struct Extent {
+    int B;        // real samples / pixels on the input side (N*H*W)
+    int Bh;       // pairs on the input side
+    int Bo;       // real samples / pixels on the output side
+    int Bho;      // pairs on the output side
+    int H, W;     // input image
+    int Ho, Wo;   // output image
+    int Nh;       // image pairs (CONV); FC: Bh
+};
+
+struct Epilogue {
+    const float* bias;  // device, length m, or nullptr
+    int relu;
+};
+
+// ---------------------------------------------------------------------------------------------
+// The layer object behind circ_handle.
+// ---------------------------------------------------------------------------------------------
+struct Layer {
+    int kind;  // 0 = FC, 1 = CONV
+    int device;
+    int m, n;  // FC: output / input width; CONV: c_out / c_in
+    Geometry geo;
+    int convention;
+    int relu;
+    int x_dtype, y_dtype;
+    int variant;
+    int last_variant;
+
+    float* w_dev;       // retained copy of the defining vectors [taps][p][q][k]
+    float* bias_dev;    // [m] or nullptr
+    float2* tw256;      // exp(-2 pi i n / 256), n < 256
+    float* w_stream;    // spectra for the fused kernel: [taps][p][q][k] packed half spectra
+    float* a_f32;       // embedded float32 operand for the staged FMA contraction
+    __nv_bfloat16* a_bf16;  // embedded bfloat16 operand (hi | lo split) for the tensor-core contraction
+    size_t a_elems;     // elements of a_f32
+
+    void* ws;           // workspace: frequency-domain operands X and Y
+    size_t ws_bytes;
+    int* dev_status;    // device error word (bounded waits report here)
+};
+
+// Thread-local error record.
+void set_error(int code, const char* fmt, ...);
+void count_launches(long n);
+
+#define CIRC_CUDA_TRY(expr, ret)                                                             \
+    do {                                                                                     \
+        cudaError_t e_ = (expr);                                                             \
+        if (e_ != cudaSuccess) {                                                             \
+            ::circ::set_error(CIRC_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+            return ret;                                                                      \
+        }                                                                                    \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Kernel launchers (one translation unit each).  All return a CIRC_* code and only enqueue.
+// ---------------------------------------------------------------------------------------------
+
+// S0: spectra of the defining vectors, in every stored layout.
+int launch_precompute(Layer* L, cudaStream_t stream);
+
+// S1 / C1: forward transforms of the input -> operand X (float32, layout above).
+int launch_input_fft(const Layer* L, const void* x, float* xop, const Extent& ext, cudaStream_t stream);
+
+// S2 / C2 on the float32 FMA pipes: Y = A . X per problem.
+int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream);
+
+// S3 / C3: inverse transforms + bias + activation -> y.
+int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);
+
+// S4: the whole FC forward in one launch (small batch, weight-streaming).
+int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStream_t stream);
+bool fused_fc_supported(const Layer* L, int batch);
+
+}  // namespace circ

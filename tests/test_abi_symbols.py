@@ -1,0 +1,55 @@
+"""The C-ABI library builds, loads and exports every symbol include/circ.h declares (no GPU needed)."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_1708_08917_b200 import build
+    return ctypes.CDLL(str(build.build()))
+
+
+def declared_functions():
+    text = (ROOT / "include" / "circ.h").read_text()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(circ_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_four_calls():
+    names = declared_functions()
+    for must in ("circ_fc_create", "circ_fc_forward", "circ_conv_forward", "circ_destroy"):
+        assert must in names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    for name in declared_functions():
+        assert hasattr(lib, name), f"{name} declared in circ.h but not exported by libcirc.so"
+
+
+def test_binding_mirrors_header(lib):
+    from paper_1708_08917_b200 import binding
+    assert sorted(binding.SIGNATURES) == declared_functions()
+    for name in declared_functions():
+        assert callable(getattr(binding, name))
+
+
+def test_argument_errors_need_no_gpu(lib):
+    # shape / argument validation happens before any CUDA call
+    lib.circ_fc_create.restype = ctypes.c_void_p
+    lib.circ_last_error.restype = ctypes.c_char_p
+    buf = (ctypes.c_float * 64)()
+    assert lib.circ_fc_create(8, 8, 3, buf) is None and lib.circ_last_code() == -2       # k not a power of two
+    assert lib.circ_fc_create(8, 8, 512, buf) is None and lib.circ_last_code() == -2     # k out of range
+    assert lib.circ_fc_create(10, 8, 4, buf) is None and lib.circ_last_code() == -2      # k does not divide m
+    assert lib.circ_fc_create(8, 8, 4, None) is None and lib.circ_last_code() == -1      # NULL weights
+    assert b"k=" in lib.circ_last_error() or b"NULL" in lib.circ_last_error()
+    lib.circ_conv_create.restype = ctypes.c_void_p
+    assert lib.circ_conv_create(8, 8, 9, 1, 4, buf) is None and lib.circ_last_code() == -2
+    assert lib.circ_fc_forward(None, None, None, 1, None) == -1
+    assert lib.circ_set_activation(None, 1) == -1
+    lib.circ_destroy(None)                                                               # NULL is a no-op

@@ -1,0 +1,85 @@
+"""GPU parity: the CUDA fully-connected path against the fp64 dense oracle, element by element."""
+import numpy as np
+import pytest
+
+import paper_1708_08917_b200 as circ
+from paper_1708_08917_b200 import synth
+from gpu_helpers import TOL_BF16, TOL_F32, oracle_fc, run_fc, scale_rel_err
+
+pytestmark = pytest.mark.gpu
+
+VARIANTS = [circ.CIRC_VARIANT_STAGED]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_hand_cases_on_gpu(variant, golden_dir):
+    # the k=4 hand fixtures (k=2, 3 are below the library's block-size range)
+    w = np.array([1, 2, 3, 4], dtype=np.float32).reshape(1, 1, 4)
+    for conv, x, y in [(0, [1, 2, 3, 4], [26, 28, 26, 20]), (1, [1, 2, 3, 4], [30, 24, 22, 24]),
+                       (0, [0, 1, 0, 0], [4, 1, 2, 3]), (1, [0, 1, 0, 0], [2, 1, 4, 3])]:
+        case = synth.FcCase("hand", 4, 4, 4, 1, w, np.array([x], dtype=np.float32))
+        got, _ = run_fc(case, variant, convention=conv)
+        np.testing.assert_allclose(got[0], y, atol=1e-5)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("k", [4, 8, 16, 32, 64, 128, 256])
+@pytest.mark.parametrize("p,q,batch", [(1, 1, 1), (2, 3, 2), (3, 2, 3), (5, 7, 17), (3, 3, 64)])
+def test_small_shapes_all_block_sizes(variant, k, p, q, batch):
+    case = synth.fc_case(f"small_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
+                         bias_var=0.01, relu=(batch % 2 == 0))
+    got, used = run_fc(case, variant)
+    assert used == variant
+    assert not np.isnan(got).any()
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_convention_flag(variant):
+    case = synth.fc_case("conv_flag", 64, 96, 16, 3, w_var=0.01, x_dist="normal")
+    g0, _ = run_fc(case, variant, convention=0)
+    g1, _ = run_fc(case, variant, convention=1)
+    assert scale_rel_err(g0, oracle_fc(case, 0)) <= TOL_F32
+    assert scale_rel_err(g1, oracle_fc(case, 1)) <= TOL_F32
+    assert scale_rel_err(g0, oracle_fc(case, 1)) > 1e-2     # the flag is observable
+
+
+def test_config1():
+    case = synth.config1()
+    got, _ = run_fc(case)
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
+
+
+@pytest.mark.parametrize("batch", [1, 16, 256])
+def test_config2(batch):
+    case = synth.config2(batch)
+    got, _ = run_fc(case)
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
+
+
+def test_config3_stack():
+    layers = synth.config3_layers(128)
+    x = layers[0].x
+    for c in layers:
+        c.x = x
+        got, _ = run_fc(c)
+        ref = oracle_fc(c)
+        assert scale_rel_err(got, ref) <= TOL_F32
+        x = got.astype(np.float32)   # feed the GPU activations forward, as a real stack does
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("k,p,q,batch", [(16, 4, 4, 5), (64, 2, 2, 8), (4, 8, 8, 3)])
+def test_bf16_io(variant, k, p, q, batch):
+    case = synth.fc_case(f"bf16_{k}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="uniform", bf16_io=True)
+    got, _ = run_fc(case, variant)
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_BF16
+    got32, _ = run_fc(case, variant, y_bf16=False)     # bf16 in, float32 out: only the input was rounded
+    assert scale_rel_err(got32, oracle_fc(case)) <= TOL_F32
+
+
+def test_repeatable_bitwise():
+    case = synth.config2(16)
+    a, _ = run_fc(case)
+    b, _ = run_fc(case)
+    assert np.array_equal(a, b)
