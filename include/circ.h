@@ -108,6 +108,16 @@ CIRC_API circ_handle circ_conv_create(int c_out, int c_in, int r, int pad, int k
  */
 CIRC_API int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W, void* stream);
 
+/*
+ * circ_fc_forward_host / circ_conv_forward_host -- the same layers for callers whose tensors live
+ * in HOST memory (pinned memory makes the copies asynchronous).  Enqueues on `stream`: a
+ * host-to-device copy of x into a staging buffer owned by the handle, the forward pass, and a
+ * device-to-host copy of y.  y_host is valid after the stream has been synchronised.  The staging
+ * buffers grow on demand (cudaMalloc) and are reused by later calls.
+ */
+CIRC_API int circ_fc_forward_host(circ_handle h, const void* x_host, void* y_host, int batch, void* stream);
+CIRC_API int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int N, int H, int W, void* stream);
+
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);
 
@@ -141,6 +151,17 @@ CIRC_API long circ_workspace_bytes(circ_handle h);
 
 /* circ_last_variant -- the CIRC_VARIANT_* the most recent forward on this handle used. */
 CIRC_API int circ_last_variant(circ_handle h);
+
+/*
+ * circ_profile_begin / circ_profile_end -- per-kernel device times.  Between the two calls every
+ * kernel the handle launches is bracketed by CUDA events on its stream.  circ_profile_end waits
+ * for them and returns, per stage, the summed milliseconds and the number of launches:
+ *   stage 0 = input transforms, 1 = per-frequency contraction, 2 = inverse transforms + epilogue,
+ *   stage 3 = the fused one-launch kernel.  Both output arrays have 4 entries (HOST pointers).
+ * Profiling adds event records between kernels; do not time whole forwards while it is on.
+ */
+CIRC_API int circ_profile_begin(circ_handle h);
+CIRC_API int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage);
 
 /* circ_launch_count -- kernels this library has launched in this process so far. */
 CIRC_API long circ_launch_count(void);

@@ -27,6 +27,10 @@ SIGNATURES = {
     "circ_fc_forward": (_ci, [_vp, _vp, _vp, _ci, _vp]),
     "circ_conv_create": (_vp, [_ci, _ci, _ci, _ci, _ci, _vp]),
     "circ_conv_forward": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
+    "circ_fc_forward_host": (_ci, [_vp, _vp, _vp, _ci, _vp]),
+    "circ_conv_forward_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
+    "circ_profile_begin": (_ci, [_vp]),
+    "circ_profile_end": (_ci, [_vp, _vp, _vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
     "circ_set_activation": (_ci, [_vp, _ci]),
@@ -132,6 +136,27 @@ def circ_fc_forward(h: int, x, y, batch: int, stream=None) -> None:
 def circ_conv_forward(h: int, x, y, N: int, H: int, W: int, stream=None) -> None:
     """Enqueue the channel-last convolution ``x[N][H][W][C] -> y[N][Ho][Wo][P]``."""
     _check(load().circ_conv_forward(h, _ptr(x), _ptr(y), N, H, W, _stream(stream)))
+
+
+def circ_fc_forward_host(h: int, x_host, y_host, batch: int, stream=None) -> None:
+    """Host-memory variant: ``x_host`` / ``y_host`` are (pinned) CPU tensors, numpy arrays or addresses."""
+    _check(load().circ_fc_forward_host(h, _ptr(x_host), _ptr(y_host), batch, _stream(stream)))
+
+
+def circ_conv_forward_host(h: int, x_host, y_host, N: int, H: int, W: int, stream=None) -> None:
+    _check(load().circ_conv_forward_host(h, _ptr(x_host), _ptr(y_host), N, H, W, _stream(stream)))
+
+
+def circ_profile_begin(h: int) -> None:
+    _check(load().circ_profile_begin(h))
+
+
+def circ_profile_end(h: int):
+    """Returns (ms_by_stage[4], launches_by_stage[4]) as Python lists."""
+    ms = (ctypes.c_float * 4)()
+    cnt = (ctypes.c_int * 4)()
+    _check(load().circ_profile_end(h, ctypes.addressof(ms), ctypes.addressof(cnt)))
+    return list(ms), list(cnt)
 
 
 def circ_destroy(h: int | None) -> None:

@@ -6,6 +6,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "circ_common.cuh"
 
@@ -24,6 +25,34 @@ void set_error(int code, const char* fmt, ...) {
     if (getenv("CIRC_LOG")) fprintf(stderr, "[circ] error %d: %s\n", code, g_err);
 }
 void count_launches(long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Optional per-kernel device timing (circ_profile_begin / circ_profile_end).
+struct ProfRec {
+    cudaEvent_t start, stop;
+    int stage;
+};
+struct Profiler {
+    std::vector<ProfRec> recs;
+};
+struct StageTimer {
+    Profiler* prof;
+    cudaStream_t stream;
+    ProfRec rec;
+    StageTimer(Layer* L, int stage, cudaStream_t s) : prof(static_cast<Profiler*>(L->prof)), stream(s) {
+        if (!prof) return;
+        rec.stage = stage;
+        if (cudaEventCreate(&rec.start) != cudaSuccess || cudaEventCreate(&rec.stop) != cudaSuccess) {
+            prof = nullptr;
+            return;
+        }
+        cudaEventRecord(rec.start, stream);
+    }
+    ~StageTimer() {
+        if (!prof) return;
+        cudaEventRecord(rec.stop, stream);
+        prof->recs.push_back(rec);
+    }
+};
 
 static bool pow2_in_range(int k) { return k >= 4 && k <= 256 && (k & (k - 1)) == 0; }
 
@@ -59,6 +88,15 @@ static void free_layer(Layer* L) {
     cudaFree(L->a_bf16);
     cudaFree(L->ws);
     cudaFree(L->dev_status);
+    cudaFree(L->x_stage);
+    cudaFree(L->y_stage);
+    if (L->prof) {
+        for (auto& r : static_cast<Profiler*>(L->prof)->recs) {
+            cudaEventDestroy(r.start);
+            cudaEventDestroy(r.stop);
+        }
+        delete static_cast<Profiler*>(L->prof);
+    }
     if (prev != L->device && prev >= 0) cudaSetDevice(prev);
     delete L;
 }
@@ -197,9 +235,18 @@ static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStr
     if (rc != CIRC_OK) return rc;
     float* xop = static_cast<float*>(L->ws);
     float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
-    if ((rc = launch_input_fft(L, x, xop, e, stream)) != CIRC_OK) return rc;
-    if ((rc = launch_contract_fma(L, xop, yop, e, stream)) != CIRC_OK) return rc;
-    if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
+    {
+        StageTimer t(L, 0, stream);
+        if ((rc = launch_input_fft(L, x, xop, e, stream)) != CIRC_OK) return rc;
+    }
+    {
+        StageTimer t(L, 1, stream);
+        if ((rc = launch_contract_fma(L, xop, yop, e, stream)) != CIRC_OK) return rc;
+    }
+    {
+        StageTimer t(L, 2, stream);
+        if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
+    }
     L->last_variant = CIRC_VARIANT_STAGED;
     return CIRC_OK;
 }
@@ -244,7 +291,10 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
             set_error(CIRC_ERR_UNSUPPORTED, "the fused kernel does not serve batch=%d for this layer", batch);
             return CIRC_ERR_UNSUPPORTED;
         }
-        rc = launch_fused_fc(L, x, y, batch, s);
+        {
+            StageTimer t(L, 3, s);
+            rc = launch_fused_fc(L, x, y, batch, s);
+        }
         if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
         return rc;
     }
@@ -276,6 +326,115 @@ int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W
         return CIRC_ERR_UNSUPPORTED;
     }
     return run_staged(L, x, y, conv_extent(L, N, H, W), static_cast<cudaStream_t>(stream));
+}
+
+// Grow the device staging buffers of the host-pointer entry points.
+static int ensure_stage(Layer* L, size_t xbytes, size_t ybytes) {
+    if (L->x_stage_bytes < xbytes) {
+        cudaFree(L->x_stage);
+        L->x_stage = nullptr;
+        L->x_stage_bytes = 0;
+        if (cudaMalloc(&L->x_stage, xbytes) != cudaSuccess) {
+            cudaGetLastError();
+            set_error(CIRC_ERR_ALLOC, "staging allocation of %zu bytes failed", xbytes);
+            return CIRC_ERR_ALLOC;
+        }
+        L->x_stage_bytes = xbytes;
+    }
+    if (L->y_stage_bytes < ybytes) {
+        cudaFree(L->y_stage);
+        L->y_stage = nullptr;
+        L->y_stage_bytes = 0;
+        if (cudaMalloc(&L->y_stage, ybytes) != cudaSuccess) {
+            cudaGetLastError();
+            set_error(CIRC_ERR_ALLOC, "staging allocation of %zu bytes failed", ybytes);
+            return CIRC_ERR_ALLOC;
+        }
+        L->y_stage_bytes = ybytes;
+    }
+    return CIRC_OK;
+}
+
+int circ_fc_forward_host(circ_handle h, const void* x_host, void* y_host, int batch, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || !x_host || !y_host || L->kind != 0 || batch < 1) {
+        set_error(CIRC_ERR_ARG, "bad handle, NULL host pointer or batch < 1");
+        return CIRC_ERR_ARG;
+    }
+    const size_t xb = (size_t)batch * L->n * (L->x_dtype == CIRC_BF16 ? 2 : 4);
+    const size_t yb = (size_t)batch * L->m * (L->y_dtype == CIRC_BF16 ? 2 : 4);
+    int rc = ensure_stage(L, xb, yb);
+    if (rc != CIRC_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CIRC_CUDA_TRY(cudaMemcpyAsync(L->x_stage, x_host, xb, cudaMemcpyHostToDevice, s), CIRC_ERR_CUDA);
+    if ((rc = circ_fc_forward(h, L->x_stage, L->y_stage, batch, stream)) != CIRC_OK) return rc;
+    CIRC_CUDA_TRY(cudaMemcpyAsync(y_host, L->y_stage, yb, cudaMemcpyDeviceToHost, s), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int N, int H, int W, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || !x_host || !y_host || L->kind != 1 || N < 1 || H < 1 || W < 1) {
+        set_error(CIRC_ERR_ARG, "bad handle, NULL host pointer or empty image");
+        return CIRC_ERR_ARG;
+    }
+    const int Ho = H + 2 * L->geo.pad - L->geo.r + 1, Wo = W + 2 * L->geo.pad - L->geo.r + 1;
+    if (Ho < 1 || Wo < 1) {
+        set_error(CIRC_ERR_SHAPE, "image smaller than the filter");
+        return CIRC_ERR_SHAPE;
+    }
+    const size_t xb = (size_t)N * H * W * L->n * (L->x_dtype == CIRC_BF16 ? 2 : 4);
+    const size_t yb = (size_t)N * Ho * Wo * L->m * (L->y_dtype == CIRC_BF16 ? 2 : 4);
+    int rc = ensure_stage(L, xb, yb);
+    if (rc != CIRC_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CIRC_CUDA_TRY(cudaMemcpyAsync(L->x_stage, x_host, xb, cudaMemcpyHostToDevice, s), CIRC_ERR_CUDA);
+    if ((rc = circ_conv_forward(h, L->x_stage, L->y_stage, N, H, W, stream)) != CIRC_OK) return rc;
+    CIRC_CUDA_TRY(cudaMemcpyAsync(y_host, L->y_stage, yb, cudaMemcpyDeviceToHost, s), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int circ_profile_begin(circ_handle h) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L) {
+        set_error(CIRC_ERR_ARG, "handle is NULL");
+        return CIRC_ERR_ARG;
+    }
+    if (!L->prof) L->prof = new (std::nothrow) Profiler();
+    if (!L->prof) {
+        set_error(CIRC_ERR_ALLOC, "host allocation failed");
+        return CIRC_ERR_ALLOC;
+    }
+    return CIRC_OK;
+}
+
+int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || !L->prof || !ms_by_stage || !launches_by_stage) {
+        set_error(CIRC_ERR_ARG, "bad handle / profiling not started / NULL output");
+        return CIRC_ERR_ARG;
+    }
+    Profiler* P = static_cast<Profiler*>(L->prof);
+    for (int s = 0; s < 4; ++s) {
+        ms_by_stage[s] = 0.f;
+        launches_by_stage[s] = 0;
+    }
+    int rc = CIRC_OK;
+    for (auto& r : P->recs) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) {
+            set_error(CIRC_ERR_CUDA, "event timing failed: %s", cudaGetErrorString(cudaGetLastError()));
+            rc = CIRC_ERR_CUDA;
+        } else if (r.stage >= 0 && r.stage < 4) {
+            ms_by_stage[r.stage] += ms;
+            launches_by_stage[r.stage] += 1;
+        }
+        cudaEventDestroy(r.start);
+        cudaEventDestroy(r.stop);
+    }
+    delete P;
+    L->prof = nullptr;
+    return rc;
 }
 
 int circ_set_bias(circ_handle h, const float* bias) {

@@ -88,6 +88,10 @@ struct Layer {
     void* ws;           // workspace: frequency-domain operands X and Y
     size_t ws_bytes;
     int* dev_status;    // device error word (bounded waits report here)
+    void* x_stage;      // device staging buffers of the host-pointer entry points
+    void* y_stage;
+    size_t x_stage_bytes, y_stage_bytes;
+    void* prof;         // per-kernel timing records while profiling is on, else nullptr
 };
 
 // Thread-local error record.

@@ -8,7 +8,7 @@ from gpu_helpers import TOL_BF16, TOL_F32, oracle_fc, run_fc, scale_rel_err
 
 pytestmark = pytest.mark.gpu
 
-VARIANTS = [circ.CIRC_VARIANT_STAGED]
+VARIANTS = [circ.CIRC_VARIANT_STAGED, circ.CIRC_VARIANT_FUSED]
 
 
 @pytest.mark.parametrize("variant", VARIANTS)
@@ -24,10 +24,15 @@ def test_hand_cases_on_gpu(variant, golden_dir):
 
 @pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("k", [4, 8, 16, 32, 64, 128, 256])
-@pytest.mark.parametrize("p,q,batch", [(1, 1, 1), (2, 3, 2), (3, 2, 3), (5, 7, 17), (3, 3, 64)])
+@pytest.mark.parametrize("p,q,batch", [(1, 1, 1), (2, 3, 2), (3, 2, 3), (5, 7, 17), (3, 3, 64), (9, 11, 8), (40, 3, 5)])
 def test_small_shapes_all_block_sizes(variant, k, p, q, batch):
     case = synth.fc_case(f"small_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
                          bias_var=0.01, relu=(batch % 2 == 0))
+    if variant == circ.CIRC_VARIANT_FUSED and batch > 8:
+        with pytest.raises(circ.CircError) as err:      # the one-launch kernel serves batch <= 8 only
+            run_fc(case, variant)
+        assert err.value.code == circ.CIRC_ERR_UNSUPPORTED
+        return
     got, used = run_fc(case, variant)
     assert used == variant
     assert not np.isnan(got).any()
@@ -53,7 +58,17 @@ def test_config1():
 @pytest.mark.parametrize("batch", [1, 16, 256])
 def test_config2(batch):
     case = synth.config2(batch)
-    got, _ = run_fc(case)
+    got, used = run_fc(case)
+    assert used == (circ.CIRC_VARIANT_FUSED if batch == 1 else used)
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("batch", [1, 2, 7, 8])
+def test_config2_small_batches_both_variants(variant, batch):
+    case = synth.config2(batch)
+    got, used = run_fc(case, variant)
+    assert used == variant
     assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
 
 
