@@ -163,6 +163,11 @@ CIRC_API int circ_last_variant(circ_handle h);
 CIRC_API int circ_profile_begin(circ_handle h);
 CIRC_API int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage);
 
+/* circ_device_status -- waits for the device (blocking copy of the handle's error word) and
+ * returns CIRC_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up on a bounded wait (TMA /
+ * tensor-core pipeline barriers) since the last call; the word is cleared.  CIRC_OK otherwise. */
+CIRC_API int circ_device_status(circ_handle h);
+
 /* circ_launch_count -- kernels this library has launched in this process so far. */
 CIRC_API long circ_launch_count(void);
 

@@ -31,6 +31,7 @@ SIGNATURES = {
     "circ_conv_forward_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_profile_begin": (_ci, [_vp]),
     "circ_profile_end": (_ci, [_vp, _vp, _vp]),
+    "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
     "circ_set_activation": (_ci, [_vp, _ci]),
@@ -157,6 +158,11 @@ def circ_profile_end(h: int):
     cnt = (ctypes.c_int * 4)()
     _check(load().circ_profile_end(h, ctypes.addressof(ms), ctypes.addressof(cnt)))
     return list(ms), list(cnt)
+
+
+def circ_device_status(h: int) -> None:
+    """Blocks until the device is idle; raises CircError(CIRC_ERR_DEVICE_TIMEOUT) if a bounded wait expired."""
+    _check(load().circ_device_status(h))
 
 
 def circ_destroy(h: int | None) -> None:

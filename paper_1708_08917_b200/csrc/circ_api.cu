@@ -149,6 +149,7 @@ static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad
     const size_t a_real = (size_t)taps * (m / k) * (n / k);
     L->a_elems = 2 * a_real + (size_t)(k / 2 - 1) * 4 * a_real;
     bool ok = cudaMalloc(&L->tw256, sizeof(host_tw)) == cudaSuccess &&
+              cudaMalloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
               cudaMalloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&L->dev_status, sizeof(int)) == cudaSuccess;
@@ -230,24 +231,30 @@ static int check_io(const Layer* L, const void* x, const void* y) {
     return CIRC_OK;
 }
 
-static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream) {
+static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
     int rc = ensure_workspace(L, workspace_need(L, e));
     if (rc != CIRC_OK) return rc;
     float* xop = static_cast<float*>(L->ws);
     float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
     {
         StageTimer t(L, 0, stream);
-        if ((rc = launch_input_fft(L, x, xop, e, stream)) != CIRC_OK) return rc;
+        // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16
+        const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
+        if ((rc = launch_input_fft(L, x, xop, xmode, e, stream)) != CIRC_OK) return rc;
     }
     {
         StageTimer t(L, 1, stream);
-        if ((rc = launch_contract_fma(L, xop, yop, e, stream)) != CIRC_OK) return rc;
+        if (tensor)
+            rc = launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
+        else
+            rc = launch_contract_fma(L, xop, yop, e, stream);
+        if (rc != CIRC_OK) return rc;
     }
     {
         StageTimer t(L, 2, stream);
         if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
     }
-    L->last_variant = CIRC_VARIANT_STAGED;
+    L->last_variant = tensor ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
     return CIRC_OK;
 }
 
@@ -285,7 +292,10 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int variant = L->variant;
-    if (variant == CIRC_VARIANT_AUTO) variant = fused_fc_supported(L, batch) && batch <= 8 ? CIRC_VARIANT_FUSED : CIRC_VARIANT_STAGED;
+    if (variant == CIRC_VARIANT_AUTO)
+        variant = fused_fc_supported(L, batch) && batch <= 8 ? CIRC_VARIANT_FUSED
+                  : (tensor_supported(L) && batch >= 32)      ? CIRC_VARIANT_TENSOR
+                                                              : CIRC_VARIANT_STAGED;
     if (variant == CIRC_VARIANT_FUSED) {
         if (!fused_fc_supported(L, batch)) {
             set_error(CIRC_ERR_UNSUPPORTED, "the fused kernel does not serve batch=%d for this layer", batch);
@@ -298,11 +308,11 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
         if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
         return rc;
     }
-    if (variant == CIRC_VARIANT_TENSOR) {
-        set_error(CIRC_ERR_UNSUPPORTED, "tensor-core contraction not available in this build");
+    if (variant == CIRC_VARIANT_TENSOR && !tensor_supported(L)) {
+        set_error(CIRC_ERR_UNSUPPORTED, "the tensor-core contraction needs q = n/k to be a multiple of 8 (q=%d)", L->geo.q);
         return CIRC_ERR_UNSUPPORTED;
     }
-    return run_staged(L, x, y, fc_extent(batch), s);
+    return run_staged(L, x, y, fc_extent(batch), s, variant == CIRC_VARIANT_TENSOR);
 }
 
 int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W, void* stream) {
@@ -321,11 +331,12 @@ int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W
         set_error(CIRC_ERR_SHAPE, "N*H*W too large");
         return CIRC_ERR_SHAPE;
     }
-    if (L->variant == CIRC_VARIANT_FUSED || L->variant == CIRC_VARIANT_TENSOR) {
-        set_error(CIRC_ERR_UNSUPPORTED, "variant %d not available for convolutions in this build", L->variant);
+    if (L->variant == CIRC_VARIANT_FUSED || (L->variant == CIRC_VARIANT_TENSOR && !tensor_supported(L))) {
+        set_error(CIRC_ERR_UNSUPPORTED, "variant %d not available for this convolution", L->variant);
         return CIRC_ERR_UNSUPPORTED;
     }
-    return run_staged(L, x, y, conv_extent(L, N, H, W), static_cast<cudaStream_t>(stream));
+    const bool tensor = L->variant == CIRC_VARIANT_TENSOR || (L->variant == CIRC_VARIANT_AUTO && tensor_supported(L));
+    return run_staged(L, x, y, conv_extent(L, N, H, W), static_cast<cudaStream_t>(stream), tensor);
 }
 
 // Grow the device staging buffers of the host-pointer entry points.
@@ -435,6 +446,22 @@ int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage) 
     delete P;
     L->prof = nullptr;
     return rc;
+}
+
+int circ_device_status(circ_handle h) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L) {
+        set_error(CIRC_ERR_ARG, "handle is NULL");
+        return CIRC_ERR_ARG;
+    }
+    int word = 0;
+    CIRC_CUDA_TRY(cudaMemcpy(&word, L->dev_status, sizeof(int), cudaMemcpyDeviceToHost), CIRC_ERR_CUDA);
+    if (word != 0) {
+        cudaMemset(L->dev_status, 0, sizeof(int));
+        set_error(CIRC_ERR_DEVICE_TIMEOUT, "a bounded device-side wait expired (code %d); the output of that forward is invalid", word);
+        return CIRC_ERR_DEVICE_TIMEOUT;
+    }
+    return CIRC_OK;
 }
 
 int circ_set_bias(circ_handle h, const float* bias) {

@@ -114,11 +114,16 @@ void count_launches(long n);
 // S0: spectra of the defining vectors, in every stored layout.
 int launch_precompute(Layer* L, cudaStream_t stream);
 
-// S1 / C1: forward transforms of the input -> operand X (float32, layout above).
-int launch_input_fft(const Layer* L, const void* x, float* xop, const Extent& ext, cudaStream_t stream);
+// S1 / C1: forward transforms of the input -> operand X.  xmode 0: float32 [problem][col][Kq];
+// 1: bfloat16 [problem][col][hi | lo][Kq] (split of float32 values); 2: bfloat16 [problem][col][Kq].
+int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream);
 
 // S2 / C2 on the float32 FMA pipes: Y = A . X per problem.
 int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream);
+
+// S2 / C2 on the tensor cores (bfloat16 operands from xmode 1 or 2, float32 accumulate).
+int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream);
+bool tensor_supported(const Layer* L);
 
 // S3 / C3: inverse transforms + bias + activation -> y.
 int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);

@@ -14,9 +14,9 @@ constexpr int kThreads = 256;
 
 // ---- S1: x -> operand X ------------------------------------------------------------------------
 // One transform = (pair c, column block j).  A CTA takes TT = 256 / L consecutive transforms.
-template <int K, typename TIN>
+template <int K, typename TIN, int XMODE>
 __global__ void __launch_bounds__(kThreads)
-input_fft_kernel(const TIN* __restrict__ x, float* __restrict__ xop, const float2* __restrict__ tw256, int n, int q,
+input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2* __restrict__ tw256, int n, int q,
                  int B, int Bh, long total) {
     constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = kThreads / L;
     __shared__ float2 tw[K];
@@ -55,23 +55,35 @@ input_fft_kernel(const TIN* __restrict__ x, float* __restrict__ xop, const float
     if (T2 >= total) return;
     const int c = (int)(T2 / q), j = (int)(T2 % q);
     const size_t cols = 2 * (size_t)Bh;
-    const size_t real_sz = cols * q, cplx_sz = 2 * real_sz;
+    // XMODE 0: float32 operand [problem][col][Kq]; 1 / 2: bfloat16 operand [problem][col][part][Kq]
+    // with parts (hi, lo) / (hi) for the tensor-core contraction.
+    constexpr int NPART = XMODE == 1 ? 2 : 1;
+    const size_t real_sz = cols * q * NPART, cplx_sz = 2 * real_sz;
+    auto put = [&](int prob, size_t col, int kq, int kk, float val) {
+        const size_t at = problem_offset(prob, real_sz, cplx_sz) + col * (size_t)(NPART * kq) + kk;
+        if constexpr (XMODE == 0) {
+            static_cast<float*>(xop)[at] = val;
+        } else {
+            __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(xop);
+            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
+            xb[at] = hi;
+            if constexpr (XMODE == 1) xb[at + kq] = __float2bfloat16_rn(val - __bfloat162float(hi));
+        }
+    };
 #pragma unroll
     for (int it = 0; it < E; ++it) {
         const int f = f0 + L * it;
         const float2 z = zs[tl][f];
         if (f == 0 || f == K / 2) {
-            float* xg = xop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-            xg[(size_t)c * q + j] = z.x;
-            xg[((size_t)Bh + c) * q + j] = z.y;
+            const int prob = f == 0 ? 0 : 1;
+            put(prob, (size_t)c, q, j, z.x);
+            put(prob, (size_t)Bh + c, q, j, z.y);
         } else if (f < K / 2) {
-            float* xg = xop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * q;
-            xg[j] = z.x;
-            xg[q + j] = z.y;
+            put(f + 1, (size_t)c, 2 * q, j, z.x);
+            put(f + 1, (size_t)c, 2 * q, q + j, z.y);
         } else {
-            float* xg = xop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bh + c) * 2 * q;
-            xg[j] = z.x;
-            xg[q + j] = -z.y;
+            put(K - f + 1, (size_t)Bh + c, 2 * q, j, z.x);
+            put(K - f + 1, (size_t)Bh + c, 2 * q, q + j, -z.y);
         }
     }
 }
@@ -159,19 +171,27 @@ static int dispatch_k(int k, F&& f) {
     return CIRC_ERR_SHAPE;
 }
 
-int launch_input_fft(const Layer* L, const void* x, float* xop, const Extent& ext, cudaStream_t stream) {
+int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream) {
     const int q = L->geo.q, n = L->n;
     const long total = (long)ext.Bh * q;
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
         constexpr int TT = kThreads / FftShape<K>::L;
         const unsigned blocks = (unsigned)((total + TT - 1) / TT);
-        if (L->x_dtype == CIRC_BF16)
-            input_fft_kernel<K, __nv_bfloat16><<<blocks, kThreads, 0, stream>>>(
-                static_cast<const __nv_bfloat16*>(x), xop, L->tw256, n, q, ext.B, ext.Bh, total);
-        else
-            input_fft_kernel<K, float><<<blocks, kThreads, 0, stream>>>(static_cast<const float*>(x), xop, L->tw256, n, q,
-                                                                        ext.B, ext.Bh, total);
+        auto launch = [&](auto tin, auto mode) {
+            using TIN = decltype(tin);
+            constexpr int XMODE = decltype(mode)::value;
+            input_fft_kernel<K, TIN, XMODE><<<blocks, kThreads, 0, stream>>>(static_cast<const TIN*>(x), xop, L->tw256, n, q,
+                                                                            ext.B, ext.Bh, total);
+        };
+        const bool bf = L->x_dtype == CIRC_BF16;
+        if (xmode == 0) {
+            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 0>{}); else launch(float{}, std::integral_constant<int, 0>{});
+        } else if (xmode == 1) {
+            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 1>{}); else launch(float{}, std::integral_constant<int, 1>{});
+        } else {
+            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 2>{}); else launch(float{}, std::integral_constant<int, 2>{});
+        }
         return CIRC_OK;
     };
     const int rc = dispatch_k<void>(L->geo.k, go);

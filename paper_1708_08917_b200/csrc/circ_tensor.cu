@@ -1,0 +1,423 @@
+// S2 / C2 on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor memory).
+//
+// For every frequency problem (circ_common.cuh) the contraction
+//     Y[col][row] = sum_{tap, kk} A[row][tap][kk] * X[col shifted by tap][kk]
+// is a dense product once the batch (or the pixel count) is large.  One CTA computes one
+// 128-column x BN-row output tile:
+//   * the 128 batch columns / output pixels are the MMA's M dimension (TMEM lanes),
+//     the weight rows are its N dimension (TMEM columns), the contraction index is K;
+//   * operands are bfloat16, K-major, fetched by TMA (cp.async.bulk.tensor, 128-byte swizzle,
+//     no multicast) into a ring of shared-memory stages guarded by mbarriers;
+//   * a convolution tap is just a shifted TMA box over the (W, H, image) dimensions of X:
+//     out-of-image pixels are the zero fill of the copy (Eq. 6 with zero padding);
+//   * float32 inputs use the split  a = a_hi + a_lo  (two bfloat16 values, 16 mantissa bits):
+//     the three products hi*hi + lo*hi + hi*lo are three passes over the same K range into
+//     the same float32 accumulator; bfloat16 inputs take the single hi*hi pass.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue
+// (tcgen05.ld -> registers -> global).  Every wait is bounded: on expiry the CTA records an error
+// word, drains its copies, frees its tensor memory and returns.
+#include <cuda.h>
+
+#include "circ_common.cuh"
+
+namespace circ {
+
+constexpr int kTcThreads = 192;
+constexpr int kTileCols = 128;            // MMA M: batch columns / pixels per tile
+constexpr int kKBlock = 64;               // bf16 elements per stage along K (one 128-byte swizzle row)
+constexpr int kStages = 4;
+constexpr uint32_t kSpinLimit = 1u << 22; // bounded wait: polls before giving up
+
+struct TcArgs {
+    float* yop;
+    int* status;
+    int p, q, k, taps, r, pad;
+    int nsplit;              // parts of X per column: 2 (hi, lo) or 1
+    int npass;               // 3 (float32 inputs) or 1 (bfloat16 inputs)
+    int W, H, V;             // input image (FC: W = columns, H = V = 1)
+    int Wo, Ho;              // output image
+    int tw, th;              // spatial tile (tw * th <= 128)
+    int tiles_w, tiles_h;    // tiles per image
+    int bn_real, bn_cplx;    // rows per tile (multiple of 16, <= 256)
+    int nt_real, nt_cplx;    // row tiles per problem
+    int ctas_real;           // CTAs that serve the two real problems
+    long cols_out;           // V * Ho * Wo
+};
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (it > 64) __nanosleep(64);
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3,
+                                            int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
+// 128-byte swizzle (what the TMA copy writes): 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version (sm_100)
+    d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M = 128, N = bn.
+__device__ __forceinline__ uint32_t instr_desc(int bn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_constant__ CUtensorMap map_a_cplx,
+                   const __grid_constant__ CUtensorMap map_xhi_real, const __grid_constant__ CUtensorMap map_xlo_real,
+                   const __grid_constant__ CUtensorMap map_xhi_cplx, const __grid_constant__ CUtensorMap map_xlo_cplx,
+                   TcArgs g) {
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], accum_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- which tile ---------------------------------------------------------------------------
+    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
+    int cta = blockIdx.x;
+    const bool real = cta < g.ctas_real;
+    int prob_in_kind, row_tile;
+    if (real) {
+        prob_in_kind = cta / (g.nt_real * sp_tiles);
+        cta -= prob_in_kind * g.nt_real * sp_tiles;
+        row_tile = cta / sp_tiles;
+        cta -= row_tile * sp_tiles;
+    } else {
+        cta -= g.ctas_real;
+        prob_in_kind = cta / (g.nt_cplx * sp_tiles);
+        cta -= prob_in_kind * g.nt_cplx * sp_tiles;
+        row_tile = cta / sp_tiles;
+        cta -= row_tile * sp_tiles;
+    }
+    const int v = cta / (g.tiles_h * g.tiles_w);
+    const int th_i = (cta / g.tiles_w) % g.tiles_h, tw_i = cta % g.tiles_w;
+    const int ho0 = th_i * g.th, wo0 = tw_i * g.tw;
+    const int bn = real ? g.bn_real : g.bn_cplx;
+    const int Mg = real ? g.p : 2 * g.p;
+    const int Kq = real ? g.q : 2 * g.q;
+    const int row0 = row_tile * bn;
+    const int prob = real ? prob_in_kind : 2 + prob_in_kind;
+    const CUtensorMap* map_a = real ? &map_a_real : &map_a_cplx;
+    const CUtensorMap* map_xhi = real ? &map_xhi_real : &map_xhi_cplx;
+    const CUtensorMap* map_xlo = real ? &map_xlo_real : &map_xlo_cplx;
+
+    // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes)
+    const uint32_t x_bytes = kTileCols * 128, a_bytes = (uint32_t)bn * 128;
+    const uint32_t stage_bytes = x_bytes + a_bytes;
+    unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
+    const uint32_t tx_bytes = (uint32_t)(g.tw * g.th) * 128 + a_bytes;
+
+    const int kblocks = (Kq + kKBlock - 1) / kKBlock;
+    const int iters = g.npass * g.taps * kblocks;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < bn) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&tmem_base_slot, tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    if (warp == 0) {
+        // ---- TMA producer -----------------------------------------------------------------------
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % kStages, round = it / kStages;
+                if (round > 0) ok = mbar_wait(&empty_bar[s], (round - 1) & 1, &abort_flag);
+                if (!ok) break;
+                const int kb = it % kblocks;
+                const int tap = (it / kblocks) % g.taps;
+                const int pass = it / (kblocks * g.taps);
+                const int a_part = pass == 1 ? 1 : 0, x_lo = pass == 2;
+                const int di = tap / g.r - g.pad, dj = tap % g.r - g.pad;
+                unsigned char* xs = ring + (size_t)s * stage_bytes;
+                unsigned char* as = xs + x_bytes;
+                mbar_expect_tx(&full_bar[s], tx_bytes);
+                tma_load_5d(xs, x_lo ? map_xlo : map_xhi, &full_bar[s], kb * kKBlock, wo0 + dj, ho0 + di, v, prob_in_kind);
+                tma_load_4d(as, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, row0, prob_in_kind);
+                ++issued;
+            }
+            if (!ok) {
+                // drain: every copy that was issued must land before the CTA may go away
+                const int first = issued > kStages ? issued - kStages : 0;
+                for (int it = first; it < issued; ++it) {
+                    const int s = it % kStages, round = it / kStages;
+                    for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&full_bar[s], round & 1); ++spin) __nanosleep(64);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer -------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(bn);
+            bool ok = true;
+            for (int it = 0; it < iters && ok; ++it) {
+                const int s = it % kStages, round = it / kStages;
+                ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
+                const uint64_t da = smem_desc_sw128(xs), db = smem_desc_sw128(xs + x_bytes);
+#pragma unroll
+                for (int k4 = 0; k4 < kKBlock / 16; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
+                    tc_mma_bf16(tmem_base, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
+            }
+            if (ok) tc_commit(&accum_bar);  // accumulator complete
+        }
+    } else {
+        // ---- epilogue: TMEM -> registers -> Y[col][row] ------------------------------------------
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag));  // warp-uniform
+        tc_fence_after();
+        if (ok) {
+            const int quarter = warp & 3;                 // a warp may only read its own 32 TMEM lanes
+            const int r = quarter * 32 + lane;            // row of the tile = pixel within the spatial tile
+            const int hh = r / g.tw, ww = r - hh * g.tw;
+            const int ho = ho0 + hh, wo = wo0 + ww;
+            const bool live = r < g.tw * g.th && ho < g.Ho && wo < g.Wo;
+            const size_t y_real = (size_t)g.cols_out * g.p;
+            float* yrow = g.yop + problem_offset(prob, y_real, 2 * y_real) +
+                          ((size_t)((size_t)v * g.Ho + ho) * g.Wo + wo) * Mg + row0;
+            for (int c0 = 0; c0 < bn; c0 += 32) {
+                uint32_t acc[32];
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, acc);
+                if (live) {
+                    if (row0 + c0 + 32 <= Mg && (Mg & 3) == 0) {
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4)
+                            *reinterpret_cast<float4*>(yrow + c0 + e) =
+                                make_float4(__uint_as_float(acc[e]), __uint_as_float(acc[e + 1]), __uint_as_float(acc[e + 2]),
+                                            __uint_as_float(acc[e + 3]));
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (row0 + c0 + e < Mg) yrow[c0 + e] = __uint_as_float(acc[e]);
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ---------------------------------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, tmem_cols);
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(g.status, 1);
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
+                  const cuuint32_t* box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) {
+        set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        return CIRC_ERR_CUDA;
+    }
+    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, dims, strides_bytes, box, ones,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+        return CIRC_ERR_CUDA;
+    }
+    return CIRC_OK;
+}
+
+static int round_up16(int v) { return (v + 15) & ~15; }
+
+bool tensor_supported(const Layer* L) { return L->a_bf16 != nullptr && (L->geo.q % 8) == 0 && encode_fn() != nullptr; }
+
+int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream) {
+    const Geometry& geo = L->geo;
+    const int p = geo.p, q = geo.q, k = geo.k, taps = geo.taps;
+    TcArgs g;
+    g.yop = yop;
+    g.status = L->dev_status;
+    g.p = p; g.q = q; g.k = k; g.taps = taps; g.r = geo.r; g.pad = geo.pad;
+    g.nsplit = nsplit;
+    g.npass = nsplit == 2 ? 3 : 1;
+    if (L->kind == 1) {
+        g.W = ext.W; g.H = ext.H; g.V = 2 * ext.Nh; g.Wo = ext.Wo; g.Ho = ext.Ho;
+    } else {
+        g.W = g.Wo = 2 * ext.Bh; g.H = g.Ho = 1; g.V = 1;
+    }
+    g.tw = g.Wo < kTileCols ? g.Wo : kTileCols;
+    g.th = kTileCols / g.tw;
+    if (g.th > g.Ho) g.th = g.Ho;
+    g.tiles_w = (g.Wo + g.tw - 1) / g.tw;
+    g.tiles_h = (g.Ho + g.th - 1) / g.th;
+    g.bn_real = round_up16(p) > 256 ? 256 : round_up16(p);
+    g.bn_cplx = round_up16(2 * p) > 256 ? 256 : round_up16(2 * p);
+    g.nt_real = (p + g.bn_real - 1) / g.bn_real;
+    g.nt_cplx = (2 * p + g.bn_cplx - 1) / g.bn_cplx;
+    g.cols_out = (long)g.V * g.Ho * g.Wo;
+    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
+    g.ctas_real = 2 * g.nt_real * sp_tiles;
+    const long ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles;
+
+    // tensor maps.  A: [problem][row][part = tap*2 + (hi|lo)][Kq]
+    CUtensorMap ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c;
+    const size_t a_real_elems = (size_t)p * taps * 2 * q;  // one real problem of A (hi and lo)
+    int rc;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)q, (cuuint64_t)taps * 2, (cuuint64_t)p, 2};
+        cuuint64_t str[3] = {(cuuint64_t)q * 2, (cuuint64_t)taps * 2 * q * 2, (cuuint64_t)a_real_elems * 2};
+        cuuint32_t box[4] = {kKBlock, 1, (cuuint32_t)g.bn_real, 1};
+        if ((rc = encode(&ma_r, L->a_bf16, 4, dims, str, box)) != CIRC_OK) return rc;
+    }
+    {
+        const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
+        cuuint64_t dims[4] = {(cuuint64_t)2 * q, (cuuint64_t)taps * 2, (cuuint64_t)2 * p, (cuuint64_t)nc};
+        cuuint64_t str[3] = {(cuuint64_t)2 * q * 2, (cuuint64_t)taps * 2 * 2 * q * 2, (cuuint64_t)4 * a_real_elems * 2};
+        cuuint32_t box[4] = {kKBlock, 1, (cuuint32_t)g.bn_cplx, 1};
+        if ((rc = encode(&ma_c, L->a_bf16 + 2 * a_real_elems, 4, dims, str, box)) != CIRC_OK) return rc;
+    }
+    // X: [problem][v][h][w][part][Kq]
+    const size_t cols_in = (size_t)g.V * g.H * g.W;
+    const size_t x_real_elems = cols_in * nsplit * q;
+    {
+        cuuint64_t dims[5] = {(cuuint64_t)q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, 2};
+        cuuint64_t str[4] = {(cuuint64_t)nsplit * q * 2, (cuuint64_t)g.W * nsplit * q * 2,
+                             (cuuint64_t)g.H * g.W * nsplit * q * 2, (cuuint64_t)x_real_elems * 2};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.tw, (cuuint32_t)g.th, 1, 1};
+        __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb);
+        if ((rc = encode(&mxh_r, base, 5, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxl_r, base + (nsplit == 2 ? q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
+    }
+    {
+        const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
+        cuuint64_t dims[5] = {(cuuint64_t)2 * q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, (cuuint64_t)nc};
+        cuuint64_t str[4] = {(cuuint64_t)nsplit * 2 * q * 2, (cuuint64_t)g.W * nsplit * 2 * q * 2,
+                             (cuuint64_t)g.H * g.W * nsplit * 2 * q * 2, (cuuint64_t)2 * x_real_elems * 2};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.tw, (cuuint32_t)g.th, 1, 1};
+        __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb) + 2 * x_real_elems;
+        if ((rc = encode(&mxh_c, base, 5, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxl_c, base + (nsplit == 2 ? 2 * q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
+    }
+
+    const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
+    const size_t smem = (size_t)kStages * (kTileCols * 128 + (size_t)bn_max * 128) + 1024;
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (configured_device != dev) {
+        CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024),
+                      CIRC_ERR_CUDA);
+        configured_device = dev;
+    }
+    contract_tc_kernel<<<(unsigned)ctas, kTcThreads, smem, stream>>>(ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
+    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+}  // namespace circ

@@ -40,6 +40,7 @@ def run_fc(case: synth.FcCase, variant=circ.CIRC_VARIANT_AUTO, convention=0, y_b
                        dtype=torch.bfloat16 if y_bf16 else torch.float32)
         circ.circ_fc_forward(h, x, y, case.batch, stream)
         torch.cuda.synchronize()
+        circ.circ_device_status(h)
         used = circ.circ_last_variant(h)
         return y.float().cpu().numpy().astype(np.float64), used
     finally:
@@ -62,6 +63,7 @@ def run_conv(case: synth.ConvCase, variant=circ.CIRC_VARIANT_AUTO, convention=0)
                        dtype=torch.bfloat16 if case.bf16_io else torch.float32)
         circ.circ_conv_forward(h, x, y, case.N, case.H, case.W)
         torch.cuda.synchronize()
+        circ.circ_device_status(h)
         used = circ.circ_last_variant(h)
         return y.float().cpu().numpy().astype(np.float64), used
     finally:
