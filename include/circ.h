@@ -118,6 +118,33 @@ CIRC_API int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int
 CIRC_API int circ_fc_forward_host(circ_handle h, const void* x_host, void* y_host, int batch, void* stream);
 CIRC_API int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int N, int H, int W, void* stream);
 
+/*
+ * circ_fc_forward_noalloc -- circ_fc_forward for callers that must not allocate device memory.
+ * (The paper has no counterpart: this is a deployment aid of the library, not part of the method.)
+ *
+ * Meant for code that cannot call cudaMalloc at forward time: latency-critical loops where an
+ * allocation could stall the device, processes whose free memory is owned by another allocator,
+ * or plug-ins that only receive pre-made buffers.  This call never calls cudaMalloc, cudaFree or
+ * any allocating routine.  Its scratch memory (the frequency-domain operands between the three
+ * kernels of the staged path) is a fixed array of CIRC_NOALLOC_SCRATCH_BYTES compiled into the
+ * library; every GPU context that loads the library holds that array until it exits.
+ *
+ *   h, x, y, batch, stream : exactly as circ_fc_forward (x, y DEVICE pointers owned by the caller).
+ *   Limit: 4 * (2 * ceil(batch / 2)) * (n + m) bytes (+ alignment) must fit in the array; larger
+ *          requests fail with CIRC_ERR_SHAPE and a message that names both numbers.
+ *          circ_noalloc_max_bytes() returns the array size.
+ *   The first call on each device looks up the array's device address (cudaGetSymbolAddress);
+ *   make that first call outside any stream capture.
+ *   All calls, on all handles and streams, share the one array and leave their intermediate
+ *   results in it: two calls whose kernels overlap on the GPU race and corrupt each other, so
+ *   issue them on one stream or order them yourself.  Nothing in the array needs clearing between
+ *   calls (each stage overwrites everything the next one reads).
+ *   Always uses the three-launch float32 FMA path, whatever circ_set_variant says.
+ */
+#define CIRC_NOALLOC_SCRATCH_BYTES (32 * 1024 * 1024)
+CIRC_API int circ_fc_forward_noalloc(circ_handle h, const void* x, void* y, int batch, void* stream);
+CIRC_API long circ_noalloc_max_bytes(void);
+
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);
 

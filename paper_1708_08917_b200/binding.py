@@ -31,6 +31,8 @@ SIGNATURES = {
     "circ_conv_forward_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_profile_begin": (_ci, [_vp]),
     "circ_profile_end": (_ci, [_vp, _vp, _vp]),
+    "circ_fc_forward_noalloc": (_ci, [_vp, _vp, _vp, _ci, _vp]),
+    "circ_noalloc_max_bytes": (_cl, []),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -158,6 +160,20 @@ def circ_profile_end(h: int):
     cnt = (ctypes.c_int * 4)()
     _check(load().circ_profile_end(h, ctypes.addressof(ms), ctypes.addressof(cnt)))
     return list(ms), list(cnt)
+
+
+def circ_fc_forward_noalloc(h: int, x, y, batch: int, stream=None) -> None:
+    """``circ_fc_forward`` for callers that may not allocate: scratch lives in a fixed array inside the library.
+
+    Use it from code that cannot afford (or is not permitted) a ``cudaMalloc`` at forward time.  The batch is
+    limited by ``circ_noalloc_max_bytes()``; all calls share one scratch array, so do not overlap them on the GPU;
+    make the first call on a device outside stream capture.
+    """
+    _check(load().circ_fc_forward_noalloc(h, _ptr(x), _ptr(y), batch, _stream(stream)))
+
+
+def circ_noalloc_max_bytes() -> int:
+    return load().circ_noalloc_max_bytes()
 
 
 def circ_device_status(h: int) -> None:
