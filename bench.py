@@ -3,13 +3,14 @@
 
     python bench.py --gpus N --steps K --warmup W            # the CUDA library (C ABI)
     python bench.py --impl reference --steps K --warmup W    # the fp64 dense CPU oracle
+    python bench.py --workload NAME ...                      # another configuration (see workload())
 
-A step is one forward pass of the headline workload -- the 4096 x 4096, k = 64, float32 layer with
-fused bias + ReLU at batch 256 -- over one batch of seeded synthetic input.  Steps rotate through
-enough distinct (layer, x, y) sets that the working set exceeds twice the L2 cache, so every byte
-of every step comes from HBM.  With N > 1 (torchrun) every rank runs the same job on its own GPU
-and its own batches (samples are independent: no collective on the data path); the reported value
-is all samples of all ranks divided by the slowest rank's device time.
+A step is one forward pass of the workload over one batch of seeded synthetic input.  The default
+workload is the 4096 x 4096, k = 64, float32 layer with fused bias + ReLU at batch 256.  Steps
+rotate through enough distinct (layer, x, y) sets that the working set exceeds twice the L2 cache,
+so every byte of every step comes from HBM.  With N > 1 (torchrun) every rank runs the same job on
+its own GPU and its own batches (samples are independent: no collective on the data path); the
+reported value is all samples of all ranks divided by the slowest rank's device time.
 """
 from __future__ import annotations
 
@@ -17,10 +18,12 @@ import argparse
 import hashlib
 import json
 import os
+import re
 import subprocess
 import sys
 import tempfile
 import time
+from dataclasses import dataclass
 from pathlib import Path
 
 import numpy as np
@@ -33,36 +36,68 @@ from paper_1708_08917_b200 import synth  # noqa: E402
 METRIC = "block-circ layer samples/s"
 UNIT = "samples/s"
 L2_BYTES = 126 * 1024 * 1024
+STAGES = ["input_fft", "contraction", "output_ifft", "fused_fc"]
+STAGE_SOURCE = {"input_fft": "circ_staged.cu", "output_ifft": "circ_staged.cu", "contraction": "circ_tensor.cu",
+                "fused_fc": "circ_fused.cu"}
 
-# DRAM traffic of the dominant kernel from one ncu capture (dram__bytes_read.sum + dram__bytes_write.sum
-# per launch), valid only while the kernel source is unchanged: the hash ties the counters to the code.
-NCU_TRAFFIC = {
-    "kernel": None,
-    "bytes_per_launch": None,
-    "source": "paper_1708_08917_b200/csrc/circ_contract_fma.cu",
-    "source_sha256": None,
-}
+# DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum), keyed by
+# (workload, kernel).  Each entry is tied to the sha256 of the kernel's source file at capture time;
+# when the source has changed since, the figure is withheld (reported as null).
+NCU_TRAFFIC: dict = {}
 
 
-def workload(name: str):
-    """The named benchmark workload -> (FcCase, description)."""
-    if name.startswith("cfg2_b"):
-        b = int(name[len("cfg2_b"):])
-        return synth.config2(b), f"FC 4096x4096 k=64 fp32 batch {b}, bias+ReLU fused"
+@dataclass
+class Workload:
+    name: str
+    desc: str
+    kind: str            # "fc" or "conv"
+    case: object
+    samples: int         # samples (FC) or images (CONV) per step
+    alg_bytes: int       # bytes the method must move per forward
+    dense_flops: float   # flops of the equivalent dense layer per forward
+    sx: int
+    sy: int
+
+
+def workload(name: str) -> Workload:
+    """Named workloads: cfg1, cfg2_b{B}, cfg3_l{0,1,2}, cfg4, sweep_n{n}_k{k}_b{B}[_bf16]."""
+    def fc(case, desc):
+        s = 2 if case.bf16_io else 4
+        alg = 4 * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
+        return Workload(name, desc, "fc", case, case.batch, alg, 2.0 * case.m * case.n * case.batch, s, s)
+
+    if name == "cfg1":
+        return fc(synth.config1(), "FC 256x256 k=16 fp32 batch 1")
+    m = re.fullmatch(r"cfg2_b(\d+)", name)
+    if m:
+        b = int(m.group(1))
+        return fc(synth.config2(b), f"FC 4096x4096 k=64 fp32 batch {b}, bias+ReLU fused")
+    m = re.fullmatch(r"cfg3_l([012])", name)
+    if m:
+        c = synth.config3_layers(128)[int(m.group(1))]
+        if c.x.shape[0] != 128:
+            c.x = synth.normal((128, c.n), 1.0, synth.stream_id(c.name, "x"), absolute=True)
+        return fc(c, f"FC {c.n}->{c.m} k=128 fp32 batch 128 (AlexNet-FC stack layer {m.group(1)})")
+    m = re.fullmatch(r"sweep_n(\d+)_k(\d+)_b(\d+)(_bf16)?", name)
+    if m:
+        n, k, b, bf = int(m.group(1)), int(m.group(2)), int(m.group(3)), bool(m.group(4))
+        return fc(synth.sweep_point(n, k, b, bf), f"FC {n}x{n} k={k} {'bf16' if bf else 'fp32'} batch {b}")
+    if name == "cfg4":
+        c = synth.config4()
+        pix = c.N * c.H * c.W
+        alg = 4 * c.r * c.r * c.c_out * c.c_in // c.k + 2 * pix * (c.c_in + c.c_out)
+        return Workload(name, "CONV 3x3 pad 1, 256->256 ch, 28x28, batch 32, k=16, bf16 activations", "conv", c, c.N, alg,
+                        2.0 * pix * c.r * c.r * c.c_in * c.c_out, 2, 2)
     raise SystemExit(f"unknown workload {name}")
-
-
-def algorithmic_bytes(case, sx=4, sy=4, sw=4) -> int:
-    """Bytes the method itself must move per forward: stored spectra + x + y + bias."""
-    return sw * case.m * case.n // case.k + sx * case.batch * case.n + sy * case.batch * case.m + (4 * case.m if case.bias is not None else 0)
 
 
 def measured_peaks() -> dict:
     f = ROOT / "MEASURED_PEAKS.json"
     if f.exists():
         d = json.loads(f.read_text())
-        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1400.0, "source": "fallback"}
 
 
 class ClockSampler:
@@ -79,7 +114,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
+                                          "-lms", "50", "-i", str(self.index)], stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
@@ -111,57 +146,69 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def oracle_rate(case, budget_s: float = 12.0):
-    """Time the fp64 dense oracle, as it stands, on a bounded number of batch rows -> (samples/s, rows, threads, seconds)."""
+# ---- the oracle legs (CPU) -----------------------------------------------------------------------
+
+def oracle_forward(wl: Workload, units: int):
+    """Run the fp64 dense oracle on the first `units` samples (FC rows / CONV images) of the workload."""
     import oracle
-    w = case.w.astype(np.float64)
-    x = case.x.astype(np.float64)
-    bias = None if case.bias is None else case.bias.astype(np.float64)
+    c = wl.case
+    bias = None if c.bias is None else c.bias.astype(np.float64)
+    if wl.kind == "fc":
+        return oracle.fc(c.w.astype(np.float64), c.x[:units].astype(np.float64), bias=bias, relu=c.relu)
+    return oracle.conv(c.w.astype(np.float64), c.x[:units].astype(np.float64), c.pad, bias=bias, relu=c.relu)
+
+
+def oracle_rate(wl: Workload, budget_s: float = 12.0):
+    """Time the oracle, as it stands, for about `budget_s` seconds on a bounded sample -> (samples/s, description, threads)."""
+    import oracle
     t0 = time.perf_counter()
-    oracle.fc(w, x[:1], bias=bias, relu=case.relu)
-    per_row = max(time.perf_counter() - t0, 1e-6)
-    rows = int(min(case.batch, max(oracle.threads(), budget_s * oracle.threads() / per_row / 4)))
-    rows = max(1, min(rows, case.batch))
-    t0 = time.perf_counter()
-    oracle.fc(w, x[:rows], bias=bias, relu=case.relu)
-    dt = time.perf_counter() - t0
-    return rows / dt, rows, oracle.threads(), dt
+    oracle_forward(wl, 1)
+    t_one = max(time.perf_counter() - t0, 1e-6)
+    units = int(max(1, min(wl.samples, budget_s / t_one / 2)))
+    done, t0 = 0, time.perf_counter()
+    while True:
+        oracle_forward(wl, units)
+        done += units
+        dt = time.perf_counter() - t0
+        if dt >= budget_s or done >= 50 * wl.samples:
+            break
+    what = "batch rows" if wl.kind == "fc" else "images"
+    return done / dt, f"{units} of {wl.samples} {what} per pass, {done // units} passes, all outputs, {dt:.1f} s", oracle.threads()
 
 
 def run_reference(args) -> int:
     """The reference arm: the CPU oracle on the same config / metric; rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
         return 0
-    case, desc = workload(args.workload)
+    wl = workload(args.workload)
     import oracle
-    w = case.w.astype(np.float64)
-    bias = None if case.bias is None else case.bias.astype(np.float64)
-    x = case.x.astype(np.float64)
     # bounded sample of the batch per step, sized so that the whole run stays within about two minutes
     t0 = time.perf_counter()
-    oracle.fc(w, x[:1], bias=bias, relu=case.relu)
-    t_row = max(time.perf_counter() - t0, 1e-6)
-    rows = int(max(1, min(case.batch, 120.0 / ((args.steps + args.warmup) * t_row))))
+    oracle_forward(wl, 1)
+    t_one = max(time.perf_counter() - t0, 1e-6)
+    units = int(max(1, min(wl.samples, 120.0 / ((args.steps + args.warmup) * t_one))))
     for _ in range(args.warmup):
-        oracle.fc(w, x[:rows], bias=bias, relu=case.relu)
+        oracle_forward(wl, units)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.fc(w, x[:rows], bias=bias, relu=case.relu)
+        oracle_forward(wl, units)
     dt = time.perf_counter() - t0
-    value = rows * args.steps / dt
+    value = units * args.steps / dt
+    sample = f"{units} of {wl.samples} {'batch rows' if wl.kind == 'fc' else 'images'} per step, all outputs"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": args.workload, "description": desc, "sample": f"{rows} of {case.batch} batch rows per step"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
-                         "sample": f"{rows} of {case.batch} batch rows per step, all outputs"},
+        "config": {"workload": wl.name, "description": wl.desc, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
     return 0
 
+
+# ---- the CUDA arm ----------------------------------------------------------------------------------
 
 def max_over_ranks(ms: float, world: int) -> float:
     """Slowest rank's device time (all-reduce MAX over the process group when there is one)."""
@@ -174,13 +221,14 @@ def max_over_ranks(ms: float, world: int) -> float:
     return float(t.item())
 
 
-def traffic_if_current():
-    src = ROOT / NCU_TRAFFIC["source"]
-    if NCU_TRAFFIC["bytes_per_launch"] is None or not src.exists():
+def traffic_if_current(wl_name: str, kernel: str):
+    ent = NCU_TRAFFIC.get((wl_name, kernel))
+    if not ent:
         return None
-    if hashlib.sha256(src.read_bytes()).hexdigest() != NCU_TRAFFIC["source_sha256"]:
+    src = ROOT / "paper_1708_08917_b200" / "csrc" / STAGE_SOURCE[kernel]
+    if not src.exists() or hashlib.sha256(src.read_bytes()).hexdigest() != ent["source_sha256"]:
         return None        # the kernel changed since the counters were taken
-    return NCU_TRAFFIC["bytes_per_launch"]
+    return ent["bytes_per_launch"]
 
 
 def run_ours(args) -> int:
@@ -195,33 +243,76 @@ def run_ours(args) -> int:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    case, desc = workload(args.workload)
-    B = case.batch
-    alg = algorithmic_bytes(case)
+    wl = workload(args.workload)
+    c = wl.case
+    tdt = torch.bfloat16 if c.bf16_io else torch.float32
+    if wl.kind == "fc":
+        x_shape, y_shape = (c.batch, c.n), (c.batch, c.m)
+        weight_store = 3 * 4 * c.m * c.n // c.k + 4 * c.m * c.n // c.k      # stream + embedded f32 + embedded bf16 hi/lo
+        workspace = 4 * (c.batch + 1) * (c.m + c.n)
+    else:
+        Ho, Wo = c.H + 2 * c.pad - c.r + 1, c.W + 2 * c.pad - c.r + 1
+        x_shape, y_shape = (c.N, c.H, c.W, c.c_in), (c.N, Ho, Wo, c.c_out)
+        weight_store = 4 * 4 * c.r * c.r * c.c_out * c.c_in // c.k
+        workspace = 4 * (c.N + 1) * c.H * c.W * (c.c_in + c.c_out)
+    per_set = wl.alg_bytes + weight_store + workspace
     # distinct (layer, x, y) sets so that consecutive steps never touch the same bytes: > 2 x L2
-    per_set = alg + 3 * 4 * case.m * case.n // case.k + 8 * B * (case.m + case.n)   # + embedded operand + workspace
-    sets = int(min(64, max(2, -(-2 * L2_BYTES // per_set) + 1)))
+    sets = int(min(args.max_sets, max(2, -(-2 * L2_BYTES // per_set) + 1)))
     stream = torch.cuda.current_stream()
+
+    def draw_x(tag):
+        if wl.kind == "fc":
+            a = synth.uniform(x_shape, -1.0, 1.0, synth.stream_id(c.name, tag))
+        else:
+            a = synth.normal(x_shape, 1.0, synth.stream_id(c.name, tag), absolute=True)
+        return torch.from_numpy(a)
+
     handles, xs, ys = [], [], []
     for s in range(sets):
-        h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
-        if case.bias is not None:
-            circ.circ_set_bias(h, case.bias)
-        circ.circ_set_activation(h, int(case.relu))
-        circ.circ_reserve(h, B)
+        if wl.kind == "fc":
+            h = circ.circ_fc_create(c.m, c.n, c.k, c.w)
+            circ.circ_reserve(h, c.batch)
+        else:
+            h = circ.circ_conv_create(c.c_out, c.c_in, c.r, c.pad, c.k, c.w)
+            circ.circ_reserve(h, c.N * c.H * c.W)
+        if c.bias is not None:
+            circ.circ_set_bias(h, c.bias)
+        circ.circ_set_activation(h, int(c.relu))
+        code = circ.CIRC_BF16 if c.bf16_io else circ.CIRC_F32
+        circ.circ_set_io_dtype(h, code, code)
+        if args.variant:
+            circ.circ_set_variant(h, args.variant)
         handles.append(h)
         # every set and every rank gets its own batch (same distribution, different stream id)
-        xs.append(torch.from_numpy(synth.uniform((B, case.n), -1.0, 1.0, synth.stream_id(case.name, f"x{rank}_{s}"))).cuda())
-        ys.append(torch.empty(B, case.m, device="cuda", dtype=torch.float32))
+        xs.append(draw_x(f"x{rank}_{s}").cuda().to(tdt))
+        ys.append(torch.empty(y_shape, device="cuda", dtype=tdt))
     torch.cuda.synchronize()
 
-    def step(i):
-        s = i % sets
-        circ.circ_fc_forward(handles[s], xs[s], ys[s], B, stream)
+    def forward(s, st):
+        if wl.kind == "fc":
+            circ.circ_fc_forward(handles[s], xs[s], ys[s], c.batch, st)
+        else:
+            circ.circ_conv_forward(handles[s], xs[s], ys[s], c.N, c.H, c.W, st)
 
     for i in range(max(args.warmup, 3)):
-        step(i)
+        forward(i % sets, stream)
     torch.cuda.synchronize()
+    circ.circ_device_status(handles[0])
+
+    # One rotation through all sets is captured in a CUDA graph so that the GPU, not the host's
+    # launch rate, sets the pace; the timed region replays it and runs the remainder eagerly.
+    graph, cap_stream = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    cap_stream.wait_stream(stream)
+    l0 = circ.circ_launch_count()
+    with torch.cuda.graph(graph, stream=cap_stream):
+        cs = torch.cuda.current_stream()
+        for s in range(sets):
+            forward(s, cs)
+    launches_per_rotation = circ.circ_launch_count() - l0
+    graph.replay()
+    torch.cuda.synchronize()
+    replays, rest = divmod(args.steps, sets)
+
     if world > 1:
         dist.barrier()
     sampler = ClockSampler(local_rank)
@@ -230,80 +321,91 @@ def run_ours(args) -> int:
     launches0 = circ.circ_launch_count()
     torch.cuda.synchronize()
     e0.record(stream)
-    for i in range(args.steps):
-        step(i)
+    for _ in range(replays):
+        graph.replay()
+    for i in range(rest):
+        forward(i % sets, stream)
     e1.record(stream)
     torch.cuda.synchronize()
-    launches = circ.circ_launch_count() - launches0
+    launches = circ.circ_launch_count() - launches0 + replays * launches_per_rotation
     if world > 1:
         dist.barrier()
     clocks = sampler.stop()
     ms_total = max_over_ranks(e0.elapsed_time(e1), world)
     ms_step = ms_total / args.steps
-    value = world * B * args.steps / (ms_total * 1e-3)
+    value = world * wl.samples * args.steps / (ms_total * 1e-3)
     variant = circ.circ_last_variant(handles[0])
 
-    # per-kernel device times over the same rotation (separate pass: events between kernels)
-    prof_steps = min(args.steps, 200)
+    # Per-kernel device times over the same rotation: CUDA events around every kernel.  A spin
+    # kernel runs first so that the host queues the whole pass while the GPU is still busy and
+    # every kernel follows its start event without a launch gap.
+    prof_steps = min(args.steps, 4 * sets, 160)
     for h in handles:
         circ.circ_profile_begin(h)
+    torch.cuda._sleep(int(4e7))
     for i in range(prof_steps):
-        step(i)
+        forward(i % sets, stream)
     torch.cuda.synchronize()
     stage_ms, stage_n = [0.0] * 4, [0] * 4
     for h in handles:
         ms, cnt = circ.circ_profile_end(h)
         stage_ms = [a + b for a, b in zip(stage_ms, ms)]
         stage_n = [a + b for a, b in zip(stage_n, cnt)]
-    names = ["input_fft", "contraction", "output_ifft", "fused_fc"]
-    per_launch_us = {names[i]: (1e3 * stage_ms[i] / stage_n[i] if stage_n[i] else None) for i in range(4)}
+    per_launch_us = {STAGES[i]: (1e3 * stage_ms[i] / stage_n[i] if stage_n[i] else None) for i in range(4)}
     dom = max(range(4), key=lambda i: stage_ms[i])
     dom_us = 1e3 * stage_ms[dom] / max(stage_n[dom], 1)
     peaks = measured_peaks()
-    achieved = alg / (dom_us * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": names[dom], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+    achieved = wl.alg_bytes / (dom_us * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": STAGES[dom], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"], "frac_of_nominal_8000": achieved / 8000.0,
-                "traffic": traffic_if_current(), "algorithmic_bytes_per_launch": alg,
+                "traffic": traffic_if_current(wl.name, STAGES[dom]), "algorithmic_bytes_per_launch": wl.alg_bytes,
                 "kernel_us_per_launch": per_launch_us,
-                "whole_forward_frac": alg / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+                "whole_forward_frac": wl.alg_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]}
 
     # end to end through the host-pointer entry point: pinned host x -> device -> forward -> pinned host y
     e2e = None
-    if True:
-        xh = [torch.from_numpy(synth.uniform((B, case.n), -1.0, 1.0, synth.stream_id(case.name, f"xh{rank}_{s}"))).pin_memory()
-              for s in range(min(sets, 8))]
-        yh = [torch.empty(B, case.m, dtype=torch.float32).pin_memory() for _ in range(len(xh))]
+    if not args.no_e2e:
+        nh = min(sets, 4)
+        xh = [draw_x(f"xh{rank}_{s}").to(tdt).pin_memory() for s in range(nh)]
+        yh = [torch.empty(y_shape, dtype=tdt).pin_memory() for _ in range(nh)]
+
+        def forward_host(i):
+            if wl.kind == "fc":
+                circ.circ_fc_forward_host(handles[i % sets], xh[i % nh], yh[i % nh], c.batch, stream)
+            else:
+                circ.circ_conv_forward_host(handles[i % sets], xh[i % nh], yh[i % nh], c.N, c.H, c.W, stream)
+
         for i in range(3):
-            circ.circ_fc_forward_host(handles[i % sets], xh[i % len(xh)], yh[i % len(xh)], B, stream)
+            forward_host(i)
         torch.cuda.synchronize()
         e2e_steps = min(args.steps, 300)
         if world > 1:
             dist.barrier()
         e0.record(stream)
         for i in range(e2e_steps):
-            circ.circ_fc_forward_host(handles[i % sets], xh[i % len(xh)], yh[i % len(xh)], B, stream)
+            forward_host(i)
         e1.record(stream)
         torch.cuda.synchronize()
         ms_e2e = max_over_ranks(e0.elapsed_time(e1), world)
-        e2e = {"value": world * B * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 4 * B * case.n,
-               "d2h_bytes_per_step": 4 * B * case.m, "steps": e2e_steps}
+        e2e = {"value": world * wl.samples * e2e_steps / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(np.prod(x_shape)) * wl.sx, "d2h_bytes_per_step": int(np.prod(y_shape)) * wl.sy,
+               "steps": e2e_steps}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        rate, rows, threads, secs = oracle_rate(case)
-        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"{rows} of {B} batch rows, all {case.m} outputs, {secs:.1f} s"}
+        rate, what, threads = oracle_rate(wl)
+        cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what}
 
     for h in handles:
         circ.circ_destroy(h)
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic",
-            "config": {"workload": args.workload, "description": desc, "batch_per_gpu": B, "variant": variant,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if c.bf16_io else "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "description": wl.desc, "samples_per_step_per_gpu": wl.samples, "variant": variant,
                        "l2": f"steps rotate through {sets} distinct (layer, x, y) sets, {sets * per_set / 1e6:.0f} MB > 2 x L2",
-                       "dense_equiv_tflops": 2.0 * case.m * case.n * B * world / (ms_step * 1e-3) / 1e12},
+                       "dense_equiv_tflops": wl.dense_flops * world / (ms_step * 1e-3) / 1e12},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
@@ -315,11 +417,14 @@ def run_ours(args) -> int:
 def main() -> int:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_b256")
+    ap.add_argument("--variant", type=int, default=0, help="force a CIRC_VARIANT_* (0 = planner's choice)")
+    ap.add_argument("--max-sets", type=int, default=64)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -33,6 +33,15 @@ struct ProfRec {
 };
 struct Profiler {
     std::vector<ProfRec> recs;
+    std::vector<cudaEvent_t> pool;  // events made ahead of time so that recording stays cheap
+    bool take(cudaEvent_t* e) {
+        if (!pool.empty()) {
+            *e = pool.back();
+            pool.pop_back();
+            return true;
+        }
+        return cudaEventCreate(e) == cudaSuccess;
+    }
 };
 struct StageTimer {
     Profiler* prof;
@@ -41,7 +50,7 @@ struct StageTimer {
     StageTimer(Layer* L, int stage, cudaStream_t s) : prof(static_cast<Profiler*>(L->prof)), stream(s) {
         if (!prof) return;
         rec.stage = stage;
-        if (cudaEventCreate(&rec.start) != cudaSuccess || cudaEventCreate(&rec.stop) != cudaSuccess) {
+        if (!prof->take(&rec.start) || !prof->take(&rec.stop)) {
             prof = nullptr;
             return;
         }
@@ -95,6 +104,7 @@ static void free_layer(Layer* L) {
             cudaEventDestroy(r.start);
             cudaEventDestroy(r.stop);
         }
+        for (auto& e : static_cast<Profiler*>(L->prof)->pool) cudaEventDestroy(e);
         delete static_cast<Profiler*>(L->prof);
     }
     if (prev != L->device && prev >= 0) cudaSetDevice(prev);
@@ -416,6 +426,12 @@ int circ_profile_begin(circ_handle h) {
         set_error(CIRC_ERR_ALLOC, "host allocation failed");
         return CIRC_ERR_ALLOC;
     }
+    Profiler* P = static_cast<Profiler*>(L->prof);
+    while (P->pool.size() < 512) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) break;
+        P->pool.push_back(e);
+    }
     return CIRC_OK;
 }
 
@@ -443,6 +459,7 @@ int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage) 
         cudaEventDestroy(r.start);
         cudaEventDestroy(r.stop);
     }
+    for (auto& e : P->pool) cudaEventDestroy(e);
     delete P;
     L->prof = nullptr;
     return rc;

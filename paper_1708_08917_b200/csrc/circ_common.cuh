@@ -25,6 +25,9 @@ namespace circ {
 //        [Yr]   [Wr -Wi] [Zr]      M = 2p, Kd = 2q       column c      <- ( Re Z[g],    Im Z[g]   )
 //        [Yi] = [Wi  Wr] [Zi]                            column Bh+c   <- ( Re Z[K-g], -Im Z[K-g] )
 //   (the second column group is the conjugate of bin K-g, so that it multiplies What[g] too).
+//   Real and imaginary parts are interleaved: contraction index 2j / 2j+1 = Re / Im of column
+//   block j, row 2i / 2i+1 = Re / Im of row block i, so that the transforms read and write
+//   (Re, Im) pairs as one vector.
 //
 // Every problem has 2*Bh columns.  Operands are "K-major": X[col][kk], A[row][kk]; results are
 // Y[col][row].  Convolutions concatenate the taps along the contraction index:

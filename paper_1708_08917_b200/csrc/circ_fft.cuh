@@ -176,11 +176,16 @@ __device__ __forceinline__ void fft_inverse(float2 (&v)[FftShape<K>::E], int l, 
     }
 }
 
-// Fill a shared-memory twiddle table tw[n] = exp(-2 pi i n / K) from the 256-entry master table
-// (master[n] = exp(-2 pi i n / 256), computed on the host in double precision).
+// Fill a shared-memory twiddle table tw[n] = exp(-2 pi i n / K).  Computed in place (sincospif takes
+// the argument in units of pi, so the reduction is exact) rather than fetched: a table in global
+// memory would put one more dependent memory round trip at the head of every kernel.
 template <int K>
-__device__ __forceinline__ void load_twiddles(float2* tw, const float2* __restrict__ master) {
-    for (int n = threadIdx.x; n < K; n += blockDim.x) tw[n] = master[n * (256 / K)];
+__device__ __forceinline__ void load_twiddles(float2* tw, const float2* __restrict__ /*unused master table*/) {
+    for (int n = threadIdx.x; n < K; n += blockDim.x) {
+        float s, c;
+        sincospif(-2.0f * (float)n / (float)K, &s, &c);
+        tw[n] = make_float2(c, s);
+    }
 }
 
 }  // namespace circ

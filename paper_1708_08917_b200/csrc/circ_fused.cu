@@ -20,7 +20,7 @@
 
 namespace circ {
 
-constexpr int kFusedThreads = 256;
+constexpr int kFusedThreads = 512;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kMaxFusedSmem = 200 * 1024;
 
@@ -33,23 +33,26 @@ struct FusedArgs {
     int relu, x_bf16, y_bf16;
     int m, n, p, q, batch, Bh;
     int rows_per_cta;
+    int jsplit;  // warps that share one row block (power of two, divides the warp count)
 };
 
-__host__ __device__ inline size_t fused_smem_bytes(int k, int q, int pairs, int rows_per_cta) {
-    return sizeof(float2) * ((size_t)k + (size_t)pairs * q * k + (size_t)kFusedWarps * rows_per_cta * pairs * k);
+__host__ __device__ inline size_t fused_smem_bytes(int k, int q, int pairs, int rows_per_cta, int jsplit) {
+    return sizeof(float2) * ((size_t)k + (size_t)pairs * q * k + (size_t)jsplit * rows_per_cta * pairs * k);
 }
 
 template <int K, int PAIRS>
-__global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
+__global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a) {
     constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = kFusedThreads / L;
     constexpr int H = K / 2;                    // packed slots per block
     constexpr int G = K / 4;                    // threads that cover one block with 16-byte loads
     constexpr int NU = G > 32 ? G / 32 : 1;     // 16-byte loads per thread and block
     constexpr int BPW = G >= 32 ? 1 : 32 / G;   // blocks per warp-wide load
+    constexpr int UNROLL = (PAIRS == 1 ? 8 : PAIRS == 2 ? 4 : 2) / (NU > 1 ? 2 : 1);  // weight loads in flight per thread
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
-    float2* zs = tw + K;                                       // [PAIRS][q][K]
-    float2* part = zs + (size_t)PAIRS * a.q * K;               // [warps][rows][PAIRS][K]
+    float2* zlo = tw + K;                                      // [PAIRS][q][H]  Z[s]
+    float2* zhi = zlo + (size_t)PAIRS * a.q * H;               // [PAIRS][q][H]  Z[k-s], slot 0 = Z[k/2]
+    float2* part = zhi + (size_t)PAIRS * a.q * H;              // [jsplit][rows][PAIRS][K]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = a.q;
@@ -83,12 +86,13 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
             for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
             fft_forward<K>(v, l, tw);
             if (T < total) {
-                float2* dst = zs + (size_t)T * K;
+                float2* dlo = zlo + (size_t)T * H;
+                float2* dhi = zhi + (size_t)T * H;
 #pragma unroll
                 for (int f1 = 0; f1 < E; ++f1) {
                     const int f = f2 + L * f1;
-                    const int pos = f < H ? f : (f == H ? H : H + (K - f));
-                    dst[pos] = v[f1];
+                    if (f < H) dlo[f] = v[f1];
+                    else dhi[f == H ? 0 : K - f] = v[f1];
                 }
             }
         }
@@ -99,11 +103,13 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
     const int i0 = blockIdx.x * a.rows_per_cta;
     const int rows = min(a.rows_per_cta, a.p - i0);
     {
+        const int JS = a.jsplit;
+        const int slice = warp % JS, row_first = warp / JS, row_step = kFusedWarps / JS;
         const int u0 = G >= 32 ? lane : lane % G;   // first packed-slot pair of this thread
         const int jsub = G >= 32 ? 0 : lane / G;
-        const int per_warp = ((q + kFusedWarps * BPW - 1) / (kFusedWarps * BPW)) * BPW;
-        const int jb = warp * per_warp, je = min(q, jb + per_warp);
-        for (int row = 0; row < rows; ++row) {
+        const int per_slice = ((q + JS * BPW - 1) / (JS * BPW)) * BPW;
+        const int jb = slice * per_slice, je = min(q, jb + per_slice);
+        for (int row = row_first; row < rows; row += row_step) {
             const float* wrow = a.w_stream + (size_t)(i0 + row) * q * K;
             float2 acc[PAIRS][NU][4];
 #pragma unroll
@@ -113,7 +119,6 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[c][t][e] = make_float2(0.f, 0.f);
 
-            constexpr int UNROLL = 4;
             for (int j = jb + jsub; j < je; j += BPW * UNROLL) {
                 float4 wv[UNROLL][NU];
 #pragma unroll
@@ -137,9 +142,9 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
                         const float a1 = w.z, b1 = w.w;
 #pragma unroll
                         for (int c = 0; c < PAIRS; ++c) {
-                            const float2* zb = zs + ((size_t)c * q + jj) * K;
-                            const float4 zl = *reinterpret_cast<const float4*>(zb + 2 * u);
-                            const float4 zh = *reinterpret_cast<const float4*>(zb + H + 2 * u);
+                            const size_t zoff = ((size_t)c * q + jj) * H + 2 * u;
+                            const float4 zl = *reinterpret_cast<const float4*>(zlo + zoff);
+                            const float4 zh = *reinterpret_cast<const float4*>(zhi + zoff);
                             float2* ac = acc[c][t];
                             ac[0].x = fmaf(a0, zl.x, fmaf(-b0, zl.y, ac[0].x));
                             ac[0].y = fmaf(a0, zl.y, fmaf(b0, zl.x, ac[0].y));
@@ -171,7 +176,7 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
             if (jsub == 0) {
 #pragma unroll
                 for (int c = 0; c < PAIRS; ++c) {
-                    float2* dst = part + (((size_t)warp * a.rows_per_cta + row) * PAIRS + c) * K;
+                    float2* dst = part + (((size_t)slice * a.rows_per_cta + row) * PAIRS + c) * K;
 #pragma unroll
                     for (int t = 0; t < NU; ++t) {
                         const int u = u0 + 32 * t;
@@ -199,8 +204,8 @@ __global__ void __launch_bounds__(kFusedThreads) fused_fc_kernel(FusedArgs a) {
 #pragma unroll
             for (int f1 = 0; f1 < E; ++f1) v[f1] = make_float2(0.f, 0.f);
             if (live) {
-                for (int wp = 0; wp < kFusedWarps; ++wp) {
-                    const float2* src = part + (((size_t)wp * a.rows_per_cta + row) * PAIRS + c) * K;
+                for (int sl = 0; sl < a.jsplit; ++sl) {   // fixed order: bitwise repeatable
+                    const float2* src = part + (((size_t)sl * a.rows_per_cta + row) * PAIRS + c) * K;
 #pragma unroll
                     for (int f1 = 0; f1 < E; ++f1) {
                         const float2 t = src[f2 + L * f1];
@@ -240,18 +245,23 @@ static int pairs_for(int batch) {
     return bh <= 1 ? 1 : bh <= 2 ? 2 : 4;
 }
 
-static int plan_rows(const Layer* L, int pairs) {
-    // enough CTAs for two per SM when shared memory allows it, else one per SM
-    const size_t base = fused_smem_bytes(L->geo.k, L->geo.q, pairs, 1);
-    const int target = base <= 100 * 1024 ? 296 : 148;
-    int rows = (L->geo.p + target - 1) / target;
-    return rows < 1 ? 1 : rows;
+static void plan(const Layer* L, int pairs, int* rows, int* jsplit) {
+    // one CTA per SM; when a CTA has fewer row blocks than warps, several warps share a row block
+    int r = (L->geo.p + 147) / 148;
+    if (r < 1) r = 1;
+    int js = 1;
+    while (js * 2 * r <= kFusedWarps) js *= 2;
+    while (js > 1 && fused_smem_bytes(L->geo.k, L->geo.q, pairs, r, js) > (size_t)kMaxFusedSmem) js /= 2;
+    *rows = r;
+    *jsplit = js;
 }
 
 bool fused_fc_supported(const Layer* L, int batch) {
     if (L->kind != 0 || batch < 1 || batch > 8) return false;
     const int pairs = pairs_for(batch);
-    return fused_smem_bytes(L->geo.k, L->geo.q, pairs, plan_rows(L, pairs)) <= (size_t)kMaxFusedSmem;
+    int rows, js;
+    plan(L, pairs, &rows, &js);
+    return fused_smem_bytes(L->geo.k, L->geo.q, pairs, rows, js) <= (size_t)kMaxFusedSmem;
 }
 
 template <int K, int PAIRS>
@@ -292,9 +302,9 @@ int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStrea
     a.m = L->m; a.n = L->n; a.p = L->geo.p; a.q = L->geo.q;
     a.batch = batch;
     a.Bh = (batch + 1) / 2;
-    a.rows_per_cta = plan_rows(L, pairs);
+    plan(L, pairs, &a.rows_per_cta, &a.jsplit);
     const unsigned grid = (unsigned)((a.p + a.rows_per_cta - 1) / a.rows_per_cta);
-    const size_t smem = fused_smem_bytes(L->geo.k, a.q, pairs, a.rows_per_cta);
+    const size_t smem = fused_smem_bytes(L->geo.k, a.q, pairs, a.rows_per_cta, a.jsplit);
     int rc;
     switch (L->geo.k) {
         case 4: rc = launch_k<4>(a, pairs, grid, smem, stream); break;

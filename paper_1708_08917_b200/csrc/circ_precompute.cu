@@ -60,13 +60,14 @@ __global__ void precompute_spectra_kernel(const float* __restrict__ w, float* __
             if (a_f32) a_f32[at] = fre;
         } else {
             const size_t kd = (size_t)2 * q * taps;
-            const size_t r0 = base + (size_t)i * kd + (size_t)tap * 2 * q;
-            const size_t r1 = base + (size_t)(p + i) * kd + (size_t)tap * 2 * q;
+            // rows 2i (real part of the output) and 2i+1 (imaginary part); columns 2j (Re Z) and 2j+1 (Im Z)
+            const size_t r0 = base + (size_t)(2 * i) * kd + (size_t)tap * 2 * q;
+            const size_t r1 = base + (size_t)(2 * i + 1) * kd + (size_t)tap * 2 * q;
             if (a_f32) {
-                a_f32[r0 + j] = fre;
-                a_f32[r0 + q + j] = -fim;
-                a_f32[r1 + j] = fim;
-                a_f32[r1 + q + j] = fre;
+                a_f32[r0 + 2 * j] = fre;
+                a_f32[r0 + 2 * j + 1] = -fim;
+                a_f32[r1 + 2 * j] = fim;
+                a_f32[r1 + 2 * j + 1] = fre;
             }
         }
         // split bfloat16 operand for the tensor-core contraction: [problem][row][tap*2 + (hi|lo)][Kq]
@@ -83,10 +84,10 @@ __global__ void precompute_spectra_kernel(const float* __restrict__ w, float* __
             if (problem_is_real(prob)) {
                 put(i, q, j, fre);
             } else {
-                put(i, 2 * q, j, fre);
-                put(i, 2 * q, q + j, -fim);
-                put((size_t)p + i, 2 * q, j, fim);
-                put((size_t)p + i, 2 * q, q + j, fre);
+                put((size_t)2 * i, 2 * q, 2 * j, fre);
+                put((size_t)2 * i, 2 * q, 2 * j + 1, -fim);
+                put((size_t)2 * i + 1, 2 * q, 2 * j, fim);
+                put((size_t)2 * i + 1, 2 * q, 2 * j + 1, fre);
             }
         }
     }

@@ -2,6 +2,11 @@
 // staged path.  Both kernels hold whole transforms in registers (circ_fft.cuh) and use shared
 // memory only to turn the "one transform = contiguous k samples" view of x and y into the
 // "one frequency = one matrix" view the per-frequency contraction needs (circ_common.cuh).
+//
+// The staging tile is bin-major: zs[bin][transform].  The side that holds transforms in
+// registers touches (bin f2 + L*f1, transform gi); the side that talks to the operand in global
+// memory walks along a row (consecutive transforms of one bin), which is also the direction in
+// which the operand is contiguous, so those global accesses are full coalesced runs.
 #include <type_traits>
 
 #include "circ_common.cuh"
@@ -12,119 +17,189 @@ namespace circ {
 
 constexpr int kThreads = 256;
 
+// Row length of the tile: TT transforms plus a pad that makes the register side conflict-free.
+// A half warp there is (16 / L) consecutive transforms x L bins, so rows must be 16 / L float2
+// apart modulo the 16 eight-byte banks.
+template <int K>
+struct Tile {
+    static constexpr int L = FftShape<K>::L;
+    static constexpr int TT = kThreads / L;
+    static constexpr int PAD = L == 1 ? 0 : (L == 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
+    static constexpr int ROW = TT + PAD;
+};
+
+__device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
+    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&t);
+}
+// low-order part of a float32 value after its bfloat16 rounding has been taken out
+__device__ __forceinline__ float bf16_residual(float v) { return v - __bfloat162float(__float2bfloat16_rn(v)); }
+
 // ---- S1: x -> operand X ------------------------------------------------------------------------
 // One transform = (pair c, column block j).  A CTA takes TT = 256 / L consecutive transforms.
+// XMODE 0: float32 operand [problem][col][Kq]                      (FMA contraction, any q)
+// XMODE 1: bfloat16 operand [problem][col][hi | lo][Kq]            (tensor cores, float32 input split in two)
+// XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
+// Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
 template <int K, typename TIN, int XMODE>
 __global__ void __launch_bounds__(kThreads)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2* __restrict__ tw256, int n, int q,
                  int B, int Bh, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = kThreads / L;
+    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW;
     __shared__ float2 tw[K];
-    __shared__ float2 zs[TT][K + 1];
+    __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw, tw256);
-    __syncthreads();
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
     float2 v[E];
-    if (T < total) {
-        const int c = (int)(T / q), j = (int)(T % q);
+    {
         float re[E], im[E];
-        load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
-        if (c + Bh < B) {
-            load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
-        } else {
 #pragma unroll
-            for (int r = 0; r < E; ++r) im[r] = 0.f;
+        for (int r = 0; r < E; ++r) re[r] = im[r] = 0.f;
+        if (T < total) {
+            const int c = (int)(T / q), j = (int)(T % q);
+            load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
+            if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
         }
 #pragma unroll
         for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
-    } else {
-#pragma unroll
-        for (int r = 0; r < E; ++r) v[r] = make_float2(0.f, 0.f);
     }
+    __syncthreads();  // twiddles ready
     fft_forward<K>(v, l, tw);
     const int f2 = lane_residue<K>(l);
 #pragma unroll
-    for (int f1 = 0; f1 < E; ++f1) zs[gi][f2 + L * f1] = v[f1];
+    for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
 
-    // Scatter: this thread now serves transform tl for the bins f0, f0 + L, ...
-    const int tl = threadIdx.x % TT, f0 = threadIdx.x / TT;
-    const long T2 = (long)blockIdx.x * TT + tl;
-    if (T2 >= total) return;
-    const int c = (int)(T2 / q), j = (int)(T2 % q);
     const size_t cols = 2 * (size_t)Bh;
-    // XMODE 0: float32 operand [problem][col][Kq]; 1 / 2: bfloat16 operand [problem][col][part][Kq]
-    // with parts (hi, lo) / (hi) for the tensor-core contraction.
     constexpr int NPART = XMODE == 1 ? 2 : 1;
     const size_t real_sz = cols * q * NPART, cplx_sz = 2 * real_sz;
-    auto put = [&](int prob, size_t col, int kq, int kk, float val) {
-        const size_t at = problem_offset(prob, real_sz, cplx_sz) + col * (size_t)(NPART * kq) + kk;
-        if constexpr (XMODE == 0) {
-            static_cast<float*>(xop)[at] = val;
-        } else {
-            __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(xop);
-            const __nv_bfloat16 hi = __float2bfloat16_rn(val);
-            xb[at] = hi;
-            if constexpr (XMODE == 1) xb[at + kq] = __float2bfloat16_rn(val - __bfloat162float(hi));
+
+    if constexpr (XMODE == 0) {
+        // scalar scatter (any q): one work item = (bin, transform), consecutive threads = consecutive transforms
+        float* xf = static_cast<float*>(xop);
+        for (int item = threadIdx.x; item < TT * K; item += kThreads) {
+            const int tl = item % TT, f = item / TT;
+            const long T2 = (long)blockIdx.x * TT + tl;
+            if (T2 >= total) continue;
+            const int c = (int)(T2 / q), j = (int)(T2 % q);
+            const float2 z = zs[f][tl];
+            if (f == 0 || f == K / 2) {
+                float* xg = xf + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                xg[(size_t)c * q + j] = z.x;
+                xg[((size_t)Bh + c) * q + j] = z.y;
+            } else if (f < K / 2) {
+                float* xg = xf + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * q + 2 * j;
+                *reinterpret_cast<float2*>(xg) = z;
+            } else {
+                float* xg = xf + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bh + c) * 2 * q + 2 * j;
+                *reinterpret_cast<float2*>(xg) = make_float2(z.x, -z.y);
+            }
         }
-    };
-#pragma unroll
-    for (int it = 0; it < E; ++it) {
-        const int f = f0 + L * it;
-        const float2 z = zs[tl][f];
-        if (f == 0 || f == K / 2) {
-            const int prob = f == 0 ? 0 : 1;
-            put(prob, (size_t)c, q, j, z.x);
-            put(prob, (size_t)Bh + c, q, j, z.y);
-        } else if (f < K / 2) {
-            put(f + 1, (size_t)c, 2 * q, j, z.x);
-            put(f + 1, (size_t)c, 2 * q, q + j, z.y);
-        } else {
-            put(K - f + 1, (size_t)Bh + c, 2 * q, j, z.x);
-            put(K - f + 1, (size_t)Bh + c, 2 * q, q + j, -z.y);
+    } else {
+        // vector scatter: one work item = (bin, 4 consecutive transforms) = 16 bytes of (Re, Im) bfloat16
+        // pairs per part; consecutive lanes = consecutive groups = consecutive memory.
+        __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(xop);
+        constexpr int GROUPS = TT / 4;
+        for (int item = threadIdx.x; item < GROUPS * K; item += kThreads) {
+            const int grp = item % GROUPS, f = item / GROUPS;
+            const long T0 = (long)blockIdx.x * TT + grp * 4;
+            if (T0 >= total) continue;                 // total is a multiple of 8 (q % 8 == 0)
+            const int c = (int)(T0 / q), j = (int)(T0 % q);
+            const float4 za = *reinterpret_cast<const float4*>(&zs[f][grp * 4]);
+            const float4 zb = *reinterpret_cast<const float4*>(&zs[f][grp * 4 + 2]);
+            if (f == 0 || f == K / 2) {
+                __nv_bfloat16* xg = xb + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                __nv_bfloat16* d0 = xg + (size_t)c * (NPART * q) + j;
+                __nv_bfloat16* d1 = xg + ((size_t)Bh + c) * (NPART * q) + j;
+                *reinterpret_cast<uint2*>(d0) = make_uint2(bf16_pair(za.x, za.z), bf16_pair(zb.x, zb.z));
+                *reinterpret_cast<uint2*>(d1) = make_uint2(bf16_pair(za.y, za.w), bf16_pair(zb.y, zb.w));
+                if constexpr (XMODE == 1) {
+                    *reinterpret_cast<uint2*>(d0 + q) = make_uint2(bf16_pair(bf16_residual(za.x), bf16_residual(za.z)),
+                                                                   bf16_pair(bf16_residual(zb.x), bf16_residual(zb.z)));
+                    *reinterpret_cast<uint2*>(d1 + q) = make_uint2(bf16_pair(bf16_residual(za.y), bf16_residual(za.w)),
+                                                                   bf16_pair(bf16_residual(zb.y), bf16_residual(zb.w)));
+                }
+            } else {
+                const bool mirror = f > K / 2;
+                const int g = mirror ? K - f : f;
+                const float sgn = mirror ? -1.f : 1.f;
+                __nv_bfloat16* d = xb + problem_offset(g + 1, real_sz, cplx_sz) +
+                                   ((size_t)(mirror ? Bh : 0) + c) * (NPART * 2 * q) + 2 * j;
+                const float i0 = sgn * za.y, i1 = sgn * za.w, i2 = sgn * zb.y, i3 = sgn * zb.w;
+                *reinterpret_cast<uint4*>(d) =
+                    make_uint4(bf16_pair(za.x, i0), bf16_pair(za.z, i1), bf16_pair(zb.x, i2), bf16_pair(zb.z, i3));
+                if constexpr (XMODE == 1)
+                    *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(
+                        bf16_pair(bf16_residual(za.x), bf16_residual(i0)), bf16_pair(bf16_residual(za.z), bf16_residual(i1)),
+                        bf16_pair(bf16_residual(zb.x), bf16_residual(i2)), bf16_pair(bf16_residual(zb.z), bf16_residual(i3)));
+            }
         }
     }
 }
 
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
-// One transform = (pair c, row block i).
-template <int K, typename TOUT>
+// One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
+// VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
+template <int K, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const float2* __restrict__ tw256,
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = kThreads / L;
+    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW;
     __shared__ float2 tw[K];
-    __shared__ float2 zs[TT][K + 1];
+    __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw, tw256);
+    const size_t cols = 2 * (size_t)Bho;
+    const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
 
-    {
-        const int tl = threadIdx.x % TT, f0 = threadIdx.x / TT;
-        const long T2 = (long)blockIdx.x * TT + tl;
-        if (T2 < total) {
-            const int c = (int)(T2 / p), i = (int)(T2 % p);
-            const size_t cols = 2 * (size_t)Bho;
-            const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
-#pragma unroll
-            for (int it = 0; it < E; ++it) {
-                const int f = f0 + L * it;
-                float2 z;
-                if (f == 0 || f == K / 2) {
-                    const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                    z.x = yg[(size_t)c * p + i];
-                    z.y = yg[((size_t)Bho + c) * p + i];
-                } else if (f < K / 2) {
-                    const float* yg = yop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * p;
-                    z.x = yg[i];
-                    z.y = yg[p + i];
-                } else {
-                    const float* yg = yop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bho + c) * 2 * p;
-                    z.x = yg[i];
-                    z.y = -yg[p + i];
-                }
-                zs[tl][f] = z;
+    if constexpr (VEC) {
+        constexpr int GROUPS = TT / 4;
+        for (int item = threadIdx.x; item < GROUPS * K; item += kThreads) {
+            const int grp = item % GROUPS, f = item / GROUPS;
+            const long T0 = (long)blockIdx.x * TT + grp * 4;
+            if (T0 >= total) continue;
+            const int c = (int)(T0 / p), i = (int)(T0 % p);
+            float4 za, zb;
+            if (f == 0 || f == K / 2) {
+                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                const float4 a = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
+                const float4 b = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
+                za = make_float4(a.x, b.x, a.y, b.y);
+                zb = make_float4(a.z, b.z, a.w, b.w);
+            } else {
+                const bool mirror = f > K / 2;
+                const int g = mirror ? K - f : f;
+                const float sgn = mirror ? -1.f : 1.f;
+                const float4* r = reinterpret_cast<const float4*>(yop + problem_offset(g + 1, real_sz, cplx_sz) +
+                                                                  ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i);
+                za = __ldg(r);
+                zb = __ldg(r + 1);
+                za.y *= sgn; za.w *= sgn; zb.y *= sgn; zb.w *= sgn;
             }
+            *reinterpret_cast<float4*>(&zs[f][grp * 4]) = za;
+            *reinterpret_cast<float4*>(&zs[f][grp * 4 + 2]) = zb;
+        }
+    } else {
+        for (int item = threadIdx.x; item < TT * K; item += kThreads) {
+            const int tl = item % TT, f = item / TT;
+            const long T2 = (long)blockIdx.x * TT + tl;
+            if (T2 >= total) continue;
+            const int c = (int)(T2 / p), i = (int)(T2 % p);
+            float2 z;
+            if (f == 0 || f == K / 2) {
+                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                z.x = __ldg(yg + (size_t)c * p + i);
+                z.y = __ldg(yg + ((size_t)Bho + c) * p + i);
+            } else if (f < K / 2) {
+                const float* yg = yop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * p + 2 * i;
+                z = __ldg(reinterpret_cast<const float2*>(yg));
+            } else {
+                const float* yg = yop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bho + c) * 2 * p + 2 * i;
+                z = __ldg(reinterpret_cast<const float2*>(yg));
+                z.y = -z.y;
+            }
+            zs[f][tl] = z;
         }
     }
     __syncthreads();
@@ -135,7 +210,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const fl
     const int f2 = lane_residue<K>(l);
     float2 v[E];
 #pragma unroll
-    for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[gi][f2 + L * f1] : make_float2(0.f, 0.f);
+    for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[f2 + L * f1][gi] : make_float2(0.f, 0.f);
     fft_inverse<K>(v, l, tw);
     if (!live) return;
     const int c = (int)(T / p), i = (int)(T % p);
@@ -156,7 +231,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const fl
 }
 
 // ---- launchers -------------------------------------------------------------------------------------
-template <typename T, typename F>
+template <typename F>
 static int dispatch_k(int k, F&& f) {
     switch (k) {
         case 4: return f(std::integral_constant<int, 4>{});
@@ -174,9 +249,13 @@ static int dispatch_k(int k, F&& f) {
 int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream) {
     const int q = L->geo.q, n = L->n;
     const long total = (long)ext.Bh * q;
+    if (xmode != 0 && (q % 8) != 0) {
+        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need q %% 8 == 0 (q=%d)", q);
+        return CIRC_ERR_UNSUPPORTED;
+    }
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
-        constexpr int TT = kThreads / FftShape<K>::L;
+        constexpr int TT = Tile<K>::TT;
         const unsigned blocks = (unsigned)((total + TT - 1) / TT);
         auto launch = [&](auto tin, auto mode) {
             using TIN = decltype(tin);
@@ -194,7 +273,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
         }
         return CIRC_OK;
     };
-    const int rc = dispatch_k<void>(L->geo.k, go);
+    const int rc = dispatch_k(L->geo.k, go);
     if (rc != CIRC_OK) return rc;
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
@@ -206,17 +285,23 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
     const long total = (long)ext.Bho * p;
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
-        constexpr int TT = kThreads / FftShape<K>::L;
+        constexpr int TT = Tile<K>::TT;
         const unsigned blocks = (unsigned)((total + TT - 1) / TT);
-        if (L->y_dtype == CIRC_BF16)
-            output_ifft_kernel<K, __nv_bfloat16><<<blocks, kThreads, 0, stream>>>(
-                yop, static_cast<__nv_bfloat16*>(y), L->tw256, L->bias_dev, L->relu, m, p, ext.Bo, ext.Bho, total);
-        else
-            output_ifft_kernel<K, float><<<blocks, kThreads, 0, stream>>>(yop, static_cast<float*>(y), L->tw256,
-                                                                          L->bias_dev, L->relu, m, p, ext.Bo, ext.Bho, total);
+        auto launch = [&](auto tout, auto vec) {
+            using TOUT = decltype(tout);
+            constexpr bool VEC = decltype(vec)::value;
+            output_ifft_kernel<K, TOUT, VEC><<<blocks, kThreads, 0, stream>>>(yop, static_cast<TOUT*>(y), L->tw256, L->bias_dev,
+                                                                             L->relu, m, p, ext.Bo, ext.Bho, total);
+        };
+        const bool vec = (p % 4) == 0;
+        if (L->y_dtype == CIRC_BF16) {
+            if (vec) launch(__nv_bfloat16{}, std::true_type{}); else launch(__nv_bfloat16{}, std::false_type{});
+        } else {
+            if (vec) launch(float{}, std::true_type{}); else launch(float{}, std::false_type{});
+        }
         return CIRC_OK;
     };
-    const int rc = dispatch_k<void>(L->geo.k, go);
+    const int rc = dispatch_k(L->geo.k, go);
     if (rc != CIRC_OK) return rc;
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
