@@ -153,28 +153,54 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const fl
     const size_t cols = 2 * (size_t)Bho;
     const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
 
+    // the bias of this thread's outputs is fetched now, long before the epilogue needs it
+    float bv[E];
+    {
+        const long Tb = (long)blockIdx.x * TT + threadIdx.x / L;
+#pragma unroll
+        for (int r = 0; r < E; ++r) bv[r] = 0.f;
+        if (bias && Tb < total) load_run<E>(bias + (int)(Tb % p) * K + E * (threadIdx.x % L), bv);
+    }
+
     if constexpr (VEC) {
+        // all loads of the tile are issued before the first one is used
         constexpr int GROUPS = TT / 4;
-        for (int item = threadIdx.x; item < GROUPS * K; item += kThreads) {
+        constexpr int ITERS = GROUPS * K / kThreads;
+        static_assert(GROUPS * K % kThreads == 0, "tile must divide evenly among the threads");
+        float4 r0[ITERS], r1[ITERS];
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int item = threadIdx.x + it * kThreads;
             const int grp = item % GROUPS, f = item / GROUPS;
             const long T0 = (long)blockIdx.x * TT + grp * 4;
+            r0[it] = r1[it] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (T0 >= total) continue;
             const int c = (int)(T0 / p), i = (int)(T0 % p);
-            float4 za, zb;
             if (f == 0 || f == K / 2) {
                 const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                const float4 a = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
-                const float4 b = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
-                za = make_float4(a.x, b.x, a.y, b.y);
-                zb = make_float4(a.z, b.z, a.w, b.w);
+                r0[it] = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
+                r1[it] = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
             } else {
                 const bool mirror = f > K / 2;
                 const int g = mirror ? K - f : f;
-                const float sgn = mirror ? -1.f : 1.f;
                 const float4* r = reinterpret_cast<const float4*>(yop + problem_offset(g + 1, real_sz, cplx_sz) +
                                                                   ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i);
-                za = __ldg(r);
-                zb = __ldg(r + 1);
+                r0[it] = __ldg(r);
+                r1[it] = __ldg(r + 1);
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            const int item = threadIdx.x + it * kThreads;
+            const int grp = item % GROUPS, f = item / GROUPS;
+            float4 za, zb;
+            if (f == 0 || f == K / 2) {
+                za = make_float4(r0[it].x, r1[it].x, r0[it].y, r1[it].y);
+                zb = make_float4(r0[it].z, r1[it].z, r0[it].w, r1[it].w);
+            } else {
+                const float sgn = f > K / 2 ? -1.f : 1.f;
+                za = r0[it];
+                zb = r1[it];
                 za.y *= sgn; za.w *= sgn; zb.y *= sgn; zb.w *= sgn;
             }
             *reinterpret_cast<float4*>(&zs[f][grp * 4]) = za;
@@ -218,9 +244,8 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const fl
     float re[E], im[E];
 #pragma unroll
     for (int r = 0; r < E; ++r) {
-        const float b = bias ? __ldg(bias + col + r) : 0.f;
-        re[r] = v[r].x + b;
-        im[r] = v[r].y + b;
+        re[r] = v[r].x + bv[r];
+        im[r] = v[r].y + bv[r];
         if (relu) {
             re[r] = fmaxf(re[r], 0.f);
             im[r] = fmaxf(im[r], 0.f);

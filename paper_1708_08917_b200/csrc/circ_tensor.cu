@@ -25,7 +25,7 @@ namespace circ {
 constexpr int kTcThreads = 192;
 constexpr int kTileCols = 128;            // MMA M: batch columns / pixels per tile
 constexpr int kKBlock = 64;               // bf16 elements per stage along K (one 128-byte swizzle row)
-constexpr int kStages = 4;
+constexpr int kMaxStages = 8;        // ring depth is chosen per launch (as many stages as shared memory holds)
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded wait: polls before giving up
 
 struct TcArgs {
@@ -41,6 +41,7 @@ struct TcArgs {
     int bn_real, bn_cplx;    // rows per tile (multiple of 16, <= 256)
     int nt_real, nt_cplx;    // row tiles per problem
     int ctas_real;           // CTAs that serve the two real problems
+    int stages;              // depth of the shared-memory ring (<= kMaxStages)
     long cols_out;           // V * Ho * Wo
 };
 
@@ -144,7 +145,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                    const __grid_constant__ CUtensorMap map_xhi_cplx, const __grid_constant__ CUtensorMap map_xlo_cplx,
                    TcArgs g) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) uint64_t full_bar[kStages], empty_bar[kStages], accum_bar;
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -191,7 +192,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     while ((int)tmem_cols < bn) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < g.stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
@@ -211,7 +212,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             int issued = 0;
             bool ok = true;
             for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % kStages, round = it / kStages;
+                const int s = it % g.stages, round = it / g.stages;
                 if (round > 0) ok = mbar_wait(&empty_bar[s], (round - 1) & 1, &abort_flag);
                 if (!ok) break;
                 const int kb = it % kblocks;
@@ -228,9 +229,9 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             }
             if (!ok) {
                 // drain: every copy that was issued must land before the CTA may go away
-                const int first = issued > kStages ? issued - kStages : 0;
+                const int first = issued > g.stages ? issued - g.stages : 0;
                 for (int it = first; it < issued; ++it) {
-                    const int s = it % kStages, round = it / kStages;
+                    const int s = it % g.stages, round = it / g.stages;
                     for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&full_bar[s], round & 1); ++spin) __nanosleep(64);
                 }
             }
@@ -241,7 +242,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             const uint32_t idesc = instr_desc(bn);
             bool ok = true;
             for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % kStages, round = it / kStages;
+                const int s = it % g.stages, round = it / g.stages;
                 ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
                 if (!ok) break;
                 tc_fence_after();
@@ -357,12 +358,19 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     g.tiles_h = (g.Ho + g.th - 1) / g.th;
     g.bn_real = round_up16(p) > 256 ? 256 : round_up16(p);
     g.bn_cplx = round_up16(2 * p) > 256 ? 256 : round_up16(2 * p);
-    g.nt_real = (p + g.bn_real - 1) / g.bn_real;
-    g.nt_cplx = (2 * p + g.bn_cplx - 1) / g.bn_cplx;
     g.cols_out = (long)g.V * g.Ho * g.Wo;
     const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
-    g.ctas_real = 2 * g.nt_real * sp_tiles;
-    const long ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles;
+    long ctas = 0;
+    for (;;) {
+        g.nt_real = (p + g.bn_real - 1) / g.bn_real;
+        g.nt_cplx = (2 * p + g.bn_cplx - 1) / g.bn_cplx;
+        g.ctas_real = 2 * g.nt_real * sp_tiles;
+        ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles;
+        // a grid that leaves most of the 148 SMs idle is split into narrower row tiles
+        if (ctas >= 100 || g.bn_cplx <= 32) break;
+        g.bn_cplx = round_up16(g.bn_cplx / 2);
+        if (g.bn_real > 32) g.bn_real = round_up16(g.bn_real / 2);
+    }
 
     // tensor maps.  A: [problem][row][part = tap*2 + (hi|lo)][Kq]
     CUtensorMap ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c;
@@ -405,7 +413,13 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     }
 
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const size_t smem = (size_t)kStages * (kTileCols * 128 + (size_t)bn_max * 128) + 1024;
+    const size_t stage_bytes = kTileCols * 128 + (size_t)bn_max * 128;
+    const int kq_max = 2 * q;
+    const int iters_max = g.npass * taps * ((kq_max + kKBlock - 1) / kKBlock);
+    g.stages = (int)((199 * 1024) / stage_bytes);
+    if (g.stages > kMaxStages) g.stages = kMaxStages;
+    if (g.stages > iters_max) g.stages = iters_max;
+    const size_t smem = (size_t)g.stages * stage_bytes + 1024;
     static thread_local int configured_device = -1;
     int dev = 0;
     cudaGetDevice(&dev);
