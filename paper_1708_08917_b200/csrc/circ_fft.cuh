@@ -134,14 +134,18 @@ __device__ __forceinline__ void fft_forward(float2 (&v)[FftShape<K>::E], int l, 
     if constexpr (L > 1) {
 #pragma unroll
         for (int s = L / 2; s >= 1; s >>= 1) {
+            // butterfly partner is lane l ^ s.  Lower lane: v + o.  Upper lane: (o - v) * w.
+            // Written branch-free: d = o + sign * v, then d * w' with w' = w (upper) or 1 (lower).
             const bool upper = (l & s) != 0;
-            const float2 w = tw[(l & (s - 1)) * (K / (2 * s))];
+            const float sign = upper ? -1.f : 1.f;
+            const float2 wt = tw[(l & (s - 1)) * (K / (2 * s))];
+            const float2 w = upper ? wt : make_float2(1.f, 0.f);
 #pragma unroll
             for (int r = 0; r < E; ++r) {
-                float2 o;
-                o.x = __shfl_xor_sync(0xffffffffu, v[r].x, s);
-                o.y = __shfl_xor_sync(0xffffffffu, v[r].y, s);
-                v[r] = upper ? cmul(csub(o, v[r]), w) : cadd(v[r], o);
+                float2 d;
+                d.x = fmaf(sign, v[r].x, __shfl_xor_sync(0xffffffffu, v[r].x, s));
+                d.y = fmaf(sign, v[r].y, __shfl_xor_sync(0xffffffffu, v[r].y, s));
+                v[r] = cmul(d, w);
             }
         }
         const int f2 = lane_residue<K>(l);
@@ -162,15 +166,16 @@ __device__ __forceinline__ void fft_inverse(float2 (&v)[FftShape<K>::E], int l, 
         for (int r = 1; r < E; ++r) v[r] = cmulc(v[r], tw[(r * f2) & (K - 1)]);
 #pragma unroll
         for (int s = 1; s < L; s <<= 1) {
+            // inverse of the forward butterfly: t = v * conj(w') ; lower: t + o, upper: o - t
             const bool upper = (l & s) != 0;
-            const float2 w = tw[(l & (s - 1)) * (K / (2 * s))];
+            const float sign = upper ? -1.f : 1.f;
+            const float2 wt = tw[(l & (s - 1)) * (K / (2 * s))];
+            const float2 w = upper ? wt : make_float2(1.f, 0.f);
 #pragma unroll
             for (int r = 0; r < E; ++r) {
-                const float2 t = upper ? cmulc(v[r], w) : v[r];
-                float2 o;
-                o.x = __shfl_xor_sync(0xffffffffu, t.x, s);
-                o.y = __shfl_xor_sync(0xffffffffu, t.y, s);
-                v[r] = upper ? csub(o, t) : cadd(t, o);
+                const float2 t = cmulc(v[r], w);
+                v[r].x = fmaf(sign, t.x, __shfl_xor_sync(0xffffffffu, t.x, s));
+                v[r].y = fmaf(sign, t.y, __shfl_xor_sync(0xffffffffu, t.y, s));
             }
         }
     }

@@ -32,8 +32,13 @@ __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
     const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&t);
 }
-// low-order part of a float32 value after its bfloat16 rounding has been taken out
-__device__ __forceinline__ float bf16_residual(float v) { return v - __bfloat162float(__float2bfloat16_rn(v)); }
+// Split two float32 values into bfloat16 high parts (returned, packed) and low parts (`lo_pair`):
+// v = hi + lo up to 2^-17 relative, which is what the three-pass tensor-core product needs.
+__device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& lo_pair) {
+    const uint32_t hi = bf16_pair(a, b);
+    lo_pair = bf16_pair(a - __uint_as_float(hi << 16), b - __uint_as_float(hi & 0xffff0000u));
+    return hi;
+}
 
 // ---- S1: x -> operand X ------------------------------------------------------------------------
 // One transform = (pair c, column block j).  A CTA takes TT = 256 / L consecutive transforms.
@@ -113,13 +118,14 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2
                 __nv_bfloat16* xg = xb + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
                 __nv_bfloat16* d0 = xg + (size_t)c * (NPART * q) + j;
                 __nv_bfloat16* d1 = xg + ((size_t)Bh + c) * (NPART * q) + j;
-                *reinterpret_cast<uint2*>(d0) = make_uint2(bf16_pair(za.x, za.z), bf16_pair(zb.x, zb.z));
-                *reinterpret_cast<uint2*>(d1) = make_uint2(bf16_pair(za.y, za.w), bf16_pair(zb.y, zb.w));
+                uint32_t l0, l1, l2, l3;
+                const uint32_t h0 = bf16_split_pair(za.x, za.z, l0), h1 = bf16_split_pair(zb.x, zb.z, l1);
+                const uint32_t h2 = bf16_split_pair(za.y, za.w, l2), h3 = bf16_split_pair(zb.y, zb.w, l3);
+                *reinterpret_cast<uint2*>(d0) = make_uint2(h0, h1);
+                *reinterpret_cast<uint2*>(d1) = make_uint2(h2, h3);
                 if constexpr (XMODE == 1) {
-                    *reinterpret_cast<uint2*>(d0 + q) = make_uint2(bf16_pair(bf16_residual(za.x), bf16_residual(za.z)),
-                                                                   bf16_pair(bf16_residual(zb.x), bf16_residual(zb.z)));
-                    *reinterpret_cast<uint2*>(d1 + q) = make_uint2(bf16_pair(bf16_residual(za.y), bf16_residual(za.w)),
-                                                                   bf16_pair(bf16_residual(zb.y), bf16_residual(zb.w)));
+                    *reinterpret_cast<uint2*>(d0 + q) = make_uint2(l0, l1);
+                    *reinterpret_cast<uint2*>(d1 + q) = make_uint2(l2, l3);
                 }
             } else {
                 const bool mirror = f > K / 2;
@@ -128,12 +134,11 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2
                 __nv_bfloat16* d = xb + problem_offset(g + 1, real_sz, cplx_sz) +
                                    ((size_t)(mirror ? Bh : 0) + c) * (NPART * 2 * q) + 2 * j;
                 const float i0 = sgn * za.y, i1 = sgn * za.w, i2 = sgn * zb.y, i3 = sgn * zb.w;
-                *reinterpret_cast<uint4*>(d) =
-                    make_uint4(bf16_pair(za.x, i0), bf16_pair(za.z, i1), bf16_pair(zb.x, i2), bf16_pair(zb.z, i3));
-                if constexpr (XMODE == 1)
-                    *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(
-                        bf16_pair(bf16_residual(za.x), bf16_residual(i0)), bf16_pair(bf16_residual(za.z), bf16_residual(i1)),
-                        bf16_pair(bf16_residual(zb.x), bf16_residual(i2)), bf16_pair(bf16_residual(zb.z), bf16_residual(i3)));
+                uint32_t l0, l1, l2, l3;
+                const uint32_t h0 = bf16_split_pair(za.x, i0, l0), h1 = bf16_split_pair(za.z, i1, l1);
+                const uint32_t h2 = bf16_split_pair(zb.x, i2, l2), h3 = bf16_split_pair(zb.z, i3, l3);
+                *reinterpret_cast<uint4*>(d) = make_uint4(h0, h1, h2, h3);
+                if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0, l1, l2, l3);
             }
         }
     }

@@ -419,6 +419,13 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     g.stages = (int)((199 * 1024) / stage_bytes);
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages > iters_max) g.stages = iters_max;
+    // many short CTAs (several waves): keep the ring small enough for three CTAs per SM, so that one
+    // CTA's load latency and epilogue overlap another's MMAs
+    if (ctas > 2 * 148) {
+        int fit = (int)((72 * 1024) / stage_bytes);
+        if (fit < 2) fit = 2;
+        if (g.stages > fit) g.stages = fit;
+    }
     const size_t smem = (size_t)g.stages * stage_bytes + 1024;
     static thread_local int configured_device = -1;
     int dev = 0;
