@@ -8,8 +8,10 @@
 //     the weight rows are its N dimension (TMEM columns), the contraction index is K;
 //   * operands are bfloat16, K-major, fetched by TMA (cp.async.bulk.tensor, 128-byte swizzle,
 //     no multicast) into a ring of shared-memory stages guarded by mbarriers;
-//   * a convolution tap is just a shifted TMA box over the (W, H, image) dimensions of X:
-//     out-of-image pixels are the zero fill of the copy (Eq. 6 with zero padding);
+//   * a convolution loads ONE input tile with its halo per K block -- a TMA box over the (W, H,
+//     image) dimensions of X whose out-of-image pixels are the zero fill of the copy (Eq. 6 with
+//     zero padding) -- and every filter tap multiplies a row-shifted view of that same tile
+//     (the MMA's row index is the flattened halo-tile pixel index, so a tap is a start offset);
 //   * float32 inputs use the split  a = a_hi + a_lo  (two bfloat16 values, 16 mantissa bits):
 //     the three products hi*hi + lo*hi + hi*lo are three passes over the same K range into
 //     the same float32 accumulator; bfloat16 inputs take the single hi*hi pass.
@@ -36,7 +38,10 @@ struct TcArgs {
     int npass;               // 3 (float32 inputs) or 1 (bfloat16 inputs)
     int W, H, V;             // input image (FC: W = columns, H = V = 1)
     int Wo, Ho;              // output image
-    int tw, th;              // spatial tile (tw * th <= 128)
+    int tw, th;              // output pixels per tile (tw wide, th high)
+    int pitch;               // input tile row pitch in pixels: tw + r - 1 (halo included)
+    int xrows;               // pixels of the input tile that the TMA box brings: pitch * (th + r - 1)
+    int xalloc;              // pixels reserved per stage for the input tile (covers every tap's 128-row view)
     int tiles_w, tiles_h;    // tiles per image
     int bn_real, bn_cplx;    // rows per tile (multiple of 16, <= 256)
     int nt_real, nt_cplx;    // row tiles per problem
@@ -127,6 +132,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     uint64_t d = 0;
     d |= (uint64_t)((saddr & 0x3FFFF) >> 4);        // start address, 16-byte units
+    // (row-shifted starts need no phase field: the swizzle is applied to the absolute shared-memory address)
     d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
     d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
     d |= (uint64_t)1 << 46;                          // descriptor version (sm_100)
@@ -181,13 +187,13 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     const CUtensorMap* map_xlo = real ? &map_xlo_real : &map_xlo_cplx;
 
     // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes)
-    const uint32_t x_bytes = kTileCols * 128, a_bytes = (uint32_t)bn * 128;
-    const uint32_t stage_bytes = x_bytes + a_bytes;
+    const uint32_t x_bytes = (uint32_t)g.xalloc * 128, a_bytes = (uint32_t)bn * 128;   // a_bytes: one tap's weight tile
+    const uint32_t stage_bytes = x_bytes + (uint32_t)g.taps * a_bytes;
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-    const uint32_t tx_bytes = (uint32_t)(g.tw * g.th) * 128 + a_bytes;
+    const uint32_t tx_bytes = (uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes;
 
     const int kblocks = (Kq + kKBlock - 1) / kKBlock;
-    const int iters = g.npass * g.taps * kblocks;
+    const int iters = g.npass * kblocks;   // one iteration = one K block of one pass, all taps
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < bn) tmem_cols <<= 1;
 
@@ -216,15 +222,16 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 if (round > 0) ok = mbar_wait(&empty_bar[s], (round - 1) & 1, &abort_flag);
                 if (!ok) break;
                 const int kb = it % kblocks;
-                const int tap = (it / kblocks) % g.taps;
-                const int pass = it / (kblocks * g.taps);
+                const int pass = it / kblocks;
                 const int a_part = pass == 1 ? 1 : 0, x_lo = pass == 2;
-                const int di = tap / g.r - g.pad, dj = tap % g.r - g.pad;
                 unsigned char* xs = ring + (size_t)s * stage_bytes;
                 unsigned char* as = xs + x_bytes;
                 mbar_expect_tx(&full_bar[s], tx_bytes);
-                tma_load_5d(xs, x_lo ? map_xlo : map_xhi, &full_bar[s], kb * kKBlock, wo0 + dj, ho0 + di, v, prob_in_kind);
-                tma_load_4d(as, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, row0, prob_in_kind);
+                // input tile with its halo: starts pad pixels before the output tile (negative and
+                // out-of-image coordinates read the zero fill)
+                tma_load_5d(xs, x_lo ? map_xlo : map_xhi, &full_bar[s], kb * kKBlock, wo0 - g.pad, ho0 - g.pad, v, prob_in_kind);
+                for (int tap = 0; tap < g.taps; ++tap)
+                    tma_load_4d(as + (size_t)tap * a_bytes, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, row0, prob_in_kind);
                 ++issued;
             }
             if (!ok) {
@@ -247,10 +254,18 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
-                const uint64_t da = smem_desc_sw128(xs), db = smem_desc_sw128(xs + x_bytes);
-#pragma unroll
-                for (int k4 = 0; k4 < kKBlock / 16; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
-                    tc_mma_bf16(tmem_base, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, (it > 0 || k4 > 0) ? 1u : 0u);
+                const int kb = it % kblocks;
+                const int krem = Kq - kb * kKBlock;                      // valid contraction entries in this block
+                const int ksteps = krem >= kKBlock ? kKBlock / 16 : (krem + 15) / 16;   // the rest is zero fill
+                for (int tap = 0; tap < g.taps; ++tap) {
+                    // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
+                    const uint32_t shift = (uint32_t)((tap / g.r) * g.pitch + (tap % g.r));
+                    const uint64_t da = smem_desc_sw128(xs + shift * 128u);
+                    const uint64_t db = smem_desc_sw128(xs + x_bytes + (uint32_t)tap * a_bytes);
+                    for (int k4 = 0; k4 < ksteps; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
+                        tc_mma_bf16(tmem_base, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc,
+                                    (it > 0 || tap > 0 || k4 > 0) ? 1u : 0u);
+                }
                 tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
             }
             if (ok) tc_commit(&accum_bar);  // accumulator complete
@@ -261,10 +276,10 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
         tc_fence_after();
         if (ok) {
             const int quarter = warp & 3;                 // a warp may only read its own 32 TMEM lanes
-            const int r = quarter * 32 + lane;            // row of the tile = pixel within the spatial tile
-            const int hh = r / g.tw, ww = r - hh * g.tw;
+            const int r = quarter * 32 + lane;            // row of the tile = flattened pixel index at the input pitch
+            const int hh = r / g.pitch, ww = r - hh * g.pitch;
             const int ho = ho0 + hh, wo = wo0 + ww;
-            const bool live = r < g.tw * g.th && ho < g.Ho && wo < g.Wo;
+            const bool live = hh < g.th && ww < g.tw && ho < g.Ho && wo < g.Wo;
             const size_t y_real = (size_t)g.cols_out * g.p;
             float* yrow = g.yop + problem_offset(prob, y_real, 2 * y_real) +
                           ((size_t)((size_t)v * g.Ho + ho) * g.Wo + wo) * Mg + row0;
@@ -351,13 +366,32 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     } else {
         g.W = g.Wo = 2 * ext.Bh; g.H = g.Ho = 1; g.V = 1;
     }
-    g.tw = g.Wo < kTileCols ? g.Wo : kTileCols;
-    g.th = kTileCols / g.tw;
+    const int halo = geo.r - 1;
+    g.tw = g.Wo < kTileCols - halo ? g.Wo : kTileCols - halo;
+    g.pitch = g.tw + halo;
+    g.th = (kTileCols - g.tw) / g.pitch + 1;          // (th - 1) * pitch + tw <= 128 MMA rows
     if (g.th > g.Ho) g.th = g.Ho;
+    g.xrows = g.pitch * (g.th + halo);
+    {
+        const int reach = halo * g.pitch + halo + kTileCols;   // last row any tap's 128-row view touches, plus one
+        const int need = g.xrows > reach ? g.xrows : reach;
+        g.xalloc = (need + 7) & ~7;                            // whole 1024-byte swizzle groups
+    }
     g.tiles_w = (g.Wo + g.tw - 1) / g.tw;
     g.tiles_h = (g.Ho + g.th - 1) / g.th;
     g.bn_real = round_up16(p) > 256 ? 256 : round_up16(p);
     g.bn_cplx = round_up16(2 * p) > 256 ? 256 : round_up16(2 * p);
+    {
+        // all taps' weight tiles of one K block share a stage with the input tile: narrow the row
+        // tile until a stage fits half of the shared memory (two stages), or all of it at worst
+        const long x_b = (long)g.xalloc * 128;
+        long room = 96 * 1024 - x_b;
+        if (room < (long)taps * 16 * 128) room = 198 * 1024 - x_b;
+        int cap = (int)(room / ((long)taps * 128)) & ~15;
+        if (cap < 16) cap = 16;
+        if (g.bn_real > cap) g.bn_real = cap;
+        if (g.bn_cplx > cap) g.bn_cplx = cap;
+    }
     g.cols_out = (long)g.V * g.Ho * g.Wo;
     const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
     long ctas = 0;
@@ -396,7 +430,7 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         cuuint64_t dims[5] = {(cuuint64_t)q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, 2};
         cuuint64_t str[4] = {(cuuint64_t)nsplit * q * 2, (cuuint64_t)g.W * nsplit * q * 2,
                              (cuuint64_t)g.H * g.W * nsplit * q * 2, (cuuint64_t)x_real_elems * 2};
-        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.tw, (cuuint32_t)g.th, 1, 1};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, (cuuint32_t)(g.th + halo), 1, 1};
         __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb);
         if ((rc = encode(&mxh_r, base, 5, dims, str, box)) != CIRC_OK) return rc;
         if ((rc = encode(&mxl_r, base + (nsplit == 2 ? q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
@@ -406,16 +440,20 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         cuuint64_t dims[5] = {(cuuint64_t)2 * q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, (cuuint64_t)nc};
         cuuint64_t str[4] = {(cuuint64_t)nsplit * 2 * q * 2, (cuuint64_t)g.W * nsplit * 2 * q * 2,
                              (cuuint64_t)g.H * g.W * nsplit * 2 * q * 2, (cuuint64_t)2 * x_real_elems * 2};
-        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.tw, (cuuint32_t)g.th, 1, 1};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, (cuuint32_t)(g.th + halo), 1, 1};
         __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb) + 2 * x_real_elems;
         if ((rc = encode(&mxh_c, base, 5, dims, str, box)) != CIRC_OK) return rc;
         if ((rc = encode(&mxl_c, base + (nsplit == 2 ? 2 * q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
     }
 
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const size_t stage_bytes = kTileCols * 128 + (size_t)bn_max * 128;
+    const size_t stage_bytes = (size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128;
+    if (stage_bytes + 1024 > 199 * 1024) {
+        set_error(CIRC_ERR_UNSUPPORTED, "filter taps x row tile do not fit one shared-memory stage (%zu bytes)", stage_bytes);
+        return CIRC_ERR_UNSUPPORTED;
+    }
     const int kq_max = 2 * q;
-    const int iters_max = g.npass * taps * ((kq_max + kKBlock - 1) / kKBlock);
+    const int iters_max = g.npass * ((kq_max + kKBlock - 1) / kKBlock);
     g.stages = (int)((199 * 1024) / stage_bytes);
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages > iters_max) g.stages = iters_max;
