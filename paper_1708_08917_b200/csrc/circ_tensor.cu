@@ -47,6 +47,7 @@ struct TcArgs {
     int nt_real, nt_cplx;    // row tiles per problem
     int ctas_real;           // CTAs that serve the two real problems
     int stages;              // depth of the shared-memory ring (<= kMaxStages)
+    long tiles;              // output tiles in total; CTAs walk them with a grid stride
     long cols_out;           // V * Ho * Wo
 };
 
@@ -145,64 +146,80 @@ __device__ __forceinline__ uint32_t instr_desc(int bn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
 }
 
+// Where a tile sits: which problem, which row tile, which spatial tile.
+struct TileCoord {
+    bool real;
+    int prob_in_kind, prob, row0, bn, Mg, Kq, v, ho0, wo0;
+};
+__device__ __forceinline__ TileCoord decode_tile(const TcArgs& g, long tile) {
+    TileCoord t;
+    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
+    long cta = tile;
+    t.real = cta < g.ctas_real;
+    int row_tile;
+    if (t.real) {
+        t.prob_in_kind = (int)(cta / ((long)g.nt_real * sp_tiles));
+        cta -= (long)t.prob_in_kind * g.nt_real * sp_tiles;
+        row_tile = (int)(cta / sp_tiles);
+        cta -= (long)row_tile * sp_tiles;
+    } else {
+        cta -= g.ctas_real;
+        t.prob_in_kind = (int)(cta / ((long)g.nt_cplx * sp_tiles));
+        cta -= (long)t.prob_in_kind * g.nt_cplx * sp_tiles;
+        row_tile = (int)(cta / sp_tiles);
+        cta -= (long)row_tile * sp_tiles;
+    }
+    t.v = (int)(cta / (g.tiles_h * g.tiles_w));
+    const int th_i = (int)((cta / g.tiles_w) % g.tiles_h), tw_i = (int)(cta % g.tiles_w);
+    t.ho0 = th_i * g.th;
+    t.wo0 = tw_i * g.tw;
+    t.bn = t.real ? g.bn_real : g.bn_cplx;
+    t.Mg = t.real ? g.p : 2 * g.p;
+    t.Kq = t.real ? g.q : 2 * g.q;
+    t.row0 = row_tile * t.bn;
+    t.prob = t.real ? t.prob_in_kind : 2 + t.prob_in_kind;
+    return t;
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The three roles run
+// ahead of one another: the producer keeps the shared-memory ring full across tile boundaries, the
+// MMA warp alternates between two accumulators in tensor memory, and the epilogue warps drain one
+// accumulator while the next tile's products are being formed in the other.
 __global__ void __launch_bounds__(kTcThreads, 1)
 contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_constant__ CUtensorMap map_a_cplx,
                    const __grid_constant__ CUtensorMap map_xhi_real, const __grid_constant__ CUtensorMap map_xlo_real,
                    const __grid_constant__ CUtensorMap map_xhi_cplx, const __grid_constant__ CUtensorMap map_xlo_cplx,
                    TcArgs g) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- which tile ---------------------------------------------------------------------------
-    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
-    int cta = blockIdx.x;
-    const bool real = cta < g.ctas_real;
-    int prob_in_kind, row_tile;
-    if (real) {
-        prob_in_kind = cta / (g.nt_real * sp_tiles);
-        cta -= prob_in_kind * g.nt_real * sp_tiles;
-        row_tile = cta / sp_tiles;
-        cta -= row_tile * sp_tiles;
-    } else {
-        cta -= g.ctas_real;
-        prob_in_kind = cta / (g.nt_cplx * sp_tiles);
-        cta -= prob_in_kind * g.nt_cplx * sp_tiles;
-        row_tile = cta / sp_tiles;
-        cta -= row_tile * sp_tiles;
-    }
-    const int v = cta / (g.tiles_h * g.tiles_w);
-    const int th_i = (cta / g.tiles_w) % g.tiles_h, tw_i = cta % g.tiles_w;
-    const int ho0 = th_i * g.th, wo0 = tw_i * g.tw;
-    const int bn = real ? g.bn_real : g.bn_cplx;
-    const int Mg = real ? g.p : 2 * g.p;
-    const int Kq = real ? g.q : 2 * g.q;
-    const int row0 = row_tile * bn;
-    const int prob = real ? prob_in_kind : 2 + prob_in_kind;
-    const CUtensorMap* map_a = real ? &map_a_real : &map_a_cplx;
-    const CUtensorMap* map_xhi = real ? &map_xhi_real : &map_xhi_cplx;
-    const CUtensorMap* map_xlo = real ? &map_xlo_real : &map_xlo_cplx;
-
-    // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes)
-    const uint32_t x_bytes = (uint32_t)g.xalloc * 128, a_bytes = (uint32_t)bn * 128;   // a_bytes: one tap's weight tile
-    const uint32_t stage_bytes = x_bytes + (uint32_t)g.taps * a_bytes;
+    // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes); every stage has room
+    // for the input tile and for all taps' weight tiles of the widest row tile
+    const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
+    const uint32_t x_bytes = (uint32_t)g.xalloc * 128;
+    const uint32_t stage_bytes = x_bytes + (uint32_t)g.taps * (uint32_t)bn_max * 128;
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
-    const uint32_t tx_bytes = (uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes;
-
-    const int kblocks = (Kq + kKBlock - 1) / kKBlock;
-    const int iters = g.npass * kblocks;   // one iteration = one K block of one pass, all taps
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < bn) tmem_cols <<= 1;
+    uint32_t acc_cols = 32;                      // columns of one accumulator
+    while ((int)acc_cols < bn_max) acc_cols <<= 1;
+    const uint32_t tmem_cols = 2 * acc_cols;     // two accumulators (<= 512 columns)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 4);         // one arrival per epilogue warp
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -215,79 +232,144 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     if (warp == 0) {
         // ---- TMA producer -----------------------------------------------------------------------
         if (lane == 0) {
-            int issued = 0;
-            bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % g.stages, round = it / g.stages;
-                if (round > 0) ok = mbar_wait(&empty_bar[s], (round - 1) & 1, &abort_flag);
-                if (!ok) break;
-                const int kb = it % kblocks;
-                const int pass = it / kblocks;
-                const int a_part = pass == 1 ? 1 : 0, x_lo = pass == 2;
-                unsigned char* xs = ring + (size_t)s * stage_bytes;
-                unsigned char* as = xs + x_bytes;
-                mbar_expect_tx(&full_bar[s], tx_bytes);
-                // input tile with its halo: starts pad pixels before the output tile (negative and
-                // out-of-image coordinates read the zero fill)
-                tma_load_5d(xs, x_lo ? map_xlo : map_xhi, &full_bar[s], kb * kKBlock, wo0 - g.pad, ho0 - g.pad, v, prob_in_kind);
-                for (int tap = 0; tap < g.taps; ++tap)
-                    tma_load_4d(as + (size_t)tap * a_bytes, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, row0, prob_in_kind);
-                ++issued;
+            // ring position: stage s, and the parity of the current trip around the ring.  Counters
+            // only -- no divisions on this thread's critical path.
+            int s = 0, issued = 0;
+            uint32_t par = 0;
+            bool wrapped = false, ok = true;
+            for (long tile = blockIdx.x; tile < g.tiles && ok; tile += gridDim.x) {
+                const TileCoord t = decode_tile(g, tile);
+                const CUtensorMap* map_a = t.real ? &map_a_real : &map_a_cplx;
+                const CUtensorMap* map_xhi = t.real ? &map_xhi_real : &map_xhi_cplx;
+                const CUtensorMap* map_xlo = t.real ? &map_xlo_real : &map_xlo_cplx;
+                const uint32_t a_bytes = (uint32_t)t.bn * 128;           // one tap's weight tile
+                const uint32_t tx_bytes = (uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes;
+                const int kblocks = (t.Kq + kKBlock - 1) / kKBlock;
+                // one iteration = one K block of one pass (hi*hi, lo*hi, hi*lo), all taps
+                for (int pass = 0; pass < g.npass && ok; ++pass) {
+                    const int a_part = pass == 1 ? 1 : 0;
+                    const CUtensorMap* map_x = pass == 2 ? map_xlo : map_xhi;
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        if (wrapped) ok = mbar_wait(&empty_bar[s], par ^ 1u, &abort_flag);
+                        if (!ok) break;
+                        unsigned char* xs = ring + (size_t)s * stage_bytes;
+                        unsigned char* as = xs + x_bytes;
+                        mbar_expect_tx(&full_bar[s], tx_bytes);
+                        // input tile with its halo: starts pad pixels before the output tile (negative and
+                        // out-of-image coordinates read the zero fill)
+                        tma_load_5d(xs, map_x, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v, t.prob_in_kind);
+                        for (int tap = 0; tap < g.taps; ++tap)
+                            tma_load_4d(as + (size_t)tap * a_bytes, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, t.row0,
+                                        t.prob_in_kind);
+                        if (issued < g.stages) ++issued;
+                        if (++s == g.stages) {
+                            s = 0;
+                            par ^= 1u;
+                            wrapped = true;
+                        }
+                    }
+                }
             }
             if (!ok) {
-                // drain: every copy that was issued must land before the CTA may go away
-                const int first = issued > g.stages ? issued - g.stages : 0;
-                for (int it = first; it < issued; ++it) {
-                    const int s = it % g.stages, round = it / g.stages;
-                    for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&full_bar[s], round & 1); ++spin) __nanosleep(64);
+                // drain: every copy that was issued must land before the CTA may go away.  The last
+                // `issued` stages, walking backwards from the current ring position.
+                int ds = s;
+                uint32_t dpar = par;
+                for (int n = 0; n < issued; ++n) {
+                    if (ds == 0) {
+                        ds = g.stages;
+                        dpar ^= 1u;
+                    }
+                    --ds;
+                    for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&full_bar[ds], dpar); ++spin) __nanosleep(64);
                 }
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer -------------------------------------------------------------------------
         if (lane == 0) {
-            const uint32_t idesc = instr_desc(bn);
-            bool ok = true;
-            for (int it = 0; it < iters && ok; ++it) {
-                const int s = it % g.stages, round = it / g.stages;
-                ok = mbar_wait(&full_bar[s], round & 1, &abort_flag);
+            int s = 0;
+            uint32_t par = 0;
+            int buf = 0;
+            uint32_t acc_par = 0;                 // parity of the accumulator pair's current use
+            bool acc_wrapped = false, ok = true;
+            for (long tile = blockIdx.x; tile < g.tiles && ok; tile += gridDim.x) {
+                const TileCoord t = decode_tile(g, tile);
+                const uint32_t a_bytes = (uint32_t)t.bn * 128;
+                const uint32_t idesc = instr_desc(t.bn);
+                const int kblocks = (t.Kq + kKBlock - 1) / kKBlock;
+                if (acc_wrapped) ok = mbar_wait(&acc_empty[buf], acc_par ^ 1u, &abort_flag);   // epilogue done with it
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
-                const int kb = it % kblocks;
-                const int krem = Kq - kb * kKBlock;                      // valid contraction entries in this block
-                const int ksteps = krem >= kKBlock ? kKBlock / 16 : (krem + 15) / 16;   // the rest is zero fill
-                for (int tap = 0; tap < g.taps; ++tap) {
-                    // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
-                    const uint32_t shift = (uint32_t)((tap / g.r) * g.pitch + (tap % g.r));
-                    const uint64_t da = smem_desc_sw128(xs + shift * 128u);
-                    const uint64_t db = smem_desc_sw128(xs + x_bytes + (uint32_t)tap * a_bytes);
-                    for (int k4 = 0; k4 < ksteps; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
-                        tc_mma_bf16(tmem_base, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc,
-                                    (it > 0 || tap > 0 || k4 > 0) ? 1u : 0u);
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_cols;
+                uint32_t accumulate = 0;
+                for (int pass = 0; pass < g.npass && ok; ++pass) {
+                    for (int kb = 0; kb < kblocks; ++kb) {
+                        ok = mbar_wait(&full_bar[s], par, &abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
+                        const int krem = t.Kq - kb * kKBlock;                    // valid contraction entries in this block
+                        if (g.taps == 1 && krem >= kKBlock) {
+                            // fully-connected fast path: one tile pair, four K steps of 16
+                            const uint64_t da = smem_desc_sw128(xs), db = smem_desc_sw128(xs + x_bytes);
+                            tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+                            tc_mma_bf16(d_tmem, da + 2, db + 2, idesc, 1u);
+                            tc_mma_bf16(d_tmem, da + 4, db + 4, idesc, 1u);
+                            tc_mma_bf16(d_tmem, da + 6, db + 6, idesc, 1u);
+                            accumulate = 1u;
+                        } else {
+                            const int ksteps = krem >= kKBlock ? kKBlock / 16 : (krem + 15) / 16;   // the rest is zero fill
+                            uint32_t b_addr = xs + x_bytes;
+                            for (int di = 0; di < g.r; ++di) {
+                                // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
+                                uint32_t a_addr = xs + (uint32_t)(di * g.pitch) * 128u;
+                                for (int dj = 0; dj < g.r; ++dj, a_addr += 128u, b_addr += a_bytes) {
+                                    const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
+                                    for (int k4 = 0; k4 < ksteps; ++k4) {   // 16 bf16 = 32 bytes per MMA step along K
+                                        tc_mma_bf16(d_tmem, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, accumulate);
+                                        accumulate = 1u;
+                                    }
+                                }
+                            }
+                        }
+                        tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
+                        if (++s == g.stages) {
+                            s = 0;
+                            par ^= 1u;
+                        }
+                    }
                 }
-                tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
+                if (ok) tc_commit(&acc_full[buf]);  // accumulator complete
+                if (buf == 1) {
+                    acc_par ^= 1u;
+                    acc_wrapped = true;
+                }
+                buf ^= 1;
             }
-            if (ok) tc_commit(&accum_bar);  // accumulator complete
         }
     } else {
         // ---- epilogue: TMEM -> registers -> Y[col][row] ------------------------------------------
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag));  // warp-uniform
-        tc_fence_after();
-        if (ok) {
-            const int quarter = warp & 3;                 // a warp may only read its own 32 TMEM lanes
-            const int r = quarter * 32 + lane;            // row of the tile = flattened pixel index at the input pitch
-            const int hh = r / g.pitch, ww = r - hh * g.pitch;
-            const int ho = ho0 + hh, wo = wo0 + ww;
+        const int quarter = warp & 3;                 // a warp may only read its own 32 TMEM lanes
+        const int r = quarter * 32 + lane;            // row of the tile = flattened pixel index at the input pitch
+        const int hh = r / g.pitch, ww = r - hh * g.pitch;
+        int buf = 0;
+        uint32_t acc_par = 0;
+        for (long tile = blockIdx.x; tile < g.tiles; tile += gridDim.x) {
+            const TileCoord t = decode_tile(g, tile);
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], acc_par, &abort_flag));  // warp-uniform
+            if (!ok) break;
+            tc_fence_after();
+            const int ho = t.ho0 + hh, wo = t.wo0 + ww;
             const bool live = hh < g.th && ww < g.tw && ho < g.Ho && wo < g.Wo;
             const size_t y_real = (size_t)g.cols_out * g.p;
-            float* yrow = g.yop + problem_offset(prob, y_real, 2 * y_real) +
-                          ((size_t)((size_t)v * g.Ho + ho) * g.Wo + wo) * Mg + row0;
-            for (int c0 = 0; c0 < bn; c0 += 32) {
+            float* yrow = g.yop + problem_offset(t.prob, y_real, 2 * y_real) +
+                          ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg + t.row0;
+            for (int c0 = 0; c0 < t.bn; c0 += 32) {
                 uint32_t acc[32];
-                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, acc);
+                tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * acc_cols + (uint32_t)c0, acc);
                 if (live) {
-                    if (row0 + c0 + 32 <= Mg && (Mg & 3) == 0) {
+                    if (t.row0 + c0 + 32 <= t.Mg && (t.Mg & 3) == 0) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 4)
                             *reinterpret_cast<float4*>(yrow + c0 + e) =
@@ -296,10 +378,16 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                     } else {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (row0 + c0 + e < Mg) yrow[c0 + e] = __uint_as_float(acc[e]);
+                            if (t.row0 + c0 + e < t.Mg) yrow[c0 + e] = __uint_as_float(acc[e]);
                     }
                 }
             }
+            // this accumulator may be overwritten by the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+            if (buf == 1) acc_par ^= 1u;
+            buf ^= 1;
         }
     }
 
@@ -457,12 +545,20 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     g.stages = (int)((199 * 1024) / stage_bytes);
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages > iters_max) g.stages = iters_max;
-    // many short CTAs (several waves): keep the ring small enough for three CTAs per SM, so that one
-    // CTA's load latency and epilogue overlap another's MMAs
-    if (ctas > 2 * 148) {
-        int fit = (int)((72 * 1024) / stage_bytes);
-        if (fit < 2) fit = 2;
+    // Persistent CTAs.  Short tiles (few ring iterations each) run two CTAs per SM, each with half of
+    // the shared memory, so that one CTA's start-up and tail overlap the other's steady state; two
+    // accumulators of bn_max columns per CTA keep both within the 512 columns of tensor memory.
+    int ctas_per_sm = 1;
+    if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && 2 * stage_bytes + 2048 <= 199 * 1024) {
+        ctas_per_sm = 2;
+        const int fit = (int)((99 * 1024 - 1024) / stage_bytes);
         if (g.stages > fit) g.stages = fit;
+    }
+    {
+        // the ring may run ahead into the next tile, so it is worth filling even when one tile needs fewer stages
+        int deep = (int)(((ctas_per_sm == 2 ? 98 : 198) * 1024) / stage_bytes);
+        if (deep > kMaxStages) deep = kMaxStages;
+        if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
     }
     const size_t smem = (size_t)g.stages * stage_bytes + 1024;
     static thread_local int configured_device = -1;
@@ -473,7 +569,9 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
                       CIRC_ERR_CUDA);
         configured_device = dev;
     }
-    contract_tc_kernel<<<(unsigned)ctas, kTcThreads, smem, stream>>>(ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
+    g.tiles = ctas;
+    const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
+    contract_tc_kernel<<<grid, kTcThreads, smem, stream>>>(ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
     return CIRC_OK;
