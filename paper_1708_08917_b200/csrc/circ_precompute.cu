@@ -70,16 +70,16 @@ __global__ void precompute_spectra_kernel(const float* __restrict__ w, float* __
                 a_f32[r1 + 2 * j + 1] = fre;
             }
         }
-        // split bfloat16 operand for the tensor-core contraction: [problem][row][tap*2 + (hi|lo)][Kq]
+        // split bfloat16 operand for the tensor-core contraction: [problem][row][hi|lo][tap][Kq]
         if (a_bf16) {
             const size_t rsz = (size_t)p * taps * 2 * q;  // one real problem, hi and lo
             const size_t b0 = problem_offset(prob, rsz, 4 * rsz);
             auto put = [&](size_t row, int kq, int kk, float val) {
                 const __nv_bfloat16 hi = __float2bfloat16_rn(val);
                 const __nv_bfloat16 lo = __float2bfloat16_rn(val - __bfloat162float(hi));
-                const size_t at = b0 + (row * taps * 2 + (size_t)tap * 2) * kq + kk;
+                const size_t at = b0 + (row * 2 * taps + (size_t)tap) * kq + kk;
                 a_bf16[at] = hi;
-                a_bf16[at + kq] = lo;
+                a_bf16[at + (size_t)taps * kq] = lo;
             };
             if (problem_is_real(prob)) {
                 put(i, q, j, fre);

@@ -13,8 +13,9 @@
 //     zero padding) -- and every filter tap multiplies a row-shifted view of that same tile
 //     (the MMA's row index is the flattened halo-tile pixel index, so a tap is a start offset);
 //   * float32 inputs use the split  a = a_hi + a_lo  (two bfloat16 values, 16 mantissa bits):
-//     the three products hi*hi + lo*hi + hi*lo are three passes over the same K range into
-//     the same float32 accumulator; bfloat16 inputs take the single hi*hi pass.
+//     a stage holds the hi and lo parts of both operands for one K block and the three products
+//     hi*hi + lo*hi + hi*lo go into the same float32 accumulator; bfloat16 inputs have the hi
+//     part only and take the single hi*hi product.
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue
 // (tcgen05.ld -> registers -> global).  Every wait is bounded: on expiry the CTA records an error
 // word, drains its copies, frees its tensor memory and returns.
@@ -35,7 +36,7 @@ struct TcArgs {
     int* status;
     int p, q, k, taps, r, pad;
     int nsplit;              // parts of X per column: 2 (hi, lo) or 1
-    int npass;               // 3 (float32 inputs) or 1 (bfloat16 inputs)
+    int npass;               // products per K block: 3 (float32 inputs) or 1 (bfloat16 inputs)
     int W, H, V;             // input image (FC: W = columns, H = V = 1)
     int Wo, Ho;              // output image
     int tw, th;              // output pixels per tile (tw wide, th high)
@@ -204,8 +205,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes); every stage has room
     // for the input tile and for all taps' weight tiles of the widest row tile
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const uint32_t x_bytes = (uint32_t)g.xalloc * 128;
-    const uint32_t stage_bytes = x_bytes + (uint32_t)g.taps * (uint32_t)bn_max * 128;
+    const uint32_t x_bytes = (uint32_t)g.xalloc * 128;                                    // one part (hi or lo) of the input tile
+    const uint32_t stage_bytes = (uint32_t)g.nsplit * (x_bytes + (uint32_t)g.taps * (uint32_t)bn_max * 128);
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     uint32_t acc_cols = 32;                      // columns of one accumulator
     while ((int)acc_cols < bn_max) acc_cols <<= 1;
@@ -243,24 +244,24 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 const CUtensorMap* map_xhi = t.real ? &map_xhi_real : &map_xhi_cplx;
                 const CUtensorMap* map_xlo = t.real ? &map_xlo_real : &map_xlo_cplx;
                 const uint32_t a_bytes = (uint32_t)t.bn * 128;           // one tap's weight tile
-                const uint32_t tx_bytes = (uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes;
+                const uint32_t tx_bytes = (uint32_t)g.nsplit * ((uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes);
                 const int kblocks = (t.Kq + kKBlock - 1) / kKBlock;
-                // one iteration = one K block of one pass (hi*hi, lo*hi, hi*lo), all taps
-                for (int pass = 0; pass < g.npass && ok; ++pass) {
-                    const int a_part = pass == 1 ? 1 : 0;
-                    const CUtensorMap* map_x = pass == 2 ? map_xlo : map_xhi;
+                // one iteration = one K block: input tile (hi [, lo]) and all taps' weight tiles (hi [, lo])
+                {
                     for (int kb = 0; kb < kblocks; ++kb) {
                         if (wrapped) ok = mbar_wait(&empty_bar[s], par ^ 1u, &abort_flag);
                         if (!ok) break;
                         unsigned char* xs = ring + (size_t)s * stage_bytes;
-                        unsigned char* as = xs + x_bytes;
+                        unsigned char* as = xs + (size_t)g.nsplit * x_bytes;
                         mbar_expect_tx(&full_bar[s], tx_bytes);
                         // input tile with its halo: starts pad pixels before the output tile (negative and
                         // out-of-image coordinates read the zero fill)
-                        tma_load_5d(xs, map_x, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v, t.prob_in_kind);
-                        for (int tap = 0; tap < g.taps; ++tap)
-                            tma_load_4d(as + (size_t)tap * a_bytes, map_a, &full_bar[s], kb * kKBlock, tap * 2 + a_part, t.row0,
+                        tma_load_5d(xs, map_xhi, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v, t.prob_in_kind);
+                        if (g.nsplit == 2)
+                            tma_load_5d(xs + x_bytes, map_xlo, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v,
                                         t.prob_in_kind);
+                        // one box brings every tap's weight tile, hi parts first, then lo parts: [part][row][128 B]
+                        tma_load_4d(as, map_a, &full_bar[s], kb * kKBlock, t.row0, 0, t.prob_in_kind);
                         if (issued < g.stages) ++issued;
                         if (++s == g.stages) {
                             s = 0;
@@ -303,32 +304,44 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_cols;
                 uint32_t accumulate = 0;
-                for (int pass = 0; pass < g.npass && ok; ++pass) {
+                {
                     for (int kb = 0; kb < kblocks; ++kb) {
                         ok = mbar_wait(&full_bar[s], par, &abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
+                        const uint32_t as = xs + (uint32_t)g.nsplit * x_bytes;
+                        const uint32_t a_lo = as + (uint32_t)g.taps * a_bytes;   // lo parts of the weight tiles
                         const int krem = t.Kq - kb * kKBlock;                    // valid contraction entries in this block
                         if (g.taps == 1 && krem >= kKBlock) {
-                            // fully-connected fast path: one tile pair, four K steps of 16
-                            const uint64_t da = smem_desc_sw128(xs), db = smem_desc_sw128(xs + x_bytes);
-                            tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
-                            tc_mma_bf16(d_tmem, da + 2, db + 2, idesc, 1u);
-                            tc_mma_bf16(d_tmem, da + 4, db + 4, idesc, 1u);
-                            tc_mma_bf16(d_tmem, da + 6, db + 6, idesc, 1u);
+                            // fully-connected fast path: four K steps of 16 per product
+                            const uint64_t dxh = smem_desc_sw128(xs), dah = smem_desc_sw128(as);
+                            tc_mma_bf16(d_tmem, dxh, dah, idesc, accumulate);
+                            tc_mma_bf16(d_tmem, dxh + 2, dah + 2, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dxh + 4, dah + 4, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dxh + 6, dah + 6, idesc, 1u);
+                            if (g.npass == 3) {
+                                const uint64_t dxl = smem_desc_sw128(xs + x_bytes), dal = smem_desc_sw128(a_lo);
+#pragma unroll
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxh + 2 * k4, dal + 2 * k4, idesc, 1u);
+#pragma unroll
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxl + 2 * k4, dah + 2 * k4, idesc, 1u);
+                            }
                             accumulate = 1u;
                         } else {
                             const int ksteps = krem >= kKBlock ? kKBlock / 16 : (krem + 15) / 16;   // the rest is zero fill
-                            uint32_t b_addr = xs + x_bytes;
-                            for (int di = 0; di < g.r; ++di) {
-                                // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
-                                uint32_t a_addr = xs + (uint32_t)(di * g.pitch) * 128u;
-                                for (int dj = 0; dj < g.r; ++dj, a_addr += 128u, b_addr += a_bytes) {
-                                    const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
-                                    for (int k4 = 0; k4 < ksteps; ++k4) {   // 16 bf16 = 32 bytes per MMA step along K
-                                        tc_mma_bf16(d_tmem, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, accumulate);
-                                        accumulate = 1u;
+                            for (int prod = 0; prod < g.npass; ++prod) {          // hi*hi, hi*lo(A), lo(X)*hi
+                                const uint32_t x_part = xs + (prod == 2 ? x_bytes : 0u);
+                                uint32_t b_addr = prod == 1 ? a_lo : as;
+                                for (int di = 0; di < g.r; ++di) {
+                                    // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
+                                    uint32_t a_addr = x_part + (uint32_t)(di * g.pitch) * 128u;
+                                    for (int dj = 0; dj < g.r; ++dj, a_addr += 128u, b_addr += a_bytes) {
+                                        const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
+                                        for (int k4 = 0; k4 < ksteps; ++k4) {   // 16 bf16 = 32 bytes per MMA step along K
+                                            tc_mma_bf16(d_tmem, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, accumulate);
+                                            accumulate = 1u;
+                                        }
                                     }
                                 }
                             }
@@ -472,10 +485,10 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     {
         // all taps' weight tiles of one K block share a stage with the input tile: narrow the row
         // tile until a stage fits half of the shared memory (two stages), or all of it at worst
-        const long x_b = (long)g.xalloc * 128;
+        const long x_b = (long)nsplit * g.xalloc * 128;
         long room = 96 * 1024 - x_b;
-        if (room < (long)taps * 16 * 128) room = 198 * 1024 - x_b;
-        int cap = (int)(room / ((long)taps * 128)) & ~15;
+        if (room < (long)nsplit * taps * 16 * 128) room = 198 * 1024 - x_b;
+        int cap = (int)(room / ((long)nsplit * taps * 128)) & ~15;
         if (cap < 16) cap = 16;
         if (g.bn_real > cap) g.bn_real = cap;
         if (g.bn_cplx > cap) g.bn_cplx = cap;
@@ -494,21 +507,22 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         if (g.bn_real > 32) g.bn_real = round_up16(g.bn_real / 2);
     }
 
-    // tensor maps.  A: [problem][row][part = tap*2 + (hi|lo)][Kq]
+    // tensor maps.  A: [problem][row][hi|lo][tap][Kq]; one box = (K block, bn rows, all taps of the parts in use)
     CUtensorMap ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c;
     const size_t a_real_elems = (size_t)p * taps * 2 * q;  // one real problem of A (hi and lo)
+    const cuuint32_t a_parts = (cuuint32_t)(nsplit * taps);
     int rc;
     {
-        cuuint64_t dims[4] = {(cuuint64_t)q, (cuuint64_t)taps * 2, (cuuint64_t)p, 2};
-        cuuint64_t str[3] = {(cuuint64_t)q * 2, (cuuint64_t)taps * 2 * q * 2, (cuuint64_t)a_real_elems * 2};
-        cuuint32_t box[4] = {kKBlock, 1, (cuuint32_t)g.bn_real, 1};
+        cuuint64_t dims[4] = {(cuuint64_t)q, (cuuint64_t)p, (cuuint64_t)taps * 2, 2};
+        cuuint64_t str[3] = {(cuuint64_t)taps * 2 * q * 2, (cuuint64_t)q * 2, (cuuint64_t)a_real_elems * 2};
+        cuuint32_t box[4] = {kKBlock, (cuuint32_t)g.bn_real, a_parts, 1};
         if ((rc = encode(&ma_r, L->a_bf16, 4, dims, str, box)) != CIRC_OK) return rc;
     }
     {
         const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
-        cuuint64_t dims[4] = {(cuuint64_t)2 * q, (cuuint64_t)taps * 2, (cuuint64_t)2 * p, (cuuint64_t)nc};
-        cuuint64_t str[3] = {(cuuint64_t)2 * q * 2, (cuuint64_t)taps * 2 * 2 * q * 2, (cuuint64_t)4 * a_real_elems * 2};
-        cuuint32_t box[4] = {kKBlock, 1, (cuuint32_t)g.bn_cplx, 1};
+        cuuint64_t dims[4] = {(cuuint64_t)2 * q, (cuuint64_t)2 * p, (cuuint64_t)taps * 2, (cuuint64_t)nc};
+        cuuint64_t str[3] = {(cuuint64_t)taps * 2 * 2 * q * 2, (cuuint64_t)2 * q * 2, (cuuint64_t)4 * a_real_elems * 2};
+        cuuint32_t box[4] = {kKBlock, (cuuint32_t)g.bn_cplx, a_parts, 1};
         if ((rc = encode(&ma_c, L->a_bf16 + 2 * a_real_elems, 4, dims, str, box)) != CIRC_OK) return rc;
     }
     // X: [problem][v][h][w][part][Kq]
@@ -535,13 +549,13 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     }
 
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const size_t stage_bytes = (size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128;
+    const size_t stage_bytes = (size_t)nsplit * ((size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128);
     if (stage_bytes + 1024 > 199 * 1024) {
         set_error(CIRC_ERR_UNSUPPORTED, "filter taps x row tile do not fit one shared-memory stage (%zu bytes)", stage_bytes);
         return CIRC_ERR_UNSUPPORTED;
     }
     const int kq_max = 2 * q;
-    const int iters_max = g.npass * ((kq_max + kKBlock - 1) / kKBlock);
+    const int iters_max = (kq_max + kKBlock - 1) / kKBlock;
     g.stages = (int)((199 * 1024) / stage_bytes);
     if (g.stages > kMaxStages) g.stages = kMaxStages;
     if (g.stages > iters_max) g.stages = iters_max;
@@ -549,14 +563,14 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     // the shared memory, so that one CTA's start-up and tail overlap the other's steady state; two
     // accumulators of bn_max columns per CTA keep both within the 512 columns of tensor memory.
     int ctas_per_sm = 1;
-    if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && 2 * stage_bytes + 2048 <= 199 * 1024) {
-        ctas_per_sm = 2;
-        const int fit = (int)((99 * 1024 - 1024) / stage_bytes);
-        if (g.stages > fit) g.stages = fit;
-    }
     {
+        const int fit2 = (int)((98 * 1024) / stage_bytes);   // stages per CTA when two CTAs share an SM
+        if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && fit2 >= 3) {
+            ctas_per_sm = 2;                                  // only when each CTA still gets a ring of three or more
+            if (g.stages > fit2) g.stages = fit2;
+        }
         // the ring may run ahead into the next tile, so it is worth filling even when one tile needs fewer stages
-        int deep = (int)(((ctas_per_sm == 2 ? 98 : 198) * 1024) / stage_bytes);
+        int deep = ctas_per_sm == 2 ? fit2 : (int)((198 * 1024) / stage_bytes);
         if (deep > kMaxStages) deep = kMaxStages;
         if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
     }
