@@ -152,32 +152,36 @@ struct TileCoord {
     bool real;
     int prob_in_kind, prob, row0, bn, Mg, Kq, v, ho0, wo0;
 };
+// 32-bit arithmetic only: the roles that call this are single threads on the critical path
+// (the host refuses launches with 2^31 tiles or more).
 __device__ __forceinline__ TileCoord decode_tile(const TcArgs& g, long tile) {
     TileCoord t;
-    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
-    long cta = tile;
-    t.real = cta < g.ctas_real;
-    int row_tile;
-    if (t.real) {
-        t.prob_in_kind = (int)(cta / ((long)g.nt_real * sp_tiles));
-        cta -= (long)t.prob_in_kind * g.nt_real * sp_tiles;
-        row_tile = (int)(cta / sp_tiles);
-        cta -= (long)row_tile * sp_tiles;
+    const unsigned sp_tiles = (unsigned)(g.V * g.tiles_h * g.tiles_w);
+    unsigned cta = (unsigned)tile;
+    t.real = cta < (unsigned)g.ctas_real;
+    if (!t.real) cta -= (unsigned)g.ctas_real;
+    const unsigned nt = (unsigned)(t.real ? g.nt_real : g.nt_cplx);
+    const unsigned pr = cta / sp_tiles;              // problem * nt + row tile
+    unsigned sp = cta - pr * sp_tiles;
+    unsigned row_tile;
+    if (nt == 1) {
+        t.prob_in_kind = (int)pr;
+        row_tile = 0;
     } else {
-        cta -= g.ctas_real;
-        t.prob_in_kind = (int)(cta / ((long)g.nt_cplx * sp_tiles));
-        cta -= (long)t.prob_in_kind * g.nt_cplx * sp_tiles;
-        row_tile = (int)(cta / sp_tiles);
-        cta -= (long)row_tile * sp_tiles;
+        t.prob_in_kind = (int)(pr / nt);
+        row_tile = pr - (unsigned)t.prob_in_kind * nt;
     }
-    t.v = (int)(cta / (g.tiles_h * g.tiles_w));
-    const int th_i = (int)((cta / g.tiles_w) % g.tiles_h), tw_i = (int)(cta % g.tiles_w);
-    t.ho0 = th_i * g.th;
-    t.wo0 = tw_i * g.tw;
+    const unsigned per_img = (unsigned)(g.tiles_h * g.tiles_w);
+    t.v = (int)(sp / per_img);
+    sp -= (unsigned)t.v * per_img;
+    const unsigned th_i = g.tiles_w == 1 ? sp : sp / (unsigned)g.tiles_w;
+    const unsigned tw_i = sp - th_i * (unsigned)g.tiles_w;
+    t.ho0 = (int)th_i * g.th;
+    t.wo0 = (int)tw_i * g.tw;
     t.bn = t.real ? g.bn_real : g.bn_cplx;
     t.Mg = t.real ? g.p : 2 * g.p;
     t.Kq = t.real ? g.q : 2 * g.q;
-    t.row0 = row_tile * t.bn;
+    t.row0 = (int)row_tile * t.bn;
     t.prob = t.real ? t.prob_in_kind : 2 + t.prob_in_kind;
     return t;
 }
@@ -582,6 +586,10 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024),
                       CIRC_ERR_CUDA);
         configured_device = dev;
+    }
+    if (ctas >= (1L << 31)) {
+        set_error(CIRC_ERR_SHAPE, "too many output tiles (%ld)", ctas);
+        return CIRC_ERR_SHAPE;
     }
     g.tiles = ctas;
     const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
