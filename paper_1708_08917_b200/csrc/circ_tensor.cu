@@ -190,6 +190,37 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// Issue the MMAs of one product (one X part against one A part) for all R x R taps of a K block.
+// R is a compile-time filter size so that the tap loops unroll and the single issuing thread
+// spends its time on tcgen05.mma, not on loop bookkeeping.  Descriptors differ only in their
+// start-address field (16-byte units): 8 units per tile row, a_step per tap, 2 per K step.
+template <int R, int KSTEPS>
+__device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step, uint64_t a_step,
+                                           uint32_t idesc, uint32_t& accumulate) {
+#pragma unroll
+    for (int di = 0; di < R; ++di) {
+#pragma unroll
+        for (int dj = 0; dj < R; ++dj) {
+            const uint64_t x = dx + (uint64_t)di * row_step + (uint64_t)(dj * 8);
+            const uint64_t w = da + (uint64_t)(di * R + dj) * a_step;
+            tc_mma_bf16(d_tmem, x, w, idesc, accumulate);
+#pragma unroll
+            for (int k4 = 1; k4 < KSTEPS; ++k4) tc_mma_bf16(d_tmem, x + 2 * k4, w + 2 * k4, idesc, 1u);
+            accumulate = 1u;
+        }
+    }
+}
+template <int R>
+__device__ __forceinline__ void issue_taps_k(int ksteps, uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step,
+                                             uint64_t a_step, uint32_t idesc, uint32_t& accumulate) {
+    switch (ksteps) {
+        case 1: issue_taps<R, 1>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        case 2: issue_taps<R, 2>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        case 3: issue_taps<R, 3>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        default: issue_taps<R, 4>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+    }
+}
+
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The three roles run
 // ahead of one another: the producer keeps the shared-memory ring full across tile boundaries, the
 // MMA warp alternates between two accumulators in tensor memory, and the epilogue warps drain one
@@ -334,16 +365,27 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                             accumulate = 1u;
                         } else {
                             const int ksteps = krem >= kKBlock ? kKBlock / 16 : (krem + 15) / 16;   // the rest is zero fill
+                            // descriptors differ only in their start-address field (16-byte units): build one per
+                            // operand part and step it -- 8 units per tile row, a_bytes / 16 per tap, 2 per K step
+                            const uint64_t dx_hi = smem_desc_sw128(xs), da_hi = smem_desc_sw128(as);
+                            const uint64_t dx_lo = dx_hi + (uint64_t)(x_bytes >> 4);
+                            const uint64_t da_lo = da_hi + (uint64_t)((uint32_t)g.taps * (a_bytes >> 4));
+                            const uint64_t tap_step = (uint64_t)(a_bytes >> 4), row_step = (uint64_t)(g.pitch * 8);
                             for (int prod = 0; prod < g.npass; ++prod) {          // hi*hi, hi*lo(A), lo(X)*hi
-                                const uint32_t x_part = xs + (prod == 2 ? x_bytes : 0u);
-                                uint32_t b_addr = prod == 1 ? a_lo : as;
-                                for (int di = 0; di < g.r; ++di) {
-                                    // tap (di, dj) reads the tile shifted by di rows and dj pixels: a start offset in rows
-                                    uint32_t a_addr = x_part + (uint32_t)(di * g.pitch) * 128u;
-                                    for (int dj = 0; dj < g.r; ++dj, a_addr += 128u, b_addr += a_bytes) {
-                                        const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
-                                        for (int k4 = 0; k4 < ksteps; ++k4) {   // 16 bf16 = 32 bytes per MMA step along K
-                                            tc_mma_bf16(d_tmem, da + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, accumulate);
+                                const uint64_t dx = prod == 2 ? dx_lo : dx_hi;
+                                const uint64_t da = prod == 1 ? da_lo : da_hi;
+                                if (g.r == 3) {
+                                    issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
+                                } else if (g.r == 1) {
+                                    issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
+                                } else {
+                                    uint64_t dx_row = dx, db = da;
+                                    for (int di = 0; di < g.r; ++di, dx_row += row_step) {
+                                        uint64_t dxx = dx_row;
+                                        for (int dj = 0; dj < g.r; ++dj, dxx += 8, db += tap_step) {
+                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate);
+                                            for (int k4 = 1; k4 < ksteps; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
+                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u);
                                             accumulate = 1u;
                                         }
                                     }
