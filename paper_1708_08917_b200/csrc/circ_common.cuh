@@ -111,6 +111,37 @@ void count_launches(long n);
     } while (0)
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with the "programmatic stream serialization"
+// attribute may be scheduled while its predecessor in the stream still runs, so that its launch
+// latency and set-up overlap the predecessor's work.  The contract every forward kernel keeps:
+//   pdl_wait()     before the first access to global memory: blocks until all earlier kernels have
+//                  finished and their writes are visible;
+//   pdl_trigger()  right after that wait: lets the next kernel be scheduled.  Triggering only after
+//                  the wait keeps at most one kernel queued behind the running one.
+// Both are no-ops when the kernel was launched without the attribute.  Measured on B200: the
+// attribute shortens back-to-back one-kernel forwards (the fused path) by about 5 %, but moves the
+// three-kernel path by -7 % .. +35 % depending on the shape, so only the fused kernel asks for it
+// (`dependent` = true below).
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Kernel launchers (one translation unit each).  All return a CIRC_* code and only enqueue.
 // ---------------------------------------------------------------------------------------------
 

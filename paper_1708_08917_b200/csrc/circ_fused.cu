@@ -57,6 +57,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = a.q;
     load_twiddles<K>(tw, a.tw256);
+    pdl_wait();     // x may come from the kernel before
+    pdl_trigger();
     __syncthreads();
 
     // ---- phase A: Z_j for all column blocks ----------------------------------------------------
@@ -275,7 +277,7 @@ static int launch_one(const FusedArgs& a, unsigned grid, size_t smem, cudaStream
                       CIRC_ERR_CUDA);
         configured_device = dev;
     }
-    fused_fc_kernel<K, PAIRS><<<grid, kFusedThreads, smem, stream>>>(a);
+    launch_kernel(true, fused_fc_kernel<K, PAIRS>, dim3(grid), dim3(kFusedThreads), smem, stream, a);
     return CIRC_OK;
 }
 

@@ -15,7 +15,7 @@
 
 namespace circ {
 
-constexpr int kThreads = 256;
+constexpr int kMaxThreads = 256;
 
 // Row length of the tile: TT transforms plus a pad that makes the register side conflict-free.
 // A half warp there is (16 / L) consecutive transforms x L bins, so rows must be 16 / L float2
@@ -23,7 +23,8 @@ constexpr int kThreads = 256;
 template <int K>
 struct Tile {
     static constexpr int L = FftShape<K>::L;
-    static constexpr int TT = kThreads / L;
+    static constexpr int NT = K >= 128 ? 256 : 128;   // threads per CTA: small CTAs fill the SMs more evenly
+    static constexpr int TT = NT / L;
     static constexpr int PAD = L == 1 ? 0 : (L == 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
     static constexpr int ROW = TT + PAD;
 };
@@ -47,13 +48,15 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
 // XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
 // Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
 template <int K, typename TIN, int XMODE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(Tile<K>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2* __restrict__ tw256, int n, int q,
                  int B, int Bh, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW;
+    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw, tw256);
+    pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
+    pdl_trigger();
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
@@ -148,13 +151,15 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2
 // One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
 template <int K, typename TOUT, bool VEC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(Tile<K>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const float2* __restrict__ tw256,
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW;
+    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw, tw256);
+    pdl_wait();     // Y is written by the contraction kernel before this one
+    pdl_trigger();
     const size_t cols = 2 * (size_t)Bho;
     const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
 
@@ -290,8 +295,8 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
         auto launch = [&](auto tin, auto mode) {
             using TIN = decltype(tin);
             constexpr int XMODE = decltype(mode)::value;
-            input_fft_kernel<K, TIN, XMODE><<<blocks, kThreads, 0, stream>>>(static_cast<const TIN*>(x), xop, L->tw256, n, q,
-                                                                            ext.B, ext.Bh, total);
+            launch_kernel(false, input_fft_kernel<K, TIN, XMODE>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, static_cast<const TIN*>(x), xop,
+                       static_cast<const float2*>(L->tw256), n, q, ext.B, ext.Bh, total);
         };
         const bool bf = L->x_dtype == CIRC_BF16;
         if (xmode == 0) {
@@ -320,8 +325,9 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
         auto launch = [&](auto tout, auto vec) {
             using TOUT = decltype(tout);
             constexpr bool VEC = decltype(vec)::value;
-            output_ifft_kernel<K, TOUT, VEC><<<blocks, kThreads, 0, stream>>>(yop, static_cast<TOUT*>(y), L->tw256, L->bias_dev,
-                                                                             L->relu, m, p, ext.Bo, ext.Bho, total);
+            launch_kernel(false, output_ifft_kernel<K, TOUT, VEC>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, yop, static_cast<TOUT*>(y),
+                       static_cast<const float2*>(L->tw256), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo,
+                       ext.Bho, total);
         };
         const bool vec = (p % 4) == 0;
         if (L->y_dtype == CIRC_BF16) {

@@ -264,6 +264,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    pdl_wait();     // X is written by the transform kernel before this one; Y may still be read by an earlier one
+    pdl_trigger();
 
     if (warp == 0) {
         // ---- TMA producer -----------------------------------------------------------------------
@@ -635,7 +637,7 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     }
     g.tiles = ctas;
     const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
-    contract_tc_kernel<<<grid, kTcThreads, smem, stream>>>(ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
+    launch_kernel(false, contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
     return CIRC_OK;
