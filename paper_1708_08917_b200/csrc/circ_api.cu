@@ -304,7 +304,7 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
     int variant = L->variant;
     if (variant == CIRC_VARIANT_AUTO)
         variant = fused_fc_supported(L, batch) && batch <= 8 ? CIRC_VARIANT_FUSED
-                  : (tensor_supported(L) && batch >= 32)      ? CIRC_VARIANT_TENSOR
+                  : tensor_supported(L)                       ? CIRC_VARIANT_TENSOR
                                                               : CIRC_VARIANT_STAGED;
     if (variant == CIRC_VARIANT_FUSED) {
         if (!fused_fc_supported(L, batch)) {
