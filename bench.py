@@ -340,24 +340,42 @@ def run_ours(args) -> int:
     value = world * wl.samples * args.steps / (ms_total * 1e-3)
     variant = circ.circ_last_variant(handles[0])
 
-    # Per-kernel device times over the same rotation: CUDA events around every kernel.  A spin
-    # kernel runs first so that the host queues the whole pass while the GPU is still busy and
-    # every kernel follows its start event without a launch gap.
-    prof_steps = min(args.steps, 4 * sets, 160)
-    for h in handles:
-        circ.circ_profile_begin(h)
-    torch.cuda._sleep(int(4e7))
-    for i in range(prof_steps):
-        forward(i % sets, stream)
-    torch.cuda.synchronize()
-    stage_ms, stage_n = [0.0] * 4, [0] * 4
-    for h in handles:
-        ms, cnt = circ.circ_profile_end(h)
-        stage_ms = [a + b for a, b in zip(stage_ms, ms)]
-        stage_n = [a + b for a, b in zip(stage_n, cnt)]
-    per_launch_us = {STAGES[i]: (1e3 * stage_ms[i] / stage_n[i] if stage_n[i] else None) for i in range(4)}
-    dom = max(range(4), key=lambda i: stage_ms[i])
-    dom_us = 1e3 * stage_ms[dom] / max(stage_n[dom], 1)
+    # Per-kernel device times, measured with the same CUDA events on the same rotating buffers: the
+    # rotation is captured again with ONE stage's kernel launched 1 + R times per forward (each of
+    # these kernels rewrites its own output from unchanged inputs), and the extra time per extra
+    # launch is that kernel's duration.  Unlike events around single launches this carries no
+    # per-event overhead, which would double the reading for kernels of a few microseconds.
+    def time_rotation(nrep):
+        g2, cs2 = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+        cs2.wait_stream(stream)
+        with torch.cuda.graph(g2, stream=cs2):
+            st = torch.cuda.current_stream()
+            for s_ in range(sets):
+                forward(s_, st)
+        g2.replay()
+        torch.cuda.synchronize()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for _ in range(nrep):
+            g2.replay()
+        a1.record(stream)
+        torch.cuda.synchronize()
+        return a0.elapsed_time(a1) / (nrep * sets)       # ms per forward
+
+    R = 3
+    nrep = max(3, min(200, args.steps // sets // 4))
+    used_stages = [3] if variant == circ.CIRC_VARIANT_FUSED else [0, 1, 2]
+    base_ms = time_rotation(nrep)
+    stage_ms = [0.0] * 4
+    for st_i in used_stages:
+        for h in handles:
+            circ.circ_set_stage_repeat(h, st_i, 1 + R)
+        stage_ms[st_i] = max(0.0, (time_rotation(nrep) - base_ms) / R)
+        for h in handles:
+            circ.circ_set_stage_repeat(h, st_i, 1)
+    per_launch_us = {STAGES[i]: (1e3 * stage_ms[i] if i in used_stages else None) for i in range(4)}
+    dom = max(used_stages, key=lambda i: stage_ms[i])
+    dom_us = max(1e3 * stage_ms[dom], 1e-3)
     peaks = measured_peaks()
     # Which roofline bounds the dominant kernel: the contraction is tensor-bound when its flops at the
     # tensor peak (a third of the bf16 peak for float32 inputs: three bf16 passes) take longer than the

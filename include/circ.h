@@ -190,6 +190,15 @@ CIRC_API int circ_last_variant(circ_handle h);
 CIRC_API int circ_profile_begin(circ_handle h);
 CIRC_API int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage);
 
+/*
+ * circ_set_stage_repeat -- timing aid: launch the kernel of `stage` (0..3, numbered as in
+ * circ_profile_end) `times` times back to back in every forward of this handle (default 1).  Each of
+ * these kernels overwrites its own output from unchanged inputs, so results do not change; the
+ * difference in forward time between `times` = 1 + R and `times` = 1, divided by R, is that kernel's
+ * duration without any per-event overhead.  Not meant for production calls.
+ */
+CIRC_API int circ_set_stage_repeat(circ_handle h, int stage, int times);
+
 /* circ_device_status -- waits for the device (blocking copy of the handle's error word) and
  * returns CIRC_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up on a bounded wait (TMA /
  * tensor-core pipeline barriers) since the last call; the word is cleared.  CIRC_OK otherwise. */

@@ -33,6 +33,7 @@ SIGNATURES = {
     "circ_profile_end": (_ci, [_vp, _vp, _vp]),
     "circ_fc_forward_noalloc": (_ci, [_vp, _vp, _vp, _ci, _vp]),
     "circ_noalloc_max_bytes": (_cl, []),
+    "circ_set_stage_repeat": (_ci, [_vp, _ci, _ci]),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -174,6 +175,11 @@ def circ_fc_forward_noalloc(h: int, x, y, batch: int, stream=None) -> None:
 
 def circ_noalloc_max_bytes() -> int:
     return load().circ_noalloc_max_bytes()
+
+
+def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:
+    """Timing aid: launch the kernel of ``stage`` ``times`` times per forward (results unchanged)."""
+    _check(load().circ_set_stage_repeat(h, stage, times))
 
 
 def circ_device_status(h: int) -> None:

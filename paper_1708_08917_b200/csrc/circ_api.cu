@@ -136,6 +136,7 @@ static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad
     L->geo = Geometry{m / k, n / k, k, taps, r, pad};
     L->x_dtype = L->y_dtype = (kind == 1 ? CIRC_BF16 : CIRC_F32);
     L->variant = CIRC_VARIANT_AUTO;
+    for (int st = 0; st < 4; ++st) L->repeat[st] = 1;
     if (cudaGetDevice(&L->device) != cudaSuccess) {
         set_error(CIRC_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
         delete L;
@@ -250,19 +251,23 @@ static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStr
         StageTimer t(L, 0, stream);
         // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16
         const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
-        if ((rc = launch_input_fft(L, x, xop, xmode, e, stream)) != CIRC_OK) return rc;
+        for (int rep = 0; rep < L->repeat[0]; ++rep)
+            if ((rc = launch_input_fft(L, x, xop, xmode, e, stream)) != CIRC_OK) return rc;
     }
     {
         StageTimer t(L, 1, stream);
-        if (tensor)
-            rc = launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
-        else
-            rc = launch_contract_fma(L, xop, yop, e, stream);
-        if (rc != CIRC_OK) return rc;
+        for (int rep = 0; rep < L->repeat[1]; ++rep) {
+            if (tensor)
+                rc = launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
+            else
+                rc = launch_contract_fma(L, xop, yop, e, stream);
+            if (rc != CIRC_OK) return rc;
+        }
     }
     {
         StageTimer t(L, 2, stream);
-        if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
+        for (int rep = 0; rep < L->repeat[2]; ++rep)
+            if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
     }
     L->last_variant = tensor ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
     return CIRC_OK;
@@ -313,7 +318,7 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
         }
         {
             StageTimer t(L, 3, s);
-            rc = launch_fused_fc(L, x, y, batch, s);
+            for (int rep = 0; rep < L->repeat[3] && rc == CIRC_OK; ++rep) rc = launch_fused_fc(L, x, y, batch, s);
         }
         if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
         return rc;
@@ -412,6 +417,16 @@ int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int 
     CIRC_CUDA_TRY(cudaMemcpyAsync(L->x_stage, x_host, xb, cudaMemcpyHostToDevice, s), CIRC_ERR_CUDA);
     if ((rc = circ_conv_forward(h, L->x_stage, L->y_stage, N, H, W, stream)) != CIRC_OK) return rc;
     CIRC_CUDA_TRY(cudaMemcpyAsync(y_host, L->y_stage, yb, cudaMemcpyDeviceToHost, s), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int circ_set_stage_repeat(circ_handle h, int stage, int times) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || stage < 0 || stage > 3 || times < 1 || times > 64) {
+        set_error(CIRC_ERR_ARG, "bad handle, stage %d not in [0,3] or times %d not in [1,64]", stage, times);
+        return CIRC_ERR_ARG;
+    }
+    L->repeat[stage] = times;
     return CIRC_OK;
 }
 

@@ -95,6 +95,7 @@ struct Layer {
     void* y_stage;
     size_t x_stage_bytes, y_stage_bytes;
     void* prof;         // per-kernel timing records while profiling is on, else nullptr
+    int repeat[4];      // how many times each stage's kernel is launched per forward (1; more only for timing)
 };
 
 // Thread-local error record.
