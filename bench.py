@@ -43,7 +43,14 @@ STAGE_SOURCE = {"input_fft": "circ_staged.cu", "output_ifft": "circ_staged.cu", 
 # DRAM traffic per launch from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum), keyed by
 # (workload, kernel).  Each entry is tied to the sha256 of the kernel's source file at capture time;
 # when the source has changed since, the figure is withheld (reported as null).
-NCU_TRAFFIC: dict = {}
+NCU_TRAFFIC: dict = {
+    # profiles/dram_traffic_cfg2_b256.md
+    ("cfg2_b256", "input_fft"): {"bytes_per_launch": 4215808, "source_sha256": "f32154192a5f6c8da8d9bf09a5d4ef653d1eed2d314939d6e7667fa56032fbb7"},
+    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6315264, "source_sha256": "c6adc151739c909a3a212573a2df8c9bbd68d348676b367a94ba1e544cc42799"},
+    ("cfg2_b256", "output_ifft"): {"bytes_per_launch": 4242304, "source_sha256": "f32154192a5f6c8da8d9bf09a5d4ef653d1eed2d314939d6e7667fa56032fbb7"},
+    # profiles/fused_fc_kernel_sweep_n16384_k4_b1.md (dram read + write of one launch)
+    ("sweep_n16384_k4_b1", "fused_fc"): {"bytes_per_launch": 272830720, "source_sha256": "d38c6938aa340e0d7c008b75e8aad08d1d861d234d4a866c3bab45b14c3acabd"},
+}
 
 
 @dataclass

@@ -247,6 +247,13 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     while ((int)acc_cols < bn_max) acc_cols <<= 1;
     const uint32_t tmem_cols = 2 * acc_cols;     // two accumulators (<= 512 columns)
 
+    if (warp == 0 && lane == 0) {
+        // start fetching the copy descriptors now; the first TMA would otherwise wait for them
+        const CUtensorMap* maps[6] = {&map_a_real, &map_a_cplx, &map_xhi_real, &map_xhi_cplx, &map_xlo_real, &map_xlo_cplx};
+#pragma unroll
+        for (int i = 0; i < 6; ++i)
+            if (i < 4 || g.nsplit == 2) asm volatile("prefetch.tensormap [%0];" ::"l"(maps[i]) : "memory");
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.stages; ++s) {
             mbar_init(&full_bar[s], 1);
