@@ -91,7 +91,6 @@ static void free_layer(Layer* L) {
     if (prev != L->device) cudaSetDevice(L->device);
     cudaFree(L->w_dev);
     cudaFree(L->bias_dev);
-    cudaFree(L->tw256);
     cudaFree(L->w_stream);
     cudaFree(L->a_f32);
     cudaFree(L->a_bf16);
@@ -147,20 +146,9 @@ static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad
         free_layer(L);
         return nullptr;
     }
-    // master twiddle table exp(-2 pi i n / 256) in double precision
-    float2 host_tw[256];
-    for (int i = 0; i < 256; ++i) {
-        const double ang = -2.0 * M_PI * (double)i / 256.0;
-        host_tw[i] = make_float2((float)cos(ang), (float)sin(ang));
-    }
-    host_tw[0] = make_float2(1.f, 0.f);
-    host_tw[64] = make_float2(0.f, -1.f);
-    host_tw[128] = make_float2(-1.f, 0.f);
-    host_tw[192] = make_float2(0.f, 1.f);
     const size_t a_real = (size_t)taps * (m / k) * (n / k);
     L->a_elems = 2 * a_real + (size_t)(k / 2 - 1) * 4 * a_real;
-    bool ok = cudaMalloc(&L->tw256, sizeof(host_tw)) == cudaSuccess &&
-              cudaMalloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
+    bool ok = cudaMalloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
               cudaMalloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&L->dev_status, sizeof(int)) == cudaSuccess;
@@ -170,8 +158,7 @@ static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad
         free_layer(L);
         return nullptr;
     }
-    if (cudaMemcpy(L->tw256, host_tw, sizeof(host_tw), cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemset(L->dev_status, 0, sizeof(int)) != cudaSuccess || launch_precompute(L, 0) != CIRC_OK ||
+    if (cudaMemset(L->dev_status, 0, sizeof(int)) != cudaSuccess || launch_precompute(L, 0) != CIRC_OK ||
         cudaDeviceSynchronize() != cudaSuccess) {
         set_error(CIRC_ERR_CUDA, "spectrum precompute failed: %s", cudaGetErrorString(cudaGetLastError()));
         free_layer(L);

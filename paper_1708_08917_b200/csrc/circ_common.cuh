@@ -61,11 +61,6 @@ struct Extent {
     int Nh;       // image pairs (CONV); FC: Bh
 };
 
-struct Epilogue {
-    const float* bias;  // device, length m, or nullptr
-    int relu;
-};
-
 // ---------------------------------------------------------------------------------------------
 // The layer object behind circ_handle.
 // ---------------------------------------------------------------------------------------------
@@ -82,7 +77,6 @@ struct Layer {
 
     float* w_dev;       // retained copy of the defining vectors [taps][p][q][k]
     float* bias_dev;    // [m] or nullptr
-    float2* tw256;      // exp(-2 pi i n / 256), n < 256
     float* w_stream;    // spectra for the fused kernel: [taps][p][q][k] packed half spectra
     float* a_f32;       // embedded float32 operand for the staged FMA contraction
     __nv_bfloat16* a_bf16;  // embedded bfloat16 operand (hi | lo split) for the tensor-core contraction

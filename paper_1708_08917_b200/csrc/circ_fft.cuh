@@ -185,7 +185,7 @@ __device__ __forceinline__ void fft_inverse(float2 (&v)[FftShape<K>::E], int l, 
 // the argument in units of pi, so the reduction is exact) rather than fetched: a table in global
 // memory would put one more dependent memory round trip at the head of every kernel.
 template <int K>
-__device__ __forceinline__ void load_twiddles(float2* tw, const float2* __restrict__ /*unused master table*/) {
+__device__ __forceinline__ void load_twiddles(float2* tw) {
     for (int n = threadIdx.x; n < K; n += blockDim.x) {
         float s, c;
         sincospif(-2.0f * (float)n / (float)K, &s, &c);

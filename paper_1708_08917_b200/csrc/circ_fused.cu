@@ -28,7 +28,6 @@ struct FusedArgs {
     const void* x;
     void* y;
     const float* w_stream;
-    const float2* tw256;
     const float* bias;
     int relu, x_bf16, y_bf16;
     int m, n, p, q, batch, Bh;
@@ -56,7 +55,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = a.q;
-    load_twiddles<K>(tw, a.tw256);
+    load_twiddles<K>(tw);
     pdl_wait();     // x may come from the kernel before
     pdl_trigger();
     __syncthreads();
@@ -296,7 +295,6 @@ int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStrea
     a.x = x;
     a.y = y;
     a.w_stream = L->w_stream;
-    a.tw256 = L->tw256;
     a.bias = L->bias_dev;
     a.relu = L->relu;
     a.x_bf16 = L->x_dtype == CIRC_BF16;

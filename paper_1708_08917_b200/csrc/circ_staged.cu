@@ -49,12 +49,12 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
 // Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
 template <int K, typename TIN, int XMODE>
 __global__ void __launch_bounds__(Tile<K>::NT)
-input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2* __restrict__ tw256, int n, int q,
+input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
                  int B, int Bh, long total) {
     constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
-    load_twiddles<K>(tw, tw256);
+    load_twiddles<K>(tw);
     pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
     pdl_trigger();
 
@@ -152,12 +152,12 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, const float2
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
 template <int K, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(Tile<K>::NT)
-output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const float2* __restrict__ tw256,
+output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
     constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
-    load_twiddles<K>(tw, tw256);
+    load_twiddles<K>(tw);
     pdl_wait();     // Y is written by the contraction kernel before this one
     pdl_trigger();
     const size_t cols = 2 * (size_t)Bho;
@@ -296,7 +296,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
             using TIN = decltype(tin);
             constexpr int XMODE = decltype(mode)::value;
             launch_kernel(false, input_fft_kernel<K, TIN, XMODE>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, static_cast<const TIN*>(x), xop,
-                       static_cast<const float2*>(L->tw256), n, q, ext.B, ext.Bh, total);
+                       n, q, ext.B, ext.Bh, total);
         };
         const bool bf = L->x_dtype == CIRC_BF16;
         if (xmode == 0) {
@@ -326,7 +326,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
             using TOUT = decltype(tout);
             constexpr bool VEC = decltype(vec)::value;
             launch_kernel(false, output_ifft_kernel<K, TOUT, VEC>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, yop, static_cast<TOUT*>(y),
-                       static_cast<const float2*>(L->tw256), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo,
+                       static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo,
                        ext.Bho, total);
         };
         const bool vec = (p % 4) == 0;
