@@ -89,6 +89,24 @@ def fc(w, x, bias=None, relu: bool = False, convention: int = 0) -> np.ndarray:
     return y
 
 
+def fc_backward(w, x, g, convention: int = 0, want_gx: bool = True, want_gw: bool = True):
+    """Gradients of ``L`` through ``a = W x`` given ``g = dL/da`` (``[B][m]``): returns ``(dL/dx [B][n], dL/dw [p][q][k])``.
+
+    This is what Algorithm 2 computes; here it is the chain rule on the dense expansion, in float64.
+    """
+    w = _d(w)
+    x = _d(x)
+    g = _d(g)
+    p, q, k = w.shape
+    batch, n = x.shape
+    assert n == q * k and g.shape == (batch, p * k)
+    gx = np.empty((batch, n), dtype=np.float64) if want_gx else None
+    gw = np.empty((p, q, k), dtype=np.float64) if want_gw else None
+    _load().circ_oracle_fc_backward(ctypes.c_int(p * k), ctypes.c_int(n), ctypes.c_int(k), ctypes.c_int(convention),
+                                    _ptr(w), _ptr(x), _ptr(g), ctypes.c_long(batch), _ptr(gx), _ptr(gw))
+    return gx, gw
+
+
 def conv(w, x, pad: int, bias=None, relu: bool = False, convention: int = 0) -> np.ndarray:
     """Eq. 6 with zero padding: ``w[r][r][p][q][k]``, ``x[N][H][W][C]`` -> ``y[N][Ho][Wo][P]``."""
     w = _d(w)

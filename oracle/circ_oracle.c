@@ -161,6 +161,56 @@ ORACLE_API void circ_oracle_conv_pixels(int c_out, int c_in, int r, int pad, int
 }
 
 /*
+ * FC backward pass (what Algorithm 2 computes with FFTs), written out from the chain rule on
+ * a = W x with the block-circulant W of Eq. 3:
+ *   dL/dx_j[c]  = sum_i sum_r  g_i[r] * W_ij[r][c]                     (= W^T g)
+ *   dL/dw_ij[t] = sum_b sum_{(r,c): W_ij[r][c] is w_ij[t]} g_i^b[r] * x_j^b[c]
+ * with g = dL/da ([batch][m]).  Every entry (r, c) of a block holds w_ij[d], d = (r - c) mod k
+ * (convention 0) or (c - r) mod k (convention 1), so dL/dw_ij[d] collects g[r] x[c] over that diagonal.
+ *   gx [batch][n] and gw [p][q][k] are outputs; either may be NULL to skip it.
+ */
+ORACLE_API void circ_oracle_fc_backward(int m, int n, int k, int convention, const double* w, const double* x,
+                                        const double* g, long batch, double* gx, double* gw) {
+    const int p = m / k, q = n / k;
+    if (gx) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (long b = 0; b < batch; ++b) {
+            for (int j = 0; j < q; ++j) {
+                for (int c = 0; c < k; ++c) {
+                    double acc = 0.0;
+                    for (int i = 0; i < p; ++i) {
+                        const double* wij = w + ((size_t)i * q + j) * k;
+                        const double* gi = g + (size_t)b * m + (size_t)i * k;
+                        for (int r = 0; r < k; ++r) acc += gi[r] * block_entry(wij, k, convention, r, c);
+                    }
+                    gx[(size_t)b * n + (size_t)j * k + c] = acc;
+                }
+            }
+        }
+    }
+    if (gw) {
+#pragma omp parallel for collapse(2) schedule(static)
+        for (int i = 0; i < p; ++i) {
+            for (int j = 0; j < q; ++j) {
+                double* out = gw + ((size_t)i * q + j) * k;
+                for (int d = 0; d < k; ++d) out[d] = 0.0;
+                for (long b = 0; b < batch; ++b) {
+                    const double* gi = g + (size_t)b * m + (size_t)i * k;
+                    const double* xj = x + (size_t)b * n + (size_t)j * k;
+                    for (int r = 0; r < k; ++r) {
+                        for (int c = 0; c < k; ++c) {
+                            int d = convention == 0 ? r - c : c - r;
+                            if (d < 0) d += k;
+                            out[d] += gi[r] * xj[c];
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+/*
  * Naive discrete Fourier transform, forward kernel exp(-2 pi i f t / k), unnormalised.
  * Used by tests only, for the eigenvalue closed form (the eigenvalues of a
  * circulant block are the DFT of its defining vector) and for the single-block

@@ -207,3 +207,67 @@ def test_conv_1x1_equals_fc():
 
 def test_threads_reported():
     assert oracle.threads() >= 1
+
+
+# ---- backward pass (Algorithm 2) -------------------------------------------------------------------
+
+@pytest.mark.parametrize("p,q,k,batch", [(1, 1, 4, 1), (2, 3, 4, 2), (3, 2, 8, 3), (2, 2, 3, 2), (1, 3, 1, 2), (4, 5, 16, 3)])
+def test_backward_against_dense_transposes(p, q, k, batch):
+    # dL/dx = g W (dense expansion from the library circulant) and dL/dw = the sum of g^T x over each diagonal
+    w = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((batch, q * k))
+    g = RNG.standard_normal((batch, p * k))
+    for conv in (0, 1):
+        dense = np.block([[scipy.linalg.circulant(w[i, j]) if conv == 0 else scipy.linalg.circulant(w[i, j]).T
+                           for j in range(q)] for i in range(p)])
+        gx, gw = oracle.fc_backward(w, x, g, convention=conv)
+        np.testing.assert_allclose(gx, g @ dense, atol=1e-12)
+        full = g.T @ x                                       # dL/dW of an unstructured layer, m x n
+        for i in range(p):
+            for j in range(q):
+                blk = full[i * k:(i + 1) * k, j * k:(j + 1) * k]
+                for d in range(k):
+                    # entries (r, c) with (r - c) mod k == d (convention 0) or (c - r) mod k == d (convention 1)
+                    r = np.arange(k)
+                    c = (r - d) % k if conv == 0 else (r + d) % k
+                    assert abs(gw[i, j, d] - blk[r, c].sum()) < 1e-11
+
+
+def test_backward_is_the_gradient_of_the_forward_oracle():
+    # L = sum(g * a) is linear in x and in w, so central differences of the FORWARD oracle are exact up to rounding
+    p, q, k, batch = 2, 3, 4, 2
+    w = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((batch, q * k))
+    g = RNG.standard_normal((batch, p * k))
+    for conv in (0, 1):
+        gx, gw = oracle.fc_backward(w, x, g, convention=conv)
+        loss = lambda ww, xx: float((g * oracle.fc(ww, xx, convention=conv)).sum())
+        h = 1e-3
+        for idx in [(0, 0), (1, 5), (0, 11), (1, 7)]:
+            xp, xm = x.copy(), x.copy()
+            xp[idx] += h
+            xm[idx] -= h
+            assert abs((loss(w, xp) - loss(w, xm)) / (2 * h) - gx[idx]) < 1e-9
+        for idx in [(0, 0, 0), (1, 2, 3), (0, 1, 2), (1, 0, 1)]:
+            wp, wm = w.copy(), w.copy()
+            wp[idx] += h
+            wm[idx] -= h
+            assert abs((loss(wp, x) - loss(wm, x)) / (2 * h) - gw[idx]) < 1e-9
+
+
+@pytest.mark.parametrize("k", [4, 8, 32])
+def test_backward_matches_algorithm_2_fft_form(k):
+    # Algorithm 2 with numpy's FFT: dL/dw_ij = IFFT(FFT(g_i) o FFT(x'_j)), x' the index-reversed x (FFT(x') = conj FFT(x));
+    # dL/dx_j += IFFT(FFT(g_i) o conj(FFT(w_ij)))  -- for the default convention
+    p, q, batch = 2, 2, 3
+    w = RNG.standard_normal((p, q, k))
+    x = RNG.standard_normal((batch, q * k))
+    g = RNG.standard_normal((batch, p * k))
+    gx, gw = oracle.fc_backward(w, x, g)
+    X = np.fft.fft(x.reshape(batch, q, k), axis=2)
+    G = np.fft.fft(g.reshape(batch, p, k), axis=2)
+    W = np.fft.fft(w, axis=2)
+    gw_fft = np.fft.ifft(np.einsum("bif,bjf->ijf", G, np.conj(X)), axis=2).real
+    gx_fft = np.fft.ifft(np.einsum("bif,ijf->bjf", G, np.conj(W)), axis=2).real.reshape(batch, q * k)
+    np.testing.assert_allclose(gw, gw_fft, atol=1e-10)
+    np.testing.assert_allclose(gx, gx_fft, atol=1e-10)
