@@ -145,6 +145,22 @@ CIRC_API int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_h
 CIRC_API int circ_fc_forward_noalloc(circ_handle h, const void* x, void* y, int batch, void* stream);
 CIRC_API long circ_noalloc_max_bytes(void);
 
+/*
+ * circ_fc_backward -- gradients through a = W x (Algorithm 2), float32 tensors only.
+ *   x       : DEVICE pointer, [batch][n], the input of the forward pass (needed for grad_w only)
+ *   grad_a  : DEVICE pointer, [batch][m], dL/da, the gradient with respect to the PRE-activation output
+ *             (Algorithm 2's input; a caller that used the fused ReLU masks dL/dy with y > 0 first)
+ *   grad_x  : DEVICE pointer, [batch][n], receives dL/dx = W^T grad_a; NULL to skip
+ *   grad_w  : DEVICE pointer, float32 [p][q][k], receives dL/dw_ij = IFFT(sum_b FFT(grad_a_i) o conj(FFT(x_j)))
+ *             (the paper's x' is x with reversed indices, whose transform is conj(FFT(x))); overwritten, not
+ *             accumulated; NULL to skip.  The gradient with respect to the bias is the column sum of grad_a and is
+ *             left to the caller.
+ * Honours circ_set_convention.  The first call builds the transposed layer W^T inside the handle (allocates
+ * and synchronises); later calls only enqueue on `stream`, growing the workspace when the batch grows.
+ */
+CIRC_API int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* grad_x, float* grad_w, int batch,
+                              void* stream);
+
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);
 

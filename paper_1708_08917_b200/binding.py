@@ -34,6 +34,7 @@ SIGNATURES = {
     "circ_fc_forward_noalloc": (_ci, [_vp, _vp, _vp, _ci, _vp]),
     "circ_noalloc_max_bytes": (_cl, []),
     "circ_set_stage_repeat": (_ci, [_vp, _ci, _ci]),
+    "circ_fc_backward": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _vp]),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -175,6 +176,11 @@ def circ_fc_forward_noalloc(h: int, x, y, batch: int, stream=None) -> None:
 
 def circ_noalloc_max_bytes() -> int:
     return load().circ_noalloc_max_bytes()
+
+
+def circ_fc_backward(h: int, x, grad_a, grad_x, grad_w, batch: int, stream=None) -> None:
+    """Enqueue ``grad_x = W^T grad_a`` and ``grad_w[p][q][k]`` (either may be None) from ``grad_a = dL/da``."""
+    _check(load().circ_fc_backward(h, _ptr(x), _ptr(grad_a), _ptr(grad_x), _ptr(grad_w), batch, _stream(stream)))
 
 
 def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:

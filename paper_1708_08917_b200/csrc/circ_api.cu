@@ -84,7 +84,7 @@ static int to_device(const float* src, size_t count, float** out) {
     return CIRC_OK;
 }
 
-static void free_layer(Layer* L) {
+void free_layer(Layer* L) {
     if (!L) return;
     int prev = -1;
     cudaGetDevice(&prev);
@@ -98,6 +98,7 @@ static void free_layer(Layer* L) {
     cudaFree(L->dev_status);
     cudaFree(L->x_stage);
     cudaFree(L->y_stage);
+    if (L->transposed) free_layer(L->transposed);
     if (L->prof) {
         for (auto& r : static_cast<Profiler*>(L->prof)->recs) {
             cudaEventDestroy(r.start);
@@ -110,7 +111,7 @@ static void free_layer(Layer* L) {
     delete L;
 }
 
-static Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const float* w) {
+Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const float* w) {
     if (!w) {
         set_error(CIRC_ERR_ARG, "w is NULL");
         return nullptr;
@@ -173,7 +174,7 @@ static size_t workspace_need(const Layer* L, const Extent& e) {
     return (xin + yout) * sizeof(float) + 512;
 }
 
-static int ensure_workspace(Layer* L, size_t need) {
+int ensure_workspace(Layer* L, size_t need) {
     if (L->ws_bytes >= need) return CIRC_OK;
     if (L->ws) cudaFree(L->ws);  // implicit synchronisation: earlier forwards have finished with it
     L->ws = nullptr;
@@ -526,6 +527,10 @@ int circ_set_convention(circ_handle h, int convention) {
     if (convention == L->convention) return CIRC_OK;
     CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
     L->convention = convention;
+    if (L->transposed) {
+        free_layer(L->transposed);   // rebuilt on the next backward call
+        L->transposed = nullptr;
+    }
     int rc = launch_precompute(L, 0);
     if (rc != CIRC_OK) return rc;
     CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);

@@ -90,7 +90,13 @@ struct Layer {
     size_t x_stage_bytes, y_stage_bytes;
     void* prof;         // per-kernel timing records while profiling is on, else nullptr
     int repeat[4];      // how many times each stage's kernel is launched per forward (1; more only for timing)
+    Layer* transposed;  // the n x m layer W^T (built on first use by the backward pass), or nullptr
 };
+
+// Layer life cycle and workspace (circ_api.cu).
+Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const float* w);
+void free_layer(Layer* L);
+int ensure_workspace(Layer* L, size_t bytes);
 
 // Thread-local error record.
 void set_error(int code, const char* fmt, ...);
