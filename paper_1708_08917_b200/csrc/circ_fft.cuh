@@ -29,12 +29,17 @@
 
 namespace circ {
 
-template <int K>
+// EMAX bounds the points per lane.  16 keeps the shuffle count low (throughput); a small EMAX spreads a
+// transform over more lanes, which shortens every thread's dependent chain when the whole problem is
+// too small to fill the machine (latency).
+template <int K, int EMAX = 16>
 struct FftShape {
     static_assert(K >= 4 && K <= 256 && (K & (K - 1)) == 0, "block size must be a power of two in [4,256]");
-    static constexpr int E = K < 16 ? K : 16;  // points per lane
-    static constexpr int L = K / E;            // lanes per transform
-    static constexpr int LOG_L = L == 1 ? 0 : L == 2 ? 1 : L == 4 ? 2 : L == 8 ? 3 : 4;
+    static_assert(EMAX == 4 || EMAX == 8 || EMAX == 16, "points per lane: 4, 8 or 16");
+    static constexpr int E = K < EMAX ? K : EMAX;  // points per lane
+    static constexpr int L = K / E;                // lanes per transform
+    static_assert(L <= 32, "a transform must fit one warp");
+    static constexpr int LOG_L = L == 1 ? 0 : L == 2 ? 1 : L == 4 ? 2 : L == 8 ? 3 : L == 16 ? 4 : 5;
 };
 
 __device__ __forceinline__ float2 cadd(float2 a, float2 b) { return make_float2(a.x + b.x, a.y + b.y); }
@@ -116,9 +121,9 @@ __device__ __forceinline__ void fft_registers(float2 (&v)[E]) {
 }
 
 // Position of this lane's frequency residue: lane s of an L-lane group holds f2 = bitrev_L(s).
-template <int K>
+template <int K, int EMAX = 16>
 __device__ __forceinline__ int lane_residue(int lane_in_group) {
-    constexpr int LOG_L = FftShape<K>::LOG_L;
+    constexpr int LOG_L = FftShape<K, EMAX>::LOG_L;
     if constexpr (LOG_L == 0) {
         return 0;
     } else {
@@ -128,9 +133,9 @@ __device__ __forceinline__ int lane_residue(int lane_in_group) {
 
 // Forward transform.  In: v[r] = z[E*l + r].  Out: v[f1] = Z[f2 + L*f1], f2 = lane_residue(l).
 // tw[n] = exp(-2 pi i n / K), n < K (shared or global memory).  Every lane of the warp must call.
-template <int K>
-__device__ __forceinline__ void fft_forward(float2 (&v)[FftShape<K>::E], int l, const float2* __restrict__ tw) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L;
+template <int K, int EMAX = 16>
+__device__ __forceinline__ void fft_forward(float2 (&v)[FftShape<K, EMAX>::E], int l, const float2* __restrict__ tw) {
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L;
     if constexpr (L > 1) {
 #pragma unroll
         for (int s = L / 2; s >= 1; s >>= 1) {
@@ -148,7 +153,7 @@ __device__ __forceinline__ void fft_forward(float2 (&v)[FftShape<K>::E], int l, 
                 v[r] = cmul(d, w);
             }
         }
-        const int f2 = lane_residue<K>(l);
+        const int f2 = lane_residue<K, EMAX>(l);
 #pragma unroll
         for (int r = 1; r < E; ++r) v[r] = cmul(v[r], tw[(r * f2) & (K - 1)]);
     }
@@ -156,12 +161,12 @@ __device__ __forceinline__ void fft_forward(float2 (&v)[FftShape<K>::E], int l, 
 }
 
 // Inverse transform (unnormalised).  In: v[f1] = Y[f2 + L*f1].  Out: v[r] = K * y[E*l + r].
-template <int K>
-__device__ __forceinline__ void fft_inverse(float2 (&v)[FftShape<K>::E], int l, const float2* __restrict__ tw) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L;
+template <int K, int EMAX = 16>
+__device__ __forceinline__ void fft_inverse(float2 (&v)[FftShape<K, EMAX>::E], int l, const float2* __restrict__ tw) {
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L;
     fft_registers<E, true>(v);
     if constexpr (L > 1) {
-        const int f2 = lane_residue<K>(l);
+        const int f2 = lane_residue<K, EMAX>(l);
 #pragma unroll
         for (int r = 1; r < E; ++r) v[r] = cmulc(v[r], tw[(r * f2) & (K - 1)]);
 #pragma unroll

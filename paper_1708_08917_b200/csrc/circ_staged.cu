@@ -15,17 +15,16 @@
 
 namespace circ {
 
-constexpr int kMaxThreads = 256;
 
 // Row length of the tile: TT transforms plus a pad that makes the register side conflict-free.
 // A half warp there is (16 / L) consecutive transforms x L bins, so rows must be 16 / L float2
 // apart modulo the 16 eight-byte banks.
-template <int K>
+template <int K, int EMAX>
 struct Tile {
-    static constexpr int L = FftShape<K>::L;
-    static constexpr int NT = K >= 128 ? 256 : 128;   // threads per CTA: small CTAs fill the SMs more evenly
+    static constexpr int L = FftShape<K, EMAX>::L;
+    static constexpr int NT = (K >= 128 && EMAX == 16) ? 256 : 128;   // threads per CTA: small CTAs fill the SMs more evenly
     static constexpr int TT = NT / L;
-    static constexpr int PAD = L == 1 ? 0 : (L == 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
+    static constexpr int PAD = L == 1 ? 0 : (L >= 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
     static constexpr int ROW = TT + PAD;
 };
 
@@ -47,11 +46,12 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
 // XMODE 1: bfloat16 operand [problem][col][hi | lo][Kq]            (tensor cores, float32 input split in two)
 // XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
 // Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
-template <int K, typename TIN, int XMODE>
-__global__ void __launch_bounds__(Tile<K>::NT)
+template <int K, int EMAX, typename TIN, int XMODE>
+__global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
                  int B, int Bh, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW,
+                  kThreads = Tile<K, EMAX>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw);
@@ -74,8 +74,8 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
         for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
     }
     __syncthreads();  // twiddles ready
-    fft_forward<K>(v, l, tw);
-    const int f2 = lane_residue<K>(l);
+    fft_forward<K, EMAX>(v, l, tw);
+    const int f2 = lane_residue<K, EMAX>(l);
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
@@ -150,11 +150,12 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
 // One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
-template <int K, typename TOUT, bool VEC>
-__global__ void __launch_bounds__(Tile<K>::NT)
+template <int K, int EMAX, typename TOUT, bool VEC>
+__global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = Tile<K>::TT, ROW = Tile<K>::ROW, kThreads = Tile<K>::NT;
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW,
+                  kThreads = Tile<K, EMAX>::NT;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw);
@@ -243,11 +244,11 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
     const bool live = T < total;
-    const int f2 = lane_residue<K>(l);
+    const int f2 = lane_residue<K, EMAX>(l);
     float2 v[E];
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[f2 + L * f1][gi] : make_float2(0.f, 0.f);
-    fft_inverse<K>(v, l, tw);
+    fft_inverse<K, EMAX>(v, l, tw);
     if (!live) return;
     const int c = (int)(T / p), i = (int)(T % p);
     const int col = i * K + E * l;
@@ -281,6 +282,17 @@ static int dispatch_k(int k, F&& f) {
     return CIRC_ERR_SHAPE;
 }
 
+// Points per lane for a launch: 16 (fewest shuffles) when the transforms fill the machine, otherwise 4
+// (8 for k = 256), which quarters every thread's dependent chain for problems that are latency-bound.
+template <int K>
+struct SmallShape {
+    static constexpr int EMAX = K <= 8 ? 16 : (K <= 128 ? 4 : 8);   // k = 4, 8 already sit in one lane
+};
+static bool latency_bound(long transforms, int k) {
+    const long warps_at_16 = transforms * (k < 16 ? 1 : k / 16) / 32;
+    return k >= 16 && warps_at_16 < 148L * 8;
+}
+
 int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream) {
     const int q = L->geo.q, n = L->n;
     const long total = (long)ext.Bh * q;
@@ -288,24 +300,30 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
         set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need q %% 8 == 0 (q=%d)", q);
         return CIRC_ERR_UNSUPPORTED;
     }
+    const bool small = latency_bound(total, L->geo.k);
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
-        constexpr int TT = Tile<K>::TT;
-        const unsigned blocks = (unsigned)((total + TT - 1) / TT);
-        auto launch = [&](auto tin, auto mode) {
-            using TIN = decltype(tin);
-            constexpr int XMODE = decltype(mode)::value;
-            launch_kernel(false, input_fft_kernel<K, TIN, XMODE>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, static_cast<const TIN*>(x), xop,
-                       n, q, ext.B, ext.Bh, total);
+        auto with_shape = [&](auto ec) {
+            constexpr int EMAX = decltype(ec)::value;
+            constexpr int TT = Tile<K, EMAX>::TT;
+            const unsigned blocks = (unsigned)((total + TT - 1) / TT);
+            auto launch = [&](auto tin, auto mode) {
+                using TIN = decltype(tin);
+                constexpr int XMODE = decltype(mode)::value;
+                launch_kernel(false, input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream,
+                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total);
+            };
+            const bool bf = L->x_dtype == CIRC_BF16;
+            if (xmode == 0) {
+                if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 0>{}); else launch(float{}, std::integral_constant<int, 0>{});
+            } else if (xmode == 1) {
+                if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 1>{}); else launch(float{}, std::integral_constant<int, 1>{});
+            } else {
+                if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 2>{}); else launch(float{}, std::integral_constant<int, 2>{});
+            }
         };
-        const bool bf = L->x_dtype == CIRC_BF16;
-        if (xmode == 0) {
-            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 0>{}); else launch(float{}, std::integral_constant<int, 0>{});
-        } else if (xmode == 1) {
-            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 1>{}); else launch(float{}, std::integral_constant<int, 1>{});
-        } else {
-            if (bf) launch(__nv_bfloat16{}, std::integral_constant<int, 2>{}); else launch(float{}, std::integral_constant<int, 2>{});
-        }
+        if (small) with_shape(std::integral_constant<int, SmallShape<K>::EMAX>{});
+        else with_shape(std::integral_constant<int, 16>{});
         return CIRC_OK;
     };
     const int rc = dispatch_k(L->geo.k, go);
@@ -318,23 +336,28 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
 int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream) {
     const int p = L->geo.p, m = L->m;
     const long total = (long)ext.Bho * p;
+    const bool small = latency_bound(total, L->geo.k);
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
-        constexpr int TT = Tile<K>::TT;
-        const unsigned blocks = (unsigned)((total + TT - 1) / TT);
-        auto launch = [&](auto tout, auto vec) {
-            using TOUT = decltype(tout);
-            constexpr bool VEC = decltype(vec)::value;
-            launch_kernel(false, output_ifft_kernel<K, TOUT, VEC>, dim3(blocks), dim3(Tile<K>::NT), 0, stream, yop, static_cast<TOUT*>(y),
-                       static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo,
-                       ext.Bho, total);
+        auto with_shape = [&](auto ec) {
+            constexpr int EMAX = decltype(ec)::value;
+            constexpr int TT = Tile<K, EMAX>::TT;
+            const unsigned blocks = (unsigned)((total + TT - 1) / TT);
+            auto launch = [&](auto tout, auto vec) {
+                using TOUT = decltype(tout);
+                constexpr bool VEC = decltype(vec)::value;
+                launch_kernel(false, output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream, yop,
+                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total);
+            };
+            const bool vec = (p % 4) == 0;
+            if (L->y_dtype == CIRC_BF16) {
+                if (vec) launch(__nv_bfloat16{}, std::true_type{}); else launch(__nv_bfloat16{}, std::false_type{});
+            } else {
+                if (vec) launch(float{}, std::true_type{}); else launch(float{}, std::false_type{});
+            }
         };
-        const bool vec = (p % 4) == 0;
-        if (L->y_dtype == CIRC_BF16) {
-            if (vec) launch(__nv_bfloat16{}, std::true_type{}); else launch(__nv_bfloat16{}, std::false_type{});
-        } else {
-            if (vec) launch(float{}, std::true_type{}); else launch(float{}, std::false_type{});
-        }
+        if (small) with_shape(std::integral_constant<int, SmallShape<K>::EMAX>{});
+        else with_shape(std::integral_constant<int, 16>{});
         return CIRC_OK;
     };
     const int rc = dispatch_k(L->geo.k, go);
