@@ -41,7 +41,9 @@ __host__ __device__ inline size_t fused_smem_bytes(int k, int q, int pairs, int 
 
 template <int K, int PAIRS>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a) {
-    constexpr int E = FftShape<K>::E, L = FftShape<K>::L, TT = kFusedThreads / L;
+    // transforms here are latency, not throughput: few points per lane keep every thread's chain short
+    constexpr int EMAX = K <= 8 ? 16 : (K <= 128 ? 4 : 8);
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = kFusedThreads / L;
     constexpr int H = K / 2;                    // packed slots per block
     constexpr int G = K / 4;                    // threads that cover one block with 16-byte loads
     constexpr int NU = G > 32 ? G / 32 : 1;     // 16-byte loads per thread and block
@@ -63,7 +65,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
     // ---- phase A: Z_j for all column blocks ----------------------------------------------------
     {
         const int gi = tid / L, l = tid % L;
-        const int f2 = lane_residue<K>(l);
+        const int f2 = lane_residue<K, EMAX>(l);
         const int total = PAIRS * q;
         for (int base = 0; base < total; base += TT) {
             const int T = base + gi;
@@ -85,7 +87,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
             }
 #pragma unroll
             for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
-            fft_forward<K>(v, l, tw);
+            fft_forward<K, EMAX>(v, l, tw);
             if (T < total) {
                 float2* dlo = zlo + (size_t)T * H;
                 float2* dhi = zhi + (size_t)T * H;
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
     // ---- phase C: inverse transforms, bias, activation -----------------------------------------
     {
         const int gi = tid / L, l = tid % L;
-        const int f2 = lane_residue<K>(l);
+        const int f2 = lane_residue<K, EMAX>(l);
         const int total = rows * PAIRS;
         for (int base = 0; base < total; base += TT) {
             const int T = base + gi;
@@ -215,7 +217,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
                     }
                 }
             }
-            fft_inverse<K>(v, l, tw);
+            fft_inverse<K, EMAX>(v, l, tw);
             if (!live || c >= a.Bh) continue;
             const int col = (i0 + row) * K + E * l;
             float re[E], im[E];
