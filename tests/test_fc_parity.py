@@ -98,3 +98,13 @@ def test_repeatable_bitwise():
     a, _ = run_fc(case)
     b, _ = run_fc(case)
     assert np.array_equal(a, b)
+
+
+def test_very_large_batch_fma_path():
+    # q = 2 is not a multiple of 8, so this runs the float32 FMA contraction: 50,001 samples, ragged tiles everywhere
+    case = synth.fc_case("fma_bigbatch", 48, 32, 16, 50001, w_var=1.0 / 32, x_dist="normal", bias_var=0.01, relu=True)
+    got, used = run_fc(case)
+    assert used == circ.CIRC_VARIANT_STAGED
+    rows = [0, 25000, 25001, 50000]
+    import oracle
+    assert scale_rel_err(got[rows], oracle.fc(case.w, case.x[rows], bias=case.bias, relu=True)) <= TOL_F32

@@ -80,3 +80,20 @@ def test_config4_uses_tensor_cores():
     ref = oracle.conv_pixels(case.w, case.x, case.pad, pix)
     sel = np.stack([got[n, h, w] for (n, h, w) in pix])
     assert scale_rel_err(sel, ref) <= TOL_BF16
+
+
+def test_very_large_batch_small_layer():
+    # many columns, few rows: 70,001 samples through a 128 x 128 layer (547 column tiles, ragged last one, odd batch)
+    case = synth.fc_case("tc_bigbatch", 128, 128, 16, 70001, w_var=1.0 / 128, x_dist="uniform")
+    got, used = run_fc(case)
+    assert used == T and not np.isnan(got).any()
+    rows = [0, 1, 35000, 35001, 69999, 70000]
+    assert scale_rel_err(got[rows], oracle.fc(case.w, case.x[rows])) <= TOL_F32
+
+
+def test_conv_wide_image_several_column_tiles():
+    # 300-pixel rows: three tiles across, one-row tiles, halo crossing tile and image borders
+    case = synth.conv_case("tcconv_wide", 32, 32, 3, 1, 4, 1, 5, 300, w_var=1.0 / (9 * 32), bf16_io=False)
+    got, used = run_conv(case, T)
+    assert used == T
+    assert scale_rel_err(got, oracle_conv(case)) <= TOL_F32
