@@ -115,6 +115,78 @@ __global__ void __launch_bounds__(256) grad_w_spectrum_kernel(GradWArgs a) {
     }
 }
 
+// ---- tensor-core route for the batch sum ----------------------------------------------------------
+// The product sums over batch columns, so the operands must be contiguous along the columns to be
+// "K-major" for the MMA.  This kernel transposes one float32 operand [problem][col][width] into split
+// bfloat16 [problem][row][hi | lo][cols_padded] (width = w1 for the two real problems, 2 * w1 for the rest).
+__global__ void __launch_bounds__(256) transpose_split_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst,
+                                                              int cols, int cols_padded, int w1) {
+    __shared__ float tile[32][33];
+    const int prob = blockIdx.z;
+    const int width = problem_is_real(prob) ? w1 : 2 * w1;
+    const int col0 = blockIdx.x * 32, row0 = blockIdx.y * 32;
+    if (row0 >= width) return;
+    const float* S = src + problem_offset(prob, (size_t)cols * w1, (size_t)cols * 2 * w1);
+    __nv_bfloat16* D = dst + problem_offset(prob, (size_t)w1 * 2 * cols_padded, (size_t)2 * w1 * 2 * cols_padded);
+    const int tx = threadIdx.x % 32, ty = threadIdx.x / 32;
+    for (int r = ty; r < 32; r += 8) {
+        const int col = col0 + r, row = row0 + tx;
+        tile[r][tx] = (col < cols && row < width) ? __ldg(S + (size_t)col * width + row) : 0.f;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int row = row0 + r, col = col0 + tx;
+        if (row < width && col < cols) {
+            const float v = tile[tx][r];
+            const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+            __nv_bfloat16* d = D + (size_t)row * 2 * cols_padded + col;
+            d[0] = hi;
+            d[cols_padded] = __float2bfloat16_rn(v - __bfloat162float(hi));
+        }
+    }
+}
+
+// Turns the products P[a][b] = sum_col G[col][a] X[col][b] (stored transposed, Pt[b][a]) into the gradient
+// spectra in the inverse-transform kernel's input layout (see grad_w_spectrum_kernel for the layout).
+struct CombineArgs {
+    const float* pt_real;  // [2][q][p]
+    const float* pt_cplx;  // [k/2-1][2q][2p]
+    float* yop;
+    int p, q, k, Ph, convention;
+    float scale;
+};
+__global__ void __launch_bounds__(256) grad_w_combine_kernel(CombineArgs a) {
+    const int prob = blockIdx.z;
+    const int j = blockIdx.x * 32 + threadIdx.x % 32, c = blockIdx.y * 8 + threadIdx.x / 32;
+    if (j >= a.q || c >= a.Ph) return;
+    const size_t y_real = (size_t)2 * a.Ph * a.q;
+    float* Y = a.yop + problem_offset(prob, y_real, 2 * y_real);
+    const int i1 = c + a.Ph;
+    if (problem_is_real(prob)) {
+        const float* P = a.pt_real + (size_t)prob * a.q * a.p + (size_t)j * a.p;
+        Y[(size_t)c * a.q + j] = a.scale * P[c];
+        Y[((size_t)a.Ph + c) * a.q + j] = i1 < a.p ? a.scale * P[i1] : 0.f;
+    } else {
+        const float* P = a.pt_cplx + (size_t)(prob - 2) * 4 * a.p * a.q;
+        const float* r0 = P + (size_t)(2 * j) * 2 * a.p;      // b = 2j   : P[.][2j]
+        const float* r1 = P + (size_t)(2 * j + 1) * 2 * a.p;  // b = 2j+1 : P[.][2j+1]
+        const float s = 0.5f * a.scale;
+        // U = dWhat of row block c:  Ur = P[2i][2j] + P[2i+1][2j+1],  Ui = P[2i+1][2j] - P[2i][2j+1]
+        float ur = r0[2 * c] + r1[2 * c + 1], ui = r0[2 * c + 1] - r1[2 * c];
+        float vr = 0.f, vi = 0.f;
+        if (i1 < a.p) {
+            vr = r0[2 * i1] + r1[2 * i1 + 1];
+            vi = r0[2 * i1 + 1] - r1[2 * i1];
+        }
+        if (a.convention == 1) {
+            ui = -ui;
+            vi = -vi;
+        }
+        *reinterpret_cast<float2*>(Y + (size_t)c * 2 * a.q + 2 * j) = make_float2(s * (ur - vi), s * (ui + vr));
+        *reinterpret_cast<float2*>(Y + ((size_t)a.Ph + c) * 2 * a.q + 2 * j) = make_float2(s * (ur + vi), s * (ui - vr));
+    }
+}
+
 static int build_transposed(Layer* L) {
     if (L->transposed) return CIRC_OK;
     const int p = L->geo.p, q = L->geo.q, k = L->geo.k;
@@ -189,24 +261,53 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
         e.W = e.Wo = batch;
         e.Nh = e.Bh;
         const int Ph = (p + 1) / 2;
-        const size_t x_floats = ((size_t)2 * e.Bh * L->n + 63) & ~(size_t)63;
-        const size_t g_floats = ((size_t)2 * e.Bh * L->m + 63) & ~(size_t)63;
-        const size_t y_floats = (size_t)2 * Ph * L->n;
-        if ((rc = ensure_workspace(L, (x_floats + g_floats + y_floats) * sizeof(float) + 512)) != CIRC_OK) return rc;
+        const int cols = 2 * e.Bh, cols_padded = (cols + 7) & ~7;
+        const bool tensor = batch >= 32 && tensor_batch_product_supported(cols);
+        const size_t x_floats = ((size_t)cols * L->n + 63) & ~(size_t)63;
+        const size_t g_floats = ((size_t)cols * L->m + 63) & ~(size_t)63;
+        const size_t y_floats = ((size_t)2 * Ph * L->n + 63) & ~(size_t)63;
+        // tensor route only: transposed split operands (bfloat16) and the raw products (float32)
+        const size_t xt_halves = tensor ? (((size_t)L->n * 2 * cols_padded + 127) & ~(size_t)127) : 0;
+        const size_t gt_halves = tensor ? (((size_t)L->m * 2 * cols_padded + 127) & ~(size_t)127) : 0;
+        const size_t pt_floats = tensor ? (size_t)2 * p * q + (size_t)(k / 2 - 1) * 4 * p * q : 0;
+        const size_t need = (x_floats + g_floats + y_floats + pt_floats) * sizeof(float) + (xt_halves + gt_halves) * 2 + 1024;
+        if ((rc = ensure_workspace(L, need)) != CIRC_OK) return rc;
         float* xop = static_cast<float*>(L->ws);
         float* gop = xop + x_floats;
         float* yop = gop + g_floats;
+        float* pt = yop + y_floats;
+        __nv_bfloat16* xt = reinterpret_cast<__nv_bfloat16*>(pt + ((pt_floats + 63) & ~(size_t)63));
+        __nv_bfloat16* gt = xt + xt_halves;
         // transforms: x with this layer's geometry (n, q); g with the transposed layer's (its n is m, its q is p)
         if ((rc = launch_input_fft(L, x, xop, 0, e, s)) != CIRC_OK) return rc;
         if ((rc = launch_input_fft(T, grad_a, gop, 0, e, s)) != CIRC_OK) return rc;
-        GradWArgs a;
-        a.gop = gop; a.xop = xop; a.yop = yop;
-        a.p = p; a.q = q; a.k = k; a.cols = 2 * e.Bh; a.Ph = Ph; a.convention = L->convention;
-        a.scale = 1.0f / (float)k;
-        dim3 grid((q + 15) / 16, (Ph + 15) / 16, num_problems(k));
-        grad_w_spectrum_kernel<<<grid, 256, 0, s>>>(a);
-        count_launches(1);
-        CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+        if (tensor) {
+            const int nprob = num_problems(k);
+            transpose_split_kernel<<<dim3((cols + 31) / 32, (2 * q + 31) / 32, nprob), 256, 0, s>>>(xop, xt, cols, cols_padded, q);
+            transpose_split_kernel<<<dim3((cols + 31) / 32, (2 * p + 31) / 32, nprob), 256, 0, s>>>(gop, gt, cols, cols_padded, p);
+            count_launches(2);
+            CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+            float* pt_real = pt;
+            float* pt_cplx = pt + (size_t)2 * p * q;
+            if ((rc = launch_tc_batch_product(xt, q, gt, p, k, cols, cols_padded, pt_real, pt_cplx, L->dev_status, s)) != CIRC_OK)
+                return rc;
+            CombineArgs ca;
+            ca.pt_real = pt_real; ca.pt_cplx = pt_cplx; ca.yop = yop;
+            ca.p = p; ca.q = q; ca.k = k; ca.Ph = Ph; ca.convention = L->convention;
+            ca.scale = 1.0f / (float)k;
+            grad_w_combine_kernel<<<dim3((q + 31) / 32, (Ph + 7) / 8, nprob), 256, 0, s>>>(ca);
+            count_launches(1);
+            CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+        } else {
+            GradWArgs a;
+            a.gop = gop; a.xop = xop; a.yop = yop;
+            a.p = p; a.q = q; a.k = k; a.cols = cols; a.Ph = Ph; a.convention = L->convention;
+            a.scale = 1.0f / (float)k;
+            dim3 grid((q + 15) / 16, (Ph + 15) / 16, num_problems(k));
+            grad_w_spectrum_kernel<<<grid, 256, 0, s>>>(a);
+            count_launches(1);
+            CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+        }
         // inverse transforms over (i, j): "samples" are the p row blocks, "row blocks" the q column blocks,
         // which is the transposed layer's geometry (its m is n, its p is q); no bias, no activation
         Extent ew;

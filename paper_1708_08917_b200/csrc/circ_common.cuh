@@ -160,6 +160,14 @@ int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Exte
 int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream);
 bool tensor_supported(const Layer* L);
 
+// Tensor-core batch product of the backward pass: for every frequency problem
+//   Y[prob][xrow][arow] = sum_col X^T[prob][xrow][col] * A^T[prob][arow][col]
+// with both operands as split bfloat16 [prob][row][hi | lo][cols_padded]; real problems have q / p rows,
+// complex ones 2q / 2p.  y_real: [2][q][p], y_cplx: [k/2 - 1][2q][2p].
+int launch_tc_batch_product(const __nv_bfloat16* xt, int q, const __nv_bfloat16* at, int p, int k, int cols, int cols_padded,
+                            float* y_real, float* y_cplx, int* status, cudaStream_t stream);
+bool tensor_batch_product_supported(int cols);
+
 // S3 / C3: inverse transforms + bias + activation -> y.
 int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);
 

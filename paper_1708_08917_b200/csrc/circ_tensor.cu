@@ -508,6 +508,55 @@ static int round_up16(int v) { return (v + 15) & ~15; }
 
 bool tensor_supported(const Layer* L) { return L->a_bf16 != nullptr && (L->geo.q % 8) == 0 && encode_fn() != nullptr; }
 
+// Ring depth, CTAs per SM and grid for a planned launch; maps = {A real, A complex, X hi real, X lo real, X hi complex, X lo complex}.
+static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int taps, int kq_max, long ctas, cudaStream_t stream) {
+    const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
+    const size_t stage_bytes = (size_t)nsplit * ((size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128);
+    if (stage_bytes + 1024 > 199 * 1024) {
+        set_error(CIRC_ERR_UNSUPPORTED, "filter taps x row tile do not fit one shared-memory stage (%zu bytes)", stage_bytes);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    const int iters_max = (kq_max + kKBlock - 1) / kKBlock;
+    g.stages = (int)((199 * 1024) / stage_bytes);
+    if (g.stages > kMaxStages) g.stages = kMaxStages;
+    if (g.stages > iters_max) g.stages = iters_max;
+    // Persistent CTAs.  Short tiles (few ring iterations each) run two CTAs per SM, each with half of
+    // the shared memory, so that one CTA's start-up and tail overlap the other's steady state; two
+    // accumulators of bn_max columns per CTA keep both within the 512 columns of tensor memory.
+    int ctas_per_sm = 1;
+    {
+        const int fit2 = (int)((98 * 1024) / stage_bytes);   // stages per CTA when two CTAs share an SM
+        if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && fit2 >= 3) {
+            ctas_per_sm = 2;                                  // only when each CTA still gets a ring of three or more
+            if (g.stages > fit2) g.stages = fit2;
+        }
+        // the ring may run ahead into the next tile, so it is worth filling even when one tile needs fewer stages
+        int deep = ctas_per_sm == 2 ? fit2 : (int)((198 * 1024) / stage_bytes);
+        if (deep > kMaxStages) deep = kMaxStages;
+        if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
+    }
+    const size_t smem = (size_t)g.stages * stage_bytes + 1024;
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (configured_device != dev) {
+        CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024),
+                      CIRC_ERR_CUDA);
+        configured_device = dev;
+    }
+    if (ctas >= (1L << 31)) {
+        set_error(CIRC_ERR_SHAPE, "too many output tiles (%ld)", ctas);
+        return CIRC_ERR_SHAPE;
+    }
+    g.tiles = ctas;
+    const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
+    launch_kernel(false, contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, maps[0], maps[1], maps[2], maps[3], maps[4],
+                  maps[5], g);
+    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
 int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream) {
     const Geometry& geo = L->geo;
     const int p = geo.p, q = geo.q, k = geo.k, taps = geo.taps;
@@ -603,51 +652,79 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         if ((rc = encode(&mxl_c, base + (nsplit == 2 ? 2 * q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
     }
 
-    const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const size_t stage_bytes = (size_t)nsplit * ((size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128);
-    if (stage_bytes + 1024 > 199 * 1024) {
-        set_error(CIRC_ERR_UNSUPPORTED, "filter taps x row tile do not fit one shared-memory stage (%zu bytes)", stage_bytes);
-        return CIRC_ERR_UNSUPPORTED;
+    const CUtensorMap maps[6] = {ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c};
+    return launch_planned(g, maps, nsplit, taps, 2 * q, ctas, stream);
+}
+
+
+// One kind (real or complex problems) of a generic per-problem product  Y[prob][xrow][arow] = sum_c X[prob][xrow][c] * A[prob][arow][c]
+// with both operands stored as split bfloat16 [prob][row][hi | lo][cols_padded].  The backward pass uses it for the
+// batch sum of the weight gradient, where the contraction index is the batch column.
+static int launch_tc_one_kind(bool real, const __nv_bfloat16* xt, int x_rows, const __nv_bfloat16* at, int a_rows, int cols,
+                              int cols_padded, int nprob, float* y, int* status, cudaStream_t stream) {
+    if (nprob <= 0) return CIRC_OK;
+    TcArgs g;
+    g.status = status;
+    g.taps = 1; g.r = 1; g.pad = 0;
+    g.nsplit = 2;
+    g.npass = 3;
+    g.W = g.Wo = x_rows; g.H = g.Ho = 1; g.V = 1;
+    g.tw = x_rows < kTileCols ? x_rows : kTileCols;
+    g.pitch = g.tw;
+    g.th = 1;
+    g.xrows = g.tw;
+    g.xalloc = kTileCols;
+    g.tiles_w = (x_rows + g.tw - 1) / g.tw;
+    g.tiles_h = 1;
+    g.cols_out = x_rows;
+    int bn = round_up16(a_rows) > 256 ? 256 : round_up16(a_rows);
+    const int nt = (a_rows + bn - 1) / bn;
+    g.bn_real = g.bn_cplx = bn;
+    const int sp_tiles = g.tiles_w;
+    long ctas;
+    if (real) {                      // the kernel's real group always has two problems
+        g.p = a_rows; g.q = cols; g.k = 2;
+        g.nt_real = nt; g.nt_cplx = 1;
+        g.ctas_real = 2 * nt * sp_tiles;
+        ctas = g.ctas_real;
+        g.yop = y;
+    } else {
+        g.p = a_rows / 2; g.q = cols / 2; g.k = 2 * (nprob + 1);
+        g.nt_real = 0; g.nt_cplx = nt;
+        g.ctas_real = 0;
+        ctas = (long)nprob * nt * sp_tiles;
+        g.yop = y - 2 * (size_t)x_rows * (a_rows / 2);   // the kernel skips two real-sized problems before the complex ones
     }
-    const int kq_max = 2 * q;
-    const int iters_max = (kq_max + kKBlock - 1) / kKBlock;
-    g.stages = (int)((199 * 1024) / stage_bytes);
-    if (g.stages > kMaxStages) g.stages = kMaxStages;
-    if (g.stages > iters_max) g.stages = iters_max;
-    // Persistent CTAs.  Short tiles (few ring iterations each) run two CTAs per SM, each with half of
-    // the shared memory, so that one CTA's start-up and tail overlap the other's steady state; two
-    // accumulators of bn_max columns per CTA keep both within the 512 columns of tensor memory.
-    int ctas_per_sm = 1;
+    CUtensorMap ma, mxh, mxl;
+    int rc;
     {
-        const int fit2 = (int)((98 * 1024) / stage_bytes);   // stages per CTA when two CTAs share an SM
-        if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && fit2 >= 3) {
-            ctas_per_sm = 2;                                  // only when each CTA still gets a ring of three or more
-            if (g.stages > fit2) g.stages = fit2;
-        }
-        // the ring may run ahead into the next tile, so it is worth filling even when one tile needs fewer stages
-        int deep = ctas_per_sm == 2 ? fit2 : (int)((198 * 1024) / stage_bytes);
-        if (deep > kMaxStages) deep = kMaxStages;
-        if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
+        cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)a_rows, 2, (cuuint64_t)nprob};
+        cuuint64_t str[3] = {(cuuint64_t)2 * cols_padded * 2, (cuuint64_t)cols_padded * 2, (cuuint64_t)a_rows * 2 * cols_padded * 2};
+        cuuint32_t box[4] = {kKBlock, (cuuint32_t)bn, 2, 1};
+        if ((rc = encode(&ma, const_cast<__nv_bfloat16*>(at), 4, dims, str, box)) != CIRC_OK) return rc;
     }
-    const size_t smem = (size_t)g.stages * stage_bytes + 1024;
-    static thread_local int configured_device = -1;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (configured_device != dev) {
-        CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024),
-                      CIRC_ERR_CUDA);
-        configured_device = dev;
+    {
+        const cuuint64_t row = (cuuint64_t)2 * cols_padded * 2, img = (cuuint64_t)x_rows * row;
+        cuuint64_t dims[5] = {(cuuint64_t)cols, (cuuint64_t)x_rows, 1, 1, (cuuint64_t)nprob};
+        cuuint64_t str[4] = {row, img, img, img};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, 1, 1, 1};
+        __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xt);
+        if ((rc = encode(&mxh, base, 5, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxl, base + cols_padded, 5, dims, str, box)) != CIRC_OK) return rc;
     }
-    if (ctas >= (1L << 31)) {
-        set_error(CIRC_ERR_SHAPE, "too many output tiles (%ld)", ctas);
-        return CIRC_ERR_SHAPE;
-    }
-    g.tiles = ctas;
-    const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
-    launch_kernel(false, contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c, g);
-    count_launches(1);
-    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
-    return CIRC_OK;
+    const CUtensorMap maps[6] = {ma, ma, mxh, mxl, mxh, mxl};
+    return launch_planned(g, maps, 2, 1, cols, ctas, stream);
+}
+
+bool tensor_batch_product_supported(int cols) { return cols >= 8 && (cols % 2) == 0 && encode_fn() != nullptr; }
+
+int launch_tc_batch_product(const __nv_bfloat16* xt, int q, const __nv_bfloat16* at, int p, int k, int cols, int cols_padded,
+                            float* y_real, float* y_cplx, int* status, cudaStream_t stream) {
+    const size_t x_real = (size_t)q * 2 * cols_padded, a_real = (size_t)p * 2 * cols_padded;   // elements of one real problem
+    int rc = launch_tc_one_kind(true, xt, q, at, p, cols, cols_padded, 2, y_real, status, stream);
+    if (rc != CIRC_OK) return rc;
+    return launch_tc_one_kind(false, xt + 2 * x_real, 2 * q, at + 2 * a_real, 2 * p, cols, cols_padded, k / 2 - 1, y_cplx, status,
+                              stream);
 }
 
 }  // namespace circ
