@@ -124,6 +124,20 @@ def conv(w, x, pad: int, bias=None, relu: bool = False, convention: int = 0) -> 
     return y
 
 
+def conv_backward_input(w, g, pad: int, H: int, W: int, convention: int = 0) -> np.ndarray:
+    """dL/dx of Eq. 6 from ``g = dL/dy`` (``[N][Ho][Wo][P]``): returns ``[N][H][W][C]``."""
+    w = _d(w)
+    g = _d(g)
+    r, _, p, q, k = w.shape
+    N, Ho, Wo, P = g.shape
+    assert P == p * k and Ho == H + 2 * pad - r + 1 and Wo == W + 2 * pad - r + 1
+    gx = np.empty((N, H, W, q * k), dtype=np.float64)
+    _load().circ_oracle_conv_backward_input(ctypes.c_int(P), ctypes.c_int(q * k), ctypes.c_int(r), ctypes.c_int(pad),
+                                            ctypes.c_int(k), ctypes.c_int(convention), _ptr(w), _ptr(g), ctypes.c_int(N),
+                                            ctypes.c_int(H), ctypes.c_int(W), _ptr(gx))
+    return gx
+
+
 def conv_pixels(w, x, pad: int, pixels, bias=None, relu: bool = False, convention: int = 0) -> np.ndarray:
     """Eq. 6 at the listed output pixels only: ``pixels[t] = (n, ho, wo)`` -> ``y[t][P]``."""
     w = _d(w)

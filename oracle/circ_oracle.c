@@ -211,6 +211,45 @@ ORACLE_API void circ_oracle_fc_backward(int m, int n, int k, int convention, con
 }
 
 /*
+ * CONV backward pass with respect to the input (the CONV analogue of Algorithm 2's dL/dx line; Sec. 3.2 says the
+ * training process "can be formulated in a similar way").  From Eq. 6 with zero padding,
+ *   y[n][ho][wo][P] = sum_{ti,tj,c} F(ti,tj,c,P) x[n][ho+ti-pad][wo+tj-pad][c],
+ * the chain rule gives
+ *   dL/dx[n][h][w][c] = sum_{ti,tj,P} F(ti,tj,c,P) g[n][h-ti+pad][w-tj+pad][P]      (terms outside the output image are 0)
+ * with g = dL/dy ([N][Ho][Wo][c_out]) and F(ti,tj,c,P) the dense expansion of the block-circulant channel pair.
+ */
+ORACLE_API void circ_oracle_conv_backward_input(int c_out, int c_in, int r, int pad, int k, int convention, const double* w,
+                                                const double* g, int N, int H, int W, double* gx) {
+    const int p = c_out / k, q = c_in / k;
+    const int Ho = H + 2 * pad - r + 1, Wo = W + 2 * pad - r + 1;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int nn = 0; nn < N; ++nn)
+        for (int h = 0; h < H; ++h)
+            for (int ww = 0; ww < W; ++ww) {
+                double* out = gx + (((size_t)nn * H + h) * W + ww) * c_in;
+                for (int jb = 0; jb < q; ++jb)
+                    for (int c = 0; c < k; ++c) {
+                        double acc = 0.0;
+                        for (int ti = 0; ti < r; ++ti) {
+                            const int ho = h - ti + pad;
+                            if (ho < 0 || ho >= Ho) continue;
+                            for (int tj = 0; tj < r; ++tj) {
+                                const int wo = ww - tj + pad;
+                                if (wo < 0 || wo >= Wo) continue;
+                                const double* gp = g + (((size_t)nn * Ho + ho) * Wo + wo) * c_out;
+                                for (int ib = 0; ib < p; ++ib) {
+                                    const double* wv = w + ((((size_t)ti * r + tj) * p + ib) * q + jb) * k;
+                                    for (int rr = 0; rr < k; ++rr)
+                                        acc += block_entry(wv, k, convention, rr, c) * gp[(size_t)ib * k + rr];
+                                }
+                            }
+                        }
+                        out[(size_t)jb * k + c] = acc;
+                    }
+            }
+}
+
+/*
  * Naive discrete Fourier transform, forward kernel exp(-2 pi i f t / k), unnormalised.
  * Used by tests only, for the eigenvalue closed form (the eigenvalues of a
  * circulant block are the DFT of its defining vector) and for the single-block

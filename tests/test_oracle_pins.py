@@ -271,3 +271,35 @@ def test_backward_matches_algorithm_2_fft_form(k):
     gx_fft = np.fft.ifft(np.einsum("bif,ijf->bjf", G, np.conj(W)), axis=2).real.reshape(batch, q * k)
     np.testing.assert_allclose(gw, gw_fft, atol=1e-10)
     np.testing.assert_allclose(gx, gx_fft, atol=1e-10)
+
+
+@pytest.mark.parametrize("r,pad,p,q,k,N,H,W", [(3, 1, 2, 2, 4, 2, 5, 6), (3, 0, 1, 2, 4, 1, 4, 5), (1, 0, 2, 3, 2, 2, 3, 3),
+                                               (5, 2, 2, 1, 3, 1, 6, 5), (2, 1, 1, 2, 8, 1, 4, 3), (3, 2, 2, 2, 4, 1, 3, 3)])
+def test_conv_backward_input_against_torch_autograd(r, pad, p, q, k, N, H, W):
+    # gradient of sum(g * conv2d(x, F)) with respect to x, computed by torch's float64 autograd on the dense filters
+    import torch
+    w = RNG.standard_normal((r, r, p, q, k))
+    Ho, Wo = H + 2 * pad - r + 1, W + 2 * pad - r + 1
+    g = RNG.standard_normal((N, Ho, Wo, p * k))
+    for conv in (0, 1):
+        F = torch.from_numpy(_dense_filters(w, k, conv))
+        x = torch.zeros(N, q * k, H, W, dtype=torch.float64, requires_grad=True)
+        y = torch.nn.functional.conv2d(x, F, padding=pad)
+        (y * torch.from_numpy(g).permute(0, 3, 1, 2)).sum().backward()
+        ref = x.grad.permute(0, 2, 3, 1).numpy()
+        np.testing.assert_allclose(oracle.conv_backward_input(w, g, pad, H, W, convention=conv), ref, atol=1e-11)
+
+
+def test_conv_backward_input_is_the_gradient_of_the_forward_oracle():
+    r, pad, p, q, k, N, H, W = 3, 1, 1, 2, 4, 1, 4, 3
+    w = RNG.standard_normal((r, r, p, q, k))
+    x = RNG.standard_normal((N, H, W, q * k))
+    g = RNG.standard_normal((N, H, W, p * k))
+    gx = oracle.conv_backward_input(w, g, pad, H, W)
+    h = 1e-3
+    for idx in [(0, 0, 0, 0), (0, 3, 2, 7), (0, 1, 1, 4), (0, 2, 0, 5)]:
+        xp, xm = x.copy(), x.copy()
+        xp[idx] += h
+        xm[idx] -= h
+        fd = ((g * oracle.conv(w, xp, pad)).sum() - (g * oracle.conv(w, xm, pad)).sum()) / (2 * h)
+        assert abs(fd - gx[idx]) < 1e-9
