@@ -437,7 +437,11 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * acc_cols + (uint32_t)c0, acc);
                 if (live) {
-                    if (t.row0 + c0 + 32 <= t.Mg && (t.Mg & 3) == 0) {
+                    // columns of this chunk that belong to the tile (its row tile may be narrower than 32
+                    // columns, and the last row tile may reach past the matrix)
+                    int nvalid = t.bn - c0;
+                    if (nvalid > t.Mg - t.row0 - c0) nvalid = t.Mg - t.row0 - c0;
+                    if (nvalid >= 32 && (t.Mg & 3) == 0) {
 #pragma unroll
                         for (int e = 0; e < 32; e += 4)
                             *reinterpret_cast<float4*>(yrow + c0 + e) =
@@ -446,7 +450,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                     } else {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (t.row0 + c0 + e < t.Mg) yrow[c0 + e] = __uint_as_float(acc[e]);
+                            if (e < nvalid) yrow[c0 + e] = __uint_as_float(acc[e]);
                     }
                 }
             }

@@ -97,3 +97,23 @@ def test_conv_wide_image_several_column_tiles():
     got, used = run_conv(case, T)
     assert used == T
     assert scale_rel_err(got, oracle_conv(case)) <= TOL_F32
+
+
+@pytest.mark.parametrize("p,q,r,bf16", [(16, 16, 3, False), (16, 8, 3, False), (24, 8, 1, False), (48, 8, 1, True), (16, 16, 5, True)])
+def test_conv_tensor_narrow_row_tiles(p, q, r, bf16):
+    # many taps (or a small grid) make the planner cut the weight rows into tiles narrower than the 32-column
+    # chunks the epilogue reads from tensor memory: neighbouring row tiles must not overwrite each other
+    k = 16
+    case = synth.conv_case(f"tcconv_rows_{p}_{q}_{r}_{bf16}", p * k, q * k, r, r // 2, k, 2, 9, 28,
+                           w_var=1.0 / (r * r * q * k), bf16_io=bf16)
+    got, used = run_conv(case, T)
+    assert used == T
+    assert scale_rel_err(got, oracle_conv(case)) <= (TOL_BF16 if bf16 else TOL_F32)
+
+
+def test_fc_tensor_row_tiles_not_multiple_of_32():
+    # 2p = 96 rows with a small grid: row tiles of 48
+    case = synth.fc_case("tc_rows48", 48 * 8, 64, 8, 40, w_var=1.0 / 64, x_dist="normal")
+    got, used = run_fc(case, T)
+    assert used == T
+    assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
