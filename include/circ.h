@@ -161,6 +161,18 @@ CIRC_API long circ_noalloc_max_bytes(void);
 CIRC_API int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* grad_x, float* grad_w, int batch,
                               void* stream);
 
+/*
+ * circ_conv_backward_input -- dL/dx of the convolution (the CONV counterpart of Algorithm 2's dL/dx line; Sec. 3.2):
+ *   grad_x[n][h][w][c] = sum_{i,j<r} sum_P F(i,j,c,P) grad_y[n][h-i+pad][w-j+pad][P]      (terms outside grad_y are 0)
+ *   grad_y : DEVICE pointer, channel-last [N][H + 2 pad - r + 1][W + 2 pad - r + 1][c_out], element type = the layer's y type
+ *   grad_x : DEVICE pointer, channel-last [N][H][W][c_in], element type = the layer's x type
+ *   N, H, W : the extent of the forward INPUT (as in circ_conv_forward)
+ * It runs as a forward convolution of the transposed layer (taps flipped, channel blocks transposed, defining
+ * vectors index-reversed, padding r - 1 - pad), built inside the handle on the first call (allocates, synchronises).
+ * Gradients with respect to the convolution's weights are not provided.
+ */
+CIRC_API int circ_conv_backward_input(circ_handle h, const void* grad_y, void* grad_x, int N, int H, int W, void* stream);
+
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);
 

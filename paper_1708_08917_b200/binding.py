@@ -35,6 +35,7 @@ SIGNATURES = {
     "circ_noalloc_max_bytes": (_cl, []),
     "circ_set_stage_repeat": (_ci, [_vp, _ci, _ci]),
     "circ_fc_backward": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _vp]),
+    "circ_conv_backward_input": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -181,6 +182,11 @@ def circ_noalloc_max_bytes() -> int:
 def circ_fc_backward(h: int, x, grad_a, grad_x, grad_w, batch: int, stream=None) -> None:
     """Enqueue ``grad_x = W^T grad_a`` and ``grad_w[p][q][k]`` (either may be None) from ``grad_a = dL/da``."""
     _check(load().circ_fc_backward(h, _ptr(x), _ptr(grad_a), _ptr(grad_x), _ptr(grad_w), batch, _stream(stream)))
+
+
+def circ_conv_backward_input(h: int, grad_y, grad_x, N: int, H: int, W: int, stream=None) -> None:
+    """Enqueue ``grad_x[N][H][W][C]`` from ``grad_y[N][Ho][Wo][P]``; ``N, H, W`` are the forward input's extent."""
+    _check(load().circ_conv_backward_input(h, _ptr(grad_y), _ptr(grad_x), N, H, W, _stream(stream)))
 
 
 def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:

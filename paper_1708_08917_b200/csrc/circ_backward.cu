@@ -1,5 +1,7 @@
-// Backward pass of the fully-connected layer (Algorithm 2): gradients with respect to the input and
-// to the defining vectors, from g = dL/da.
+// Backward pass (Algorithm 2): gradients of the fully-connected layer with respect to the input and to
+// the defining vectors, from g = dL/da; and the input gradient of the convolution layer, which Sec. 3.2
+// says "can be formulated in a similar way": it is the convolution of dL/dy with the flipped taps of the
+// transposed (again block-circulant) channel blocks.
 //
 //   dL/dx   = W^T g.  W^T is itself block-circulant: its block (j, i) is defined by the index-reversed
 //             vector of w_ij, so dL/dx is an ordinary forward pass of the q x p "transposed" layer
@@ -26,6 +28,22 @@ __global__ void transpose_reverse_kernel(const float* __restrict__ w, float* __r
         const long blk = idx / k;  // j * p + i
         const int i = (int)(blk % p), j = (int)(blk / p);
         wt[idx] = w[((size_t)i * q + j) * k + ((k - t) & (k - 1))];
+    }
+}
+
+// CONV: w_t[r-1-ti][r-1-tj][j][i][t] = w[ti][tj][i][j][(-t) mod k]  (taps flipped, channel blocks transposed, vectors reversed)
+__global__ void transpose_reverse_conv_kernel(const float* __restrict__ w, float* __restrict__ wt, int r, int p, int q, int k) {
+    const long total = (long)r * r * p * q * k;
+    for (long idx = blockIdx.x * (long)blockDim.x + threadIdx.x; idx < total; idx += (long)gridDim.x * blockDim.x) {
+        const int t = (int)(idx % k);
+        long rest = idx / k;
+        const int i = (int)(rest % p);
+        rest /= p;
+        const int j = (int)(rest % q);
+        rest /= q;
+        const int tj = (int)(rest % r), ti = (int)(rest / r);     // destination tap
+        const int si = r - 1 - ti, sj = r - 1 - tj;               // source tap
+        wt[idx] = w[((((size_t)si * r + sj) * p + i) * q + j) * k + ((k - t) & (k - 1))];
     }
 }
 
@@ -189,9 +207,9 @@ __global__ void __launch_bounds__(256) grad_w_combine_kernel(CombineArgs a) {
 
 static int build_transposed(Layer* L) {
     if (L->transposed) return CIRC_OK;
-    const int p = L->geo.p, q = L->geo.q, k = L->geo.k;
+    const int p = L->geo.p, q = L->geo.q, k = L->geo.k, r = L->geo.r, taps = L->geo.taps;
     float* wt = nullptr;
-    const size_t count = (size_t)p * q * k;
+    const size_t count = (size_t)taps * p * q * k;
     if (cudaMalloc(&wt, count * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "allocation of the transposed weights (%zu bytes) failed", count * sizeof(float));
@@ -199,12 +217,19 @@ static int build_transposed(Layer* L) {
     }
     long blocks = (long)((count + 255) / 256);
     if (blocks > 148L * 32) blocks = 148L * 32;
-    transpose_reverse_kernel<<<(unsigned)blocks, 256>>>(L->w_dev, wt, p, q, k);
+    if (L->kind == 1)
+        transpose_reverse_conv_kernel<<<(unsigned)blocks, 256>>>(L->w_dev, wt, r, p, q, k);
+    else
+        transpose_reverse_kernel<<<(unsigned)blocks, 256>>>(L->w_dev, wt, p, q, k);
     count_launches(1);
     Layer* T = nullptr;
-    if (cudaDeviceSynchronize() == cudaSuccess) T = make_layer(0, L->n, L->m, k, 1, 1, 0, wt);  // copies wt, computes spectra
+    // the transposed layer maps c_out -> c_in; a convolution's gradient is a convolution with padding r - 1 - pad
+    if (cudaDeviceSynchronize() == cudaSuccess)
+        T = make_layer(L->kind, L->n, L->m, k, taps, r, L->kind == 1 ? r - 1 - L->geo.pad : 0, wt);  // copies wt, computes spectra
     cudaFree(wt);
     if (!T) return circ_last_code() != CIRC_OK ? circ_last_code() : CIRC_ERR_CUDA;
+    T->x_dtype = L->y_dtype;   // the gradient flows from the output side to the input side
+    T->y_dtype = L->x_dtype;
     if (L->convention != 0) {
         T->convention = L->convention;
         int rc = launch_precompute(T, 0);
@@ -319,6 +344,25 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
         if ((rc = launch_output_ifft(T, yop, grad_w, ew, s)) != CIRC_OK) return rc;
     }
     return CIRC_OK;
+}
+
+int circ_conv_backward_input(circ_handle h, const void* grad_y, void* grad_x, int N, int H, int W, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || L->kind != 1) {
+        set_error(CIRC_ERR_ARG, "circ_conv_backward_input needs a convolution handle");
+        return CIRC_ERR_ARG;
+    }
+    const int Ho = H + 2 * L->geo.pad - L->geo.r + 1, Wo = W + 2 * L->geo.pad - L->geo.r + 1;
+    if (N < 1 || H < 1 || W < 1 || Ho < 1 || Wo < 1) {
+        set_error(CIRC_ERR_SHAPE, "bad image extent N=%d H=%d W=%d for r=%d pad=%d", N, H, W, L->geo.r, L->geo.pad);
+        return CIRC_ERR_SHAPE;
+    }
+    int rc = build_transposed(L);  // first call: allocates and synchronises
+    if (rc != CIRC_OK) return rc;
+    // dL/dx = the transposed layer applied to dL/dy, whose image is Ho x Wo; its padding r - 1 - pad restores H x W
+    L->transposed->x_dtype = L->y_dtype;
+    L->transposed->y_dtype = L->x_dtype;
+    return circ_conv_forward(reinterpret_cast<circ_handle>(L->transposed), grad_y, grad_x, N, Ho, Wo, stream);
 }
 
 }  // extern "C"

@@ -68,3 +68,32 @@ def test_backward_config2_shape():
     ref_gx, ref_gw = oracle.fc_backward(case.w, case.x, g)
     assert scale_rel_err(gw, ref_gw) <= TOL_F32
     assert scale_rel_err(gx, ref_gx) <= TOL_F32
+
+
+@pytest.mark.parametrize("r,pad,p,q,k,N,H,W", [(3, 1, 2, 2, 4, 2, 5, 6), (3, 1, 8, 3, 16, 3, 7, 5), (1, 0, 2, 8, 8, 2, 3, 3),
+                                               (3, 0, 8, 2, 4, 1, 5, 4), (5, 2, 2, 8, 4, 1, 6, 5), (3, 2, 8, 8, 4, 2, 3, 3),
+                                               (3, 1, 16, 16, 16, 2, 28, 28)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_conv_backward_input(r, pad, p, q, k, N, H, W, bf16):
+    name = f"cbwd_{r}_{pad}_{p}_{q}_{k}_{N}_{H}_{W}"
+    w = synth.normal((r, r, p, q, k), 1.0 / (r * r * p * k), synth.stream_id(name, "w"))
+    Ho, Wo = H + 2 * pad - r + 1, W + 2 * pad - r + 1
+    g = synth.normal((N, Ho, Wo, p * k), 1.0, synth.stream_id(name, "g"))
+    if bf16:
+        g = synth.round_to_bf16(g)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    h = circ.circ_conv_create(p * k, q * k, r, pad, k, w)
+    try:
+        code = circ.CIRC_BF16 if bf16 else circ.CIRC_F32
+        circ.circ_set_io_dtype(h, code, code)
+        gd = torch.from_numpy(g).cuda().to(dt)
+        gx = torch.full((N, H, W, q * k), float("nan"), device="cuda", dtype=dt)
+        circ.circ_conv_backward_input(h, gd, gx, N, H, W, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        circ.circ_device_status(h)
+        got = gx.float().cpu().numpy().astype(np.float64)
+        assert not np.isnan(got).any()
+        ref = oracle.conv_backward_input(w, g, pad, H, W)
+        assert scale_rel_err(got, ref) <= (2e-2 if bf16 else TOL_F32)
+    finally:
+        circ.circ_destroy(h)
