@@ -303,3 +303,15 @@ def test_conv_backward_input_is_the_gradient_of_the_forward_oracle():
         xm[idx] -= h
         fd = ((g * oracle.conv(w, xp, pad)).sum() - (g * oracle.conv(w, xm, pad)).sum()) / (2 * h)
         assert abs(fd - gx[idx]) < 1e-9
+
+
+def test_conv_backward_input_is_the_adjoint_of_the_forward_oracle():
+    # <conv(x), g> = <x, conv_backward_input(g)> for any x, g: the two maps are transposes of each other
+    r, pad, p, q, k, N, H, W = 3, 1, 2, 3, 4, 2, 5, 4
+    w = RNG.standard_normal((r, r, p, q, k))
+    x = RNG.standard_normal((N, H, W, q * k))
+    g = RNG.standard_normal((N, H, W, p * k))
+    for conv in (0, 1):
+        lhs = (oracle.conv(w, x, pad, convention=conv) * g).sum()
+        rhs = (x * oracle.conv_backward_input(w, g, pad, H, W, convention=conv)).sum()
+        assert abs(lhs - rhs) < 1e-10 * max(1.0, abs(lhs))
