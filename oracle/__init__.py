@@ -138,6 +138,20 @@ def conv_backward_input(w, g, pad: int, H: int, W: int, convention: int = 0) -> 
     return gx
 
 
+def conv_backward_weight(x, g, r: int, pad: int, k: int, convention: int = 0) -> np.ndarray:
+    """dL/dw of Eq. 6 from ``x`` (``[N][H][W][C]``) and ``g = dL/dy`` (``[N][Ho][Wo][P]``): returns ``[r][r][p][q][k]``."""
+    x = _d(x)
+    g = _d(g)
+    N, H, W, C = x.shape
+    _, Ho, Wo, P = g.shape
+    assert g.shape[0] == N and Ho == H + 2 * pad - r + 1 and Wo == W + 2 * pad - r + 1 and C % k == 0 and P % k == 0
+    gw = np.empty((r, r, P // k, C // k, k), dtype=np.float64)
+    _load().circ_oracle_conv_backward_weight(ctypes.c_int(P), ctypes.c_int(C), ctypes.c_int(r), ctypes.c_int(pad),
+                                             ctypes.c_int(k), ctypes.c_int(convention), _ptr(x), _ptr(g), ctypes.c_int(N),
+                                             ctypes.c_int(H), ctypes.c_int(W), _ptr(gw))
+    return gw
+
+
 def conv_pixels(w, x, pad: int, pixels, bias=None, relu: bool = False, convention: int = 0) -> np.ndarray:
     """Eq. 6 at the listed output pixels only: ``pixels[t] = (n, ho, wo)`` -> ``y[t][P]``."""
     w = _d(w)

@@ -250,6 +250,46 @@ ORACLE_API void circ_oracle_conv_backward_input(int c_out, int c_in, int r, int 
 }
 
 /*
+ * CONV backward pass with respect to the defining vectors (the CONV analogue of Algorithm 2's dL/dw line).
+ * Entry (rr, cc) of the dense channel block (i, j) of tap (ti, tj) multiplies x[..][j*k + cc] into y[..][i*k + rr], so
+ *   dL/dF(ti,tj)[i*k+rr][j*k+cc] = sum_{n,ho,wo} g[n][ho][wo][i*k+rr] x[n][ho+ti-pad][wo+tj-pad][j*k+cc]
+ * (terms whose input pixel lies in the zero padding vanish), and every entry of a circulant block is one element of
+ * its defining vector, entry (rr, cc) being w[(rr - cc) mod k] (convention 0) or w[(cc - rr) mod k] (convention 1):
+ * dL/dw[ti][tj][i][j][d] is the sum of dL/dF over the entries that hold element d.
+ */
+ORACLE_API void circ_oracle_conv_backward_weight(int c_out, int c_in, int r, int pad, int k, int convention, const double* x,
+                                                 const double* g, int N, int H, int W, double* gw) {
+    const int p = c_out / k, q = c_in / k;
+    const int Ho = H + 2 * pad - r + 1, Wo = W + 2 * pad - r + 1;
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int tap = 0; tap < r * r; ++tap)
+        for (int ib = 0; ib < p; ++ib) {
+            const int ti = tap / r, tj = tap % r;
+            for (int jb = 0; jb < q; ++jb) {
+                double* out = gw + (((size_t)tap * p + ib) * q + jb) * k;
+                for (int d = 0; d < k; ++d) out[d] = 0.0;
+                for (int nn = 0; nn < N; ++nn)
+                    for (int ho = 0; ho < Ho; ++ho) {
+                        const int h = ho + ti - pad;
+                        if (h < 0 || h >= H) continue;
+                        for (int wo = 0; wo < Wo; ++wo) {
+                            const int ww = wo + tj - pad;
+                            if (ww < 0 || ww >= W) continue;
+                            const double* gp = g + (((size_t)nn * Ho + ho) * Wo + wo) * c_out + (size_t)ib * k;
+                            const double* xp = x + (((size_t)nn * H + h) * W + ww) * c_in + (size_t)jb * k;
+                            for (int rr = 0; rr < k; ++rr)
+                                for (int cc = 0; cc < k; ++cc) {
+                                    int d = convention == 0 ? rr - cc : cc - rr;
+                                    if (d < 0) d += k;
+                                    out[d] += gp[rr] * xp[cc];
+                                }
+                        }
+                    }
+            }
+        }
+}
+
+/*
  * Naive discrete Fourier transform, forward kernel exp(-2 pi i f t / k), unnormalised.
  * Used by tests only, for the eigenvalue closed form (the eigenvalues of a
  * circulant block are the DFT of its defining vector) and for the single-block

@@ -89,3 +89,66 @@ def test_unmutated_copy_passes(tmp_path):
 @pytest.mark.parametrize("name", sorted(MUTATIONS))
 def test_planted_mistake_is_caught(tmp_path, name):
     assert not _pins_hold(_build(tmp_path, name)), f"pins did not notice mutation {name}"
+
+
+# ---- the backward functions: mistakes planted there must break the finite-difference pins -----------------------
+BACKWARD_MUTATIONS = {
+    "fc_gx_transposed_block": ("acc += gi[r] * block_entry(wij, k, convention, r, c);", "acc += gi[r] * block_entry(wij, k, convention, c, r);"),
+    "fc_gw_swapped_operands": ("out[d] += gi[r] * xj[c];", "out[d] += gi[c] * xj[r];"),
+    "conv_gx_unflipped_tap": ("const int ho = h - ti + pad;", "const int ho = h + ti - pad;"),
+    "conv_gx_wrong_block": ("acc += block_entry(wv, k, convention, rr, c) * gp[(size_t)ib * k + rr];",
+                            "acc += block_entry(wv, k, convention, c, rr) * gp[(size_t)ib * k + rr];"),
+    "conv_gw_flipped_tap": ("const int h = ho + ti - pad;", "const int h = ho - ti + pad;"),
+    "conv_gw_wrong_diagonal": ("int d = convention == 0 ? rr - cc : cc - rr;", "int d = convention == 0 ? cc - rr : rr - cc;"),
+    "conv_gw_dropped_image": ("for (int nn = 0; nn < N; ++nn)\n                    for (int ho", "for (int nn = 0; nn < 1; ++nn)\n                    for (int ho"),
+}
+
+
+def _build_backward(tmp_path, name):
+    old, new = BACKWARD_MUTATIONS[name]
+    text = SRC.read_text()
+    assert text.count(old) == 1, f"mutation anchor for {name} must be unique"
+    out = tmp_path / f"{name}.c"
+    out.write_text(text.replace(old, new, 1))
+    lib = tmp_path / f"{name}.so"
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(lib), str(out), "-lm"], check=True)
+    return ctypes.CDLL(str(lib))
+
+
+def _backward_pins_hold(lib) -> bool:
+    """Directional derivatives of L = sum(g * forward) (linear in x and in w, so central differences are exact)."""
+    rng = np.random.default_rng(11)
+    ok = True
+    # fully-connected
+    p, q, k, B = 2, 3, 4, 3
+    w, x, g = rng.standard_normal((p, q, k)), rng.standard_normal((B, q * k)), rng.standard_normal((B, p * k))
+    gx, gw = np.empty((B, q * k)), np.empty((p, q, k))
+    lib.circ_oracle_fc_backward(p * k, q * k, k, 0, w.ctypes.data_as(_dp), x.ctypes.data_as(_dp), g.ctypes.data_as(_dp),
+                                ctypes.c_long(B), gx.ctypes.data_as(_dp), gw.ctypes.data_as(_dp))
+    dx, dw = rng.standard_normal(x.shape), rng.standard_normal(w.shape)
+    ok &= np.isclose((g * (_fc(lib, w, x + dx) - _fc(lib, w, x - dx))).sum() / 2, (gx * dx).sum(), atol=1e-9)
+    ok &= np.isclose((g * (_fc(lib, w + dw, x) - _fc(lib, w - dw, x))).sum() / 2, (gw * dw).sum(), atol=1e-9)
+    # convolution
+    r, pad, p, q, k, N, H, W = 3, 1, 2, 2, 4, 2, 4, 3
+    w, x, g = rng.standard_normal((r, r, p, q, k)), rng.standard_normal((N, H, W, q * k)), rng.standard_normal((N, H, W, p * k))
+    gx, gw = np.empty(x.shape), np.empty(w.shape)
+    lib.circ_oracle_conv_backward_input(p * k, q * k, r, pad, k, 0, w.ctypes.data_as(_dp), g.ctypes.data_as(_dp), N, H, W,
+                                        gx.ctypes.data_as(_dp))
+    lib.circ_oracle_conv_backward_weight(p * k, q * k, r, pad, k, 0, x.ctypes.data_as(_dp), g.ctypes.data_as(_dp), N, H, W,
+                                         gw.ctypes.data_as(_dp))
+    dx, dw = rng.standard_normal(x.shape), rng.standard_normal(w.shape)
+    ok &= np.isclose((g * (_conv(lib, w, x + dx, pad) - _conv(lib, w, x - dx, pad))).sum() / 2, (gx * dx).sum(), atol=1e-9)
+    ok &= np.isclose((g * (_conv(lib, w + dw, x, pad) - _conv(lib, w - dw, x, pad))).sum() / 2, (gw * dw).sum(), atol=1e-9)
+    return bool(ok)
+
+
+def test_unmutated_copy_passes_backward_pins(tmp_path):
+    (tmp_path / "plain.c").write_text(SRC.read_text())
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(tmp_path / "plain.so"), str(tmp_path / "plain.c"), "-lm"],
+                   check=True)
+    assert _backward_pins_hold(ctypes.CDLL(str(tmp_path / "plain.so")))
+
+
+@pytest.mark.parametrize("name", sorted(BACKWARD_MUTATIONS))
+def test_planted_backward_mistake_is_caught(tmp_path, name):
+    assert not _backward_pins_hold(_build_backward(tmp_path, name)), f"pins did not notice mutation {name}"

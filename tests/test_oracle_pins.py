@@ -315,3 +315,59 @@ def test_conv_backward_input_is_the_adjoint_of_the_forward_oracle():
         lhs = (oracle.conv(w, x, pad, convention=conv) * g).sum()
         rhs = (x * oracle.conv_backward_input(w, g, pad, H, W, convention=conv)).sum()
         assert abs(lhs - rhs) < 1e-10 * max(1.0, abs(lhs))
+
+
+@pytest.mark.parametrize("r,pad,p,q,k,N,H,W", [(3, 1, 2, 2, 4, 2, 5, 6), (3, 0, 1, 2, 4, 1, 4, 5), (1, 0, 2, 3, 2, 2, 3, 3),
+                                               (5, 2, 2, 1, 3, 1, 6, 5), (2, 1, 1, 2, 8, 1, 4, 3)])
+def test_conv_backward_weight_against_torch_autograd(r, pad, p, q, k, N, H, W):
+    # torch's float64 autograd gives dL/dF for the dense filters; the gradient of a defining-vector element is the sum
+    # of dL/dF over the entries of the circulant block that hold it (numpy diagonals here, index arithmetic in the oracle)
+    import torch
+    x = RNG.standard_normal((N, H, W, q * k))
+    Ho, Wo = H + 2 * pad - r + 1, W + 2 * pad - r + 1
+    g = RNG.standard_normal((N, Ho, Wo, p * k))
+    w = RNG.standard_normal((r, r, p, q, k))
+    for conv in (0, 1):
+        F = torch.from_numpy(_dense_filters(w, k, conv)).requires_grad_(True)
+        y = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2), F, padding=pad)
+        (y * torch.from_numpy(g).permute(0, 3, 1, 2)).sum().backward()
+        dF = F.grad.numpy()  # [p*k][q*k][r][r]
+        ref = np.zeros((r, r, p, q, k))
+        for ti in range(r):
+            for tj in range(r):
+                for i in range(p):
+                    for j in range(q):
+                        blk = dF[i * k:(i + 1) * k, j * k:(j + 1) * k, ti, tj]
+                        if conv == 1:
+                            blk = blk.T
+                        # scipy.linalg.circulant(c)[a][b] = c[(a - b) mod k]: element d lies on the wrapped diagonal a - b = d
+                        for d in range(k):
+                            ref[ti, tj, i, j, d] = np.trace(blk, offset=-d) + (np.trace(blk, offset=k - d) if d else 0.0)
+        np.testing.assert_allclose(oracle.conv_backward_weight(x, g, r, pad, k, convention=conv), ref, atol=1e-10)
+
+
+def test_conv_backward_weight_is_the_gradient_of_the_forward_oracle():
+    # L = sum(g * conv(w, x)) is linear in w, so a central difference is exact up to rounding
+    r, pad, p, q, k, N, H, W = 3, 1, 2, 2, 4, 2, 4, 3
+    w = RNG.standard_normal((r, r, p, q, k))
+    x = RNG.standard_normal((N, H, W, q * k))
+    g = RNG.standard_normal((N, H, W, p * k))
+    gw = oracle.conv_backward_weight(x, g, r, pad, k)
+    h = 1e-3
+    for idx in [(0, 0, 0, 0, 0), (2, 2, 1, 1, 3), (0, 2, 1, 0, 1), (1, 1, 0, 1, 2), (2, 0, 0, 0, 3)]:
+        wp, wm = w.copy(), w.copy()
+        wp[idx] += h
+        wm[idx] -= h
+        fd = ((g * oracle.conv(wp, x, pad)).sum() - (g * oracle.conv(wm, x, pad)).sum()) / (2 * h)
+        assert abs(fd - gw[idx]) < 1e-9
+
+
+def test_conv_backward_weight_one_tap_reduces_to_fc_backward():
+    # r = 1: every pixel is a sample of a fully-connected layer
+    p, q, k, N, H, W = 2, 3, 4, 2, 3, 2
+    x = RNG.standard_normal((N, H, W, q * k))
+    g = RNG.standard_normal((N, H, W, p * k))
+    w = RNG.standard_normal((p, q, k))
+    for conv in (0, 1):
+        _, gw_fc = oracle.fc_backward(w, x.reshape(-1, q * k), g.reshape(-1, p * k), convention=conv)
+        np.testing.assert_allclose(oracle.conv_backward_weight(x, g, 1, 0, k, convention=conv)[0, 0], gw_fc, atol=1e-11)
