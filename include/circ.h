@@ -169,9 +169,25 @@ CIRC_API int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, 
  *   N, H, W : the extent of the forward INPUT (as in circ_conv_forward)
  * It runs as a forward convolution of the transposed layer (taps flipped, channel blocks transposed, defining
  * vectors index-reversed, padding r - 1 - pad), built inside the handle on the first call (allocates, synchronises).
- * Gradients with respect to the convolution's weights are not provided.
  */
 CIRC_API int circ_conv_backward_input(circ_handle h, const void* grad_y, void* grad_x, int N, int H, int W, void* stream);
+
+/*
+ * circ_conv_backward_weight -- dL/dw of the convolution (the CONV counterpart of Algorithm 2's dL/dw line; Sec. 3.2):
+ *   grad_w[i][j][P-block][C-block][t] = the sum, over the entries of the dense channel block of tap (i, j) that hold
+ *   element t of its defining vector, of  sum_{n,ho,wo} grad_y[n][ho][wo][row] * x[n][ho+i-pad][wo+j-pad][column]
+ * computed in the frequency domain as IFFT( sum_pixels FFT(grad_y block) o conj(FFT(x block at the tap's offset)) ).
+ *   x      : DEVICE pointer, channel-last [N][H][W][c_in], the forward input, element type = the layer's x type
+ *   grad_y : DEVICE pointer, channel-last [N][H + 2 pad - r + 1][W + 2 pad - r + 1][c_out], dL/d(pre-activation
+ *            output), element type = the layer's y type
+ *   grad_w : DEVICE pointer, float32 [r][r][p][q][k] (the layout of circ_conv_create's w); overwritten
+ *   N, H, W : the extent of the forward INPUT
+ * r <= 7 (CIRC_ERR_UNSUPPORTED otherwise).  The pixel sum is split over thread blocks and combined with float32
+ * atomic adds, so the last bits of the result can differ from run to run.  Honours circ_set_convention; the first
+ * backward call on a handle allocates and synchronises (as circ_conv_backward_input).
+ */
+CIRC_API int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, float* grad_w, int N, int H, int W,
+                                       void* stream);
 
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);

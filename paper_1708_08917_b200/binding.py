@@ -36,6 +36,7 @@ SIGNATURES = {
     "circ_set_stage_repeat": (_ci, [_vp, _ci, _ci]),
     "circ_fc_backward": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _vp]),
     "circ_conv_backward_input": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
+    "circ_conv_backward_weight": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -187,6 +188,11 @@ def circ_fc_backward(h: int, x, grad_a, grad_x, grad_w, batch: int, stream=None)
 def circ_conv_backward_input(h: int, grad_y, grad_x, N: int, H: int, W: int, stream=None) -> None:
     """Enqueue ``grad_x[N][H][W][C]`` from ``grad_y[N][Ho][Wo][P]``; ``N, H, W`` are the forward input's extent."""
     _check(load().circ_conv_backward_input(h, _ptr(grad_y), _ptr(grad_x), N, H, W, _stream(stream)))
+
+
+def circ_conv_backward_weight(h: int, x, grad_y, grad_w, N: int, H: int, W: int, stream=None) -> None:
+    """Enqueue ``grad_w[r][r][p][q][k]`` (float32) from the forward input ``x`` and ``grad_y``."""
+    _check(load().circ_conv_backward_weight(h, _ptr(x), _ptr(grad_y), _ptr(grad_w), N, H, W, _stream(stream)))
 
 
 def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:

@@ -1,7 +1,8 @@
 // Backward pass (Algorithm 2): gradients of the fully-connected layer with respect to the input and to
 // the defining vectors, from g = dL/da; and the input gradient of the convolution layer, which Sec. 3.2
 // says "can be formulated in a similar way": it is the convolution of dL/dy with the flipped taps of the
-// transposed (again block-circulant) channel blocks.
+// transposed (again block-circulant) channel blocks; and its weight gradient, the batch sum below taken
+// over pixels with the input moved by each filter tap.
 //
 //   dL/dx   = W^T g.  W^T is itself block-circulant: its block (j, i) is defined by the index-reversed
 //             vector of w_ij, so dL/dx is an ordinary forward pass of the q x p "transposed" layer
@@ -205,6 +206,125 @@ __global__ void __launch_bounds__(256) grad_w_combine_kernel(CombineArgs a) {
     }
 }
 
+// ---- CONV: gradient with respect to the defining vectors -------------------------------------------
+// dWhat(tap)_{ij}[f] = sum over output pixels of G[f][pixel][i] * conj(X[f][pixel shifted by the tap][j]): the batch sum of
+// the fully-connected case with the pixels as the batch and the X column moved by the tap (input pixels in the
+// zero padding contribute nothing).  Channel counts per block grid are small for convolutions (p, q of 4..32), so
+// each frequency problem is a skinny product with a very long sum: float32 FMA with the sum split over CTAs.
+//
+// One CTA: one problem, 16 x 16 (i, j) blocks, one filter row a (its R taps b = 0..R-1), a strided set of output
+// image rows.  Per output row the CTA stages G of that row (Wc pixels) and the one input row ho + a - pad with
+// its R - 1 halo pixels; thread (i, j) then slides along the row keeping R accumulators.
+// The result is added (atomics; the buffer is zeroed first) into the input layout of the inverse-transform
+// kernel with "sample" s = tap * p + i: samples s < St (St = ceil(taps / 2) * p) are the real parts U of column s,
+// samples s >= St the imaginary parts V of column s - St; the kernel wants U + iV there and U - iV in the
+// mirror column St + c.
+struct ConvGradWArgs {
+    const float* gop;  // G operand [problem][2 * Bhg][p | 2p], Bhg = Nh * Ho * Wo
+    const float* xop;  // X operand [problem][2 * Bhx][q | 2q], Bhx = Nh * H * W
+    float* yop;        // [problem][2 * St][q | 2q]
+    int p, q, k, r, pad, H, W, Ho, Wo, Nh, St, convention;
+    int rows;          // 2 * Nh * Ho output rows in all (both column halves)
+    float scale;
+};
+
+constexpr int kGwRow = 32;   // output pixels staged per step
+
+template <int R>
+__global__ void __launch_bounds__(256) conv_grad_w_kernel(ConvGradWArgs a) {
+    const int prob = blockIdx.z;
+    const bool real = problem_is_real(prob);
+    const int e = real ? 1 : 2;
+    const int jt = (a.q + 15) / 16;
+    const int j0 = (blockIdx.x % jt) * 16, i0 = (blockIdx.x / jt) * 16;
+    const int fa = blockIdx.y % a.r;                       // filter row
+    const int slice = blockIdx.y / a.r, nslice = gridDim.y / a.r;
+    const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
+    const int gw_ = e * a.p, xw = e * a.q;
+    const size_t Bhg = (size_t)a.Nh * a.Ho * a.Wo, Bhx = (size_t)a.Nh * a.H * a.W;
+    const float* G = a.gop + problem_offset(prob, 2 * Bhg * a.p, 2 * Bhg * 2 * a.p);
+    const float* X = a.xop + problem_offset(prob, 2 * Bhx * a.q, 2 * Bhx * 2 * a.q);
+
+    __shared__ __align__(16) float gs[kGwRow][32];            // [pixel][(Re, Im) x 16 row blocks]
+    __shared__ __align__(16) float xs[kGwRow + R - 1][32];    // [pixel - pad + b][(Re, Im) x 16 column blocks]
+
+    float ar[R], ai[R];
+#pragma unroll
+    for (int b = 0; b < R; ++b) ar[b] = ai[b] = 0.f;
+
+    for (int row = slice; row < a.rows; row += nslice) {
+        const int ho = row % a.Ho, img = row / a.Ho;          // img = half * Nh + pair
+        const int hi = ho + fa - a.pad;
+        if (hi < 0 || hi >= a.H) continue;                    // the whole input row lies in the padding (uniform per CTA)
+        const int half = img / a.Nh, pair = img % a.Nh;
+        const float* grow = G + ((size_t)half * Bhg + ((size_t)pair * a.Ho + ho) * a.Wo) * gw_;
+        const float* xrow = X + ((size_t)half * Bhx + ((size_t)pair * a.H + hi) * a.W) * xw;
+        for (int wo0 = 0; wo0 < a.Wo; wo0 += kGwRow) {
+            const int cw = a.Wo - wo0 < kGwRow ? a.Wo - wo0 : kGwRow;
+            for (int idx = threadIdx.x; idx < cw * 16 * e; idx += 256) {
+                const int w_in = idx % (16 * e), px = idx / (16 * e);
+                const int blk = i0 + w_in / e;
+                gs[px][w_in] = blk < a.p ? __ldg(grow + (size_t)(wo0 + px) * gw_ + (size_t)blk * e + w_in % e) : 0.f;
+            }
+            for (int idx = threadIdx.x; idx < (cw + R - 1) * 16 * e; idx += 256) {
+                const int w_in = idx % (16 * e), px = idx / (16 * e);
+                const int wi = wo0 + px - a.pad, blk = j0 + w_in / e;
+                xs[px][w_in] = (wi >= 0 && wi < a.W && blk < a.q) ? __ldg(xrow + (size_t)wi * xw + (size_t)blk * e + w_in % e) : 0.f;
+            }
+            __syncthreads();
+            if (real) {
+                for (int px = 0; px < cw; ++px) {
+                    const float g = gs[px][ti];
+#pragma unroll
+                    for (int b = 0; b < R; ++b) ar[b] = fmaf(g, xs[px + b][tj], ar[b]);
+                }
+            } else {
+                for (int px = 0; px < cw; ++px) {
+                    const float2 g = *reinterpret_cast<const float2*>(&gs[px][2 * ti]);
+#pragma unroll
+                    for (int b = 0; b < R; ++b) {
+                        const float2 x = *reinterpret_cast<const float2*>(&xs[px + b][2 * tj]);
+                        // (gr + i gi) * (xr - i xi)
+                        ar[b] = fmaf(g.x, x.x, fmaf(g.y, x.y, ar[b]));
+                        ai[b] = fmaf(g.y, x.x, fmaf(-g.x, x.y, ai[b]));
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+
+    const int i = i0 + ti, j = j0 + tj;
+    if (i >= a.p || j >= a.q) return;
+    float* Y = a.yop + problem_offset(prob, (size_t)2 * a.St * a.q, (size_t)2 * a.St * 2 * a.q);
+#pragma unroll
+    for (int b = 0; b < R; ++b) {
+        const int s = (fa * R + b) * a.p + i;
+        const bool upper = s >= a.St;                 // imaginary part V of column s - St
+        const int c = upper ? s - a.St : s;
+        if (real) {
+            atomicAdd(Y + ((size_t)(upper ? a.St : 0) + c) * a.q + j, a.scale * ar[b]);
+        } else {
+            const float sc = 0.5f * a.scale;
+            const float vr = sc * ar[b], vi = sc * (a.convention == 1 ? -ai[b] : ai[b]);
+            float* y0 = Y + (size_t)c * 2 * a.q + 2 * j;
+            float* y1 = Y + ((size_t)a.St + c) * 2 * a.q + 2 * j;
+            if (!upper) {      // + U in both columns
+                atomicAdd(y0, vr); atomicAdd(y0 + 1, vi);
+                atomicAdd(y1, vr); atomicAdd(y1 + 1, vi);
+            } else {           // + iV in the column, - iV in its mirror
+                atomicAdd(y0, -vi); atomicAdd(y0 + 1, vr);
+                atomicAdd(y1, vi);  atomicAdd(y1 + 1, -vr);
+            }
+        }
+    }
+}
+
+template <int R>
+static void launch_conv_grad_w(const ConvGradWArgs& a, dim3 grid, cudaStream_t s) {
+    conv_grad_w_kernel<R><<<grid, 256, 0, s>>>(a);
+}
+
 static int build_transposed(Layer* L) {
     if (L->transposed) return CIRC_OK;
     const int p = L->geo.p, q = L->geo.q, k = L->geo.k, r = L->geo.r, taps = L->geo.taps;
@@ -363,6 +483,94 @@ int circ_conv_backward_input(circ_handle h, const void* grad_y, void* grad_x, in
     L->transposed->x_dtype = L->y_dtype;
     L->transposed->y_dtype = L->x_dtype;
     return circ_conv_forward(reinterpret_cast<circ_handle>(L->transposed), grad_y, grad_x, N, Ho, Wo, stream);
+}
+
+int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, float* grad_w, int N, int H, int W, void* stream) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || L->kind != 1) {
+        set_error(CIRC_ERR_ARG, "circ_conv_backward_weight needs a convolution handle");
+        return CIRC_ERR_ARG;
+    }
+    if (!x || !grad_y || !grad_w || (reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(grad_y) & 15u) ||
+        (reinterpret_cast<uintptr_t>(grad_w) & 15u)) {
+        set_error(CIRC_ERR_ARG, "x, grad_y and grad_w must be non-NULL and 16-byte aligned");
+        return CIRC_ERR_ARG;
+    }
+    const int p = L->geo.p, q = L->geo.q, k = L->geo.k, r = L->geo.r, pad = L->geo.pad, taps = L->geo.taps;
+    const int Ho = H + 2 * pad - r + 1, Wo = W + 2 * pad - r + 1;
+    if (N < 1 || H < 1 || W < 1 || Ho < 1 || Wo < 1 || (long)N * H * W > (1L << 30) || (long)N * Ho * Wo > (1L << 30)) {
+        set_error(CIRC_ERR_SHAPE, "bad image extent N=%d H=%d W=%d for r=%d pad=%d", N, H, W, r, pad);
+        return CIRC_ERR_SHAPE;
+    }
+    if (r > 7) {
+        set_error(CIRC_ERR_UNSUPPORTED, "weight gradients are built for filters up to 7 x 7 (r=%d)", r);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    int rc = build_transposed(L);  // first call: allocates and synchronises
+    if (rc != CIRC_OK) return rc;
+    Layer* T = L->transposed;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    Extent ex, eg;   // input-side descriptions of x and of grad_y for the transform kernel
+    ex.H = ex.Ho = H; ex.W = ex.Wo = W;
+    ex.Nh = (N + 1) / 2;
+    ex.B = ex.Bo = N * H * W;
+    ex.Bh = ex.Bho = ex.Nh * H * W;
+    eg = ex;
+    eg.H = eg.Ho = Ho; eg.W = eg.Wo = Wo;
+    eg.B = eg.Bo = N * Ho * Wo;
+    eg.Bh = eg.Bho = eg.Nh * Ho * Wo;
+    const int NhT = (taps + 1) / 2, St = NhT * p;
+    const size_t x_floats = ((size_t)2 * ex.Bh * L->n + 63) & ~(size_t)63;
+    const size_t g_floats = ((size_t)2 * eg.Bh * L->m + 63) & ~(size_t)63;
+    const size_t y_floats = ((size_t)2 * St * L->n + 63) & ~(size_t)63;
+    if ((rc = ensure_workspace(L, (x_floats + g_floats + y_floats) * sizeof(float) + 1024)) != CIRC_OK) return rc;
+    float* xop = static_cast<float*>(L->ws);
+    float* gop = xop + x_floats;
+    float* yop = gop + g_floats;
+    T->x_dtype = L->y_dtype;
+    if ((rc = launch_input_fft(L, x, xop, 0, ex, s)) != CIRC_OK) return rc;
+    if ((rc = launch_input_fft(T, grad_y, gop, 0, eg, s)) != CIRC_OK) return rc;
+    CIRC_CUDA_TRY(cudaMemsetAsync(yop, 0, y_floats * sizeof(float), s), CIRC_ERR_CUDA);
+
+    ConvGradWArgs a;
+    a.gop = gop; a.xop = xop; a.yop = yop;
+    a.p = p; a.q = q; a.k = k; a.r = r; a.pad = pad; a.H = H; a.W = W; a.Ho = Ho; a.Wo = Wo;
+    a.Nh = ex.Nh; a.St = St; a.convention = L->convention;
+    a.rows = 2 * ex.Nh * Ho;
+    a.scale = 1.0f / (float)k;
+    const int tiles = ((p + 15) / 16) * ((q + 15) / 16), nprob = num_problems(k);
+    // split the pixel sum so that about four CTAs per SM are in flight
+    long slices = (4L * 148 + (long)tiles * nprob * r - 1) / ((long)tiles * nprob * r);
+    if (slices > a.rows) slices = a.rows;
+    if (slices < 1) slices = 1;
+    if (slices * r > 65535) slices = 65535 / r;
+    const dim3 grid((unsigned)tiles, (unsigned)(slices * r), (unsigned)nprob);
+    switch (r) {
+        case 1: launch_conv_grad_w<1>(a, grid, s); break;
+        case 2: launch_conv_grad_w<2>(a, grid, s); break;
+        case 3: launch_conv_grad_w<3>(a, grid, s); break;
+        case 4: launch_conv_grad_w<4>(a, grid, s); break;
+        case 5: launch_conv_grad_w<5>(a, grid, s); break;
+        case 6: launch_conv_grad_w<6>(a, grid, s); break;
+        default: launch_conv_grad_w<7>(a, grid, s); break;
+    }
+    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+
+    // inverse transforms: "samples" are (tap, row block i), paired s with s + St; "row blocks" are the q column
+    // blocks, which is the transposed layer's output geometry; float32 out, no bias, no activation
+    Extent ew;
+    ew.B = ew.Bo = taps * p;
+    ew.Bh = ew.Bho = St;
+    ew.H = ew.Ho = 1;
+    ew.W = ew.Wo = taps * p;
+    ew.Nh = St;
+    const int keep = T->y_dtype;
+    T->y_dtype = CIRC_F32;
+    rc = launch_output_ifft(T, yop, grad_w, ew, s);
+    T->y_dtype = keep;
+    return rc;
 }
 
 }  // extern "C"

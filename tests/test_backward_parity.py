@@ -97,3 +97,60 @@ def test_conv_backward_input(r, pad, p, q, k, N, H, W, bf16):
         assert scale_rel_err(got, ref) <= (2e-2 if bf16 else TOL_F32)
     finally:
         circ.circ_destroy(h)
+
+
+@pytest.mark.parametrize("r,pad,p,q,k,N,H,W", [(3, 1, 2, 2, 4, 2, 5, 6), (3, 1, 8, 3, 16, 3, 7, 5), (1, 0, 2, 8, 8, 2, 3, 3),
+                                               (3, 0, 8, 2, 4, 1, 5, 4), (5, 2, 2, 8, 4, 1, 6, 5), (3, 2, 8, 8, 4, 2, 3, 3),
+                                               (2, 1, 3, 5, 4, 3, 4, 40), (7, 3, 1, 2, 8, 1, 9, 8), (3, 1, 20, 18, 4, 2, 6, 35),
+                                               (3, 1, 16, 16, 16, 4, 28, 28)])
+@pytest.mark.parametrize("bf16,convention", [(False, 0), (False, 1), (True, 0)])
+def test_conv_backward_weight(r, pad, p, q, k, N, H, W, bf16, convention):
+    # gradient of L = sum(g * conv(w, x)) with respect to the defining vectors; odd image counts, odd tap counts
+    # (the last tap has no partner in the paired inverse transforms), rows wider than one staged segment, p, q > 16
+    name = f"cbww_{r}_{pad}_{p}_{q}_{k}_{N}_{H}_{W}"
+    w = synth.normal((r, r, p, q, k), 1.0 / (r * r * q * k), synth.stream_id(name, "w"))
+    Ho, Wo = H + 2 * pad - r + 1, W + 2 * pad - r + 1
+    x = synth.normal((N, H, W, q * k), 1.0, synth.stream_id(name, "x"))
+    g = synth.normal((N, Ho, Wo, p * k), 1.0, synth.stream_id(name, "g"))
+    if bf16:
+        x, g = synth.round_to_bf16(x), synth.round_to_bf16(g)
+    dt = torch.bfloat16 if bf16 else torch.float32
+    h = circ.circ_conv_create(p * k, q * k, r, pad, k, w)
+    try:
+        code = circ.CIRC_BF16 if bf16 else circ.CIRC_F32
+        circ.circ_set_io_dtype(h, code, code)
+        circ.circ_set_convention(h, convention)
+        xd = torch.from_numpy(x).cuda().to(dt)
+        gd = torch.from_numpy(g).cuda().to(dt)
+        gw = torch.full((r, r, p, q, k), float("nan"), device="cuda", dtype=torch.float32)
+        for _ in range(2):   # the second call must overwrite, not accumulate
+            circ.circ_conv_backward_weight(h, xd, gd, gw, N, H, W, torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        circ.circ_device_status(h)
+        got = gw.cpu().numpy().astype(np.float64)
+        assert not np.isnan(got).any()
+        ref = oracle.conv_backward_weight(x, g, r, pad, k, convention=convention)
+        assert scale_rel_err(got, ref) <= TOL_F32   # inputs rounded to bfloat16 are exact in the float32 arithmetic
+    finally:
+        circ.circ_destroy(h)
+
+
+def test_conv_backward_weight_rejects_bad_arguments():
+    w = synth.normal((3, 3, 1, 1, 4), 1.0, 3)
+    h = circ.circ_conv_create(4, 4, 3, 1, 4, w)
+    hf = circ.circ_fc_create(4, 4, 4, w[0, 0])
+    try:
+        x = torch.zeros(1, 4, 4, 4, device="cuda")
+        gw = torch.zeros(3, 3, 1, 1, 4, device="cuda")
+        with pytest.raises(circ.CircError) as e:
+            circ.circ_conv_backward_weight(h, x, None, gw, 1, 4, 4)
+        assert e.value.code == circ.CIRC_ERR_ARG
+        with pytest.raises(circ.CircError) as e:
+            circ.circ_conv_backward_weight(hf, x, x, gw, 1, 4, 4)
+        assert e.value.code == circ.CIRC_ERR_ARG
+        with pytest.raises(circ.CircError) as e:
+            circ.circ_conv_backward_weight(h, x, x, gw, 0, 4, 4)
+        assert e.value.code == circ.CIRC_ERR_SHAPE
+    finally:
+        circ.circ_destroy(h)
+        circ.circ_destroy(hf)
