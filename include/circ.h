@@ -182,9 +182,9 @@ CIRC_API int circ_conv_backward_input(circ_handle h, const void* grad_y, void* g
  *            output), element type = the layer's y type
  *   grad_w : DEVICE pointer, float32 [r][r][p][q][k] (the layout of circ_conv_create's w); overwritten
  *   N, H, W : the extent of the forward INPUT
- * r <= 7 (CIRC_ERR_UNSUPPORTED otherwise).  The pixel sum is split over thread blocks and combined with float32
- * atomic adds, so the last bits of the result can differ from run to run.  Honours circ_set_convention; the first
- * backward call on a handle allocates and synchronises (as circ_conv_backward_input).
+ * r <= 7 (CIRC_ERR_UNSUPPORTED otherwise).  The pixel sum is split over thread blocks and added up in a fixed
+ * order, so results repeat bit for bit.  Honours circ_set_convention; the first backward call on a handle
+ * allocates and synchronises (as circ_conv_backward_input).
  */
 CIRC_API int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, float* grad_w, int N, int H, int W,
                                        void* stream);

@@ -212,117 +212,278 @@ __global__ void __launch_bounds__(256) grad_w_combine_kernel(CombineArgs a) {
 // zero padding contribute nothing).  Channel counts per block grid are small for convolutions (p, q of 4..32), so
 // each frequency problem is a skinny product with a very long sum: float32 FMA with the sum split over CTAs.
 //
-// One CTA: one problem, 16 x 16 (i, j) blocks, one filter row a (its R taps b = 0..R-1), a strided set of output
-// image rows.  Per output row the CTA stages G of that row (Wc pixels) and the one input row ho + a - pad with
-// its R - 1 halo pixels; thread (i, j) then slides along the row keeping R accumulators.
-// The result is added (atomics; the buffer is zeroed first) into the input layout of the inverse-transform
-// kernel with "sample" s = tap * p + i: samples s < St (St = ceil(taps / 2) * p) are the real parts U of column s,
-// samples s >= St the imaginary parts V of column s - St; the kernel wants U + iV there and U - iV in the
-// mirror column St + c.
+// One CTA (64 threads): one problem, 16 x 16 (i, j) blocks, one filter row a (its R taps b = 0..R-1), a strided
+// set ("slice") of output image rows.  Per output row the CTA stages G of that row and the one input row
+// ho + a - pad with its R - 1 halo pixels; each thread owns 2 x 2 (i, j) blocks and slides along the row with a
+// register window of R input pixels, keeping 4 R complex accumulators.  Partial sums go to
+// part[slice][problem][tap][i][j] (float2; real problems use .x), which a second kernel adds up in a fixed order.
 struct ConvGradWArgs {
     const float* gop;  // G operand [problem][2 * Bhg][p | 2p], Bhg = Nh * Ho * Wo
     const float* xop;  // X operand [problem][2 * Bhx][q | 2q], Bhx = Nh * H * W
-    float* yop;        // [problem][2 * St][q | 2q]
+    float2* part;      // [slices][problems][taps][p][q]
+    float* yop;        // [problem][2 * St][q | 2q]: the inverse-transform kernel's input
     int p, q, k, r, pad, H, W, Ho, Wo, Nh, St, convention;
+    int slices, slices_real;   // row slices of a complex / of a real problem
     int rows;          // 2 * Nh * Ho output rows in all (both column halves)
     float scale;
 };
 
 constexpr int kGwRow = 32;   // output pixels staged per step
 
+// One staged row segment: thread (ti, tj) adds G[px][2 ti + u] * conj(X[px + b][2 tj + v]) for all px < cw, b < R.
 template <int R>
-__global__ void __launch_bounds__(256) conv_grad_w_kernel(ConvGradWArgs a) {
+__device__ __forceinline__ void grad_w_accumulate(bool real, int cw, const float (*gs)[32], const float (*xs)[32], int ti, int tj,
+                                                  float (&ar)[R][2][2], float (&ai)[R][2][2]) {
+    if (real) {
+        float2 win[R];   // win[(px + b) % R] = xs[px + b]
+#pragma unroll
+        for (int b = 0; b + 1 < R; ++b) win[b] = *reinterpret_cast<const float2*>(&xs[b][2 * tj]);
+        for (int px0 = 0; px0 < cw; px0 += R) {
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                const int px = px0 + u;
+                if (px < cw) {
+                    win[(u + R - 1) % R] = *reinterpret_cast<const float2*>(&xs[px + R - 1][2 * tj]);
+                    const float2 g = *reinterpret_cast<const float2*>(&gs[px][2 * ti]);
+#pragma unroll
+                    for (int b = 0; b < R; ++b) {
+                        const float2 x = win[(u + b) % R];
+                        ar[b][0][0] = fmaf(g.x, x.x, ar[b][0][0]);
+                        ar[b][0][1] = fmaf(g.x, x.y, ar[b][0][1]);
+                        ar[b][1][0] = fmaf(g.y, x.x, ar[b][1][0]);
+                        ar[b][1][1] = fmaf(g.y, x.y, ar[b][1][1]);
+                    }
+                }
+            }
+        }
+    } else {
+        float4 win[R];
+#pragma unroll
+        for (int b = 0; b + 1 < R; ++b) win[b] = *reinterpret_cast<const float4*>(&xs[b][4 * tj]);
+        for (int px0 = 0; px0 < cw; px0 += R) {
+#pragma unroll
+            for (int u = 0; u < R; ++u) {
+                const int px = px0 + u;
+                if (px < cw) {
+                    win[(u + R - 1) % R] = *reinterpret_cast<const float4*>(&xs[px + R - 1][4 * tj]);
+                    const float4 g = *reinterpret_cast<const float4*>(&gs[px][4 * ti]);   // (Re, Im) of two row blocks
+#pragma unroll
+                    for (int b = 0; b < R; ++b) {
+                        const float4 x = win[(u + b) % R];                                 // (Re, Im) of two column blocks
+                        // (gr + i gi) * (xr - i xi)
+                        ar[b][0][0] = fmaf(g.x, x.x, fmaf(g.y, x.y, ar[b][0][0]));
+                        ai[b][0][0] = fmaf(g.y, x.x, fmaf(-g.x, x.y, ai[b][0][0]));
+                        ar[b][0][1] = fmaf(g.x, x.z, fmaf(g.y, x.w, ar[b][0][1]));
+                        ai[b][0][1] = fmaf(g.y, x.z, fmaf(-g.x, x.w, ai[b][0][1]));
+                        ar[b][1][0] = fmaf(g.z, x.x, fmaf(g.w, x.y, ar[b][1][0]));
+                        ai[b][1][0] = fmaf(g.w, x.x, fmaf(-g.z, x.y, ai[b][1][0]));
+                        ar[b][1][1] = fmaf(g.z, x.z, fmaf(g.w, x.w, ar[b][1][1]));
+                        ai[b][1][1] = fmaf(g.w, x.z, fmaf(-g.z, x.w, ai[b][1][1]));
+                    }
+                }
+            }
+        }
+    }
+}
+
+// VEC: p and q are multiples of 4, so every 16-byte piece of an operand row is wholly inside or outside the
+// operand; the row segments are then fetched with 128-bit loads into registers one step ahead of the arithmetic.
+template <int R, bool VEC>
+__global__ void __launch_bounds__(64, R <= 3 ? 8 : 4) conv_grad_w_kernel(ConvGradWArgs a) {
     const int prob = blockIdx.z;
     const bool real = problem_is_real(prob);
     const int e = real ? 1 : 2;
     const int jt = (a.q + 15) / 16;
     const int j0 = (blockIdx.x % jt) * 16, i0 = (blockIdx.x / jt) * 16;
     const int fa = blockIdx.y % a.r;                       // filter row
-    const int slice = blockIdx.y / a.r, nslice = gridDim.y / a.r;
-    const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
+    const int slice = blockIdx.y / a.r;
+    const int nslice = real ? a.slices_real : a.slices;
+    if (slice >= nslice) return;                           // the grid is sized for the complex problems
+    const int ti = threadIdx.x / 8, tj = threadIdx.x % 8;  // row blocks i0 + 2 ti + {0, 1}, column blocks j0 + 2 tj + {0, 1}
     const int gw_ = e * a.p, xw = e * a.q;
     const size_t Bhg = (size_t)a.Nh * a.Ho * a.Wo, Bhx = (size_t)a.Nh * a.H * a.W;
     const float* G = a.gop + problem_offset(prob, 2 * Bhg * a.p, 2 * Bhg * 2 * a.p);
     const float* X = a.xop + problem_offset(prob, 2 * Bhx * a.q, 2 * Bhx * 2 * a.q);
 
     __shared__ __align__(16) float gs[kGwRow][32];            // [pixel][(Re, Im) x 16 row blocks]
-    __shared__ __align__(16) float xs[kGwRow + R - 1][32];    // [pixel - pad + b][(Re, Im) x 16 column blocks]
+    __shared__ __align__(16) float xs[kGwRow + R - 1][32];    // [pixel + b][(Re, Im) x 16 column blocks]
 
-    float ar[R], ai[R];
+    // acc[b][u][v]: tap b, row block 2 ti + u, column block 2 tj + v
+    float ar[R][2][2], ai[R][2][2];
 #pragma unroll
-    for (int b = 0; b < R; ++b) ar[b] = ai[b] = 0.f;
+    for (int b = 0; b < R; ++b)
+#pragma unroll
+        for (int u = 0; u < 2; ++u) ar[b][u][0] = ar[b][u][1] = ai[b][u][0] = ai[b][u][1] = 0.f;
 
-    for (int row = slice; row < a.rows; row += nslice) {
+    // the steps of this CTA: its rows (slice, slice + slices, ...) times the segments of kGwRow output pixels per row
+    const int nseg = (a.Wo + kGwRow - 1) / kGwRow;
+    const int nstep = ((a.rows - slice + nslice - 1) / nslice) * nseg;
+    const float *grow = nullptr, *xrow = nullptr;
+    int wo0 = 0, cw = 0;
+    // sets grow / xrow / wo0 / cw for step t; false if the step's input row lies in the zero padding (uniform per CTA)
+    auto locate = [&](int t) -> bool {
+        const int row = slice + (t / nseg) * nslice;
         const int ho = row % a.Ho, img = row / a.Ho;          // img = half * Nh + pair
         const int hi = ho + fa - a.pad;
-        if (hi < 0 || hi >= a.H) continue;                    // the whole input row lies in the padding (uniform per CTA)
+        if (hi < 0 || hi >= a.H) return false;
         const int half = img / a.Nh, pair = img % a.Nh;
-        const float* grow = G + ((size_t)half * Bhg + ((size_t)pair * a.Ho + ho) * a.Wo) * gw_;
-        const float* xrow = X + ((size_t)half * Bhx + ((size_t)pair * a.H + hi) * a.W) * xw;
-        for (int wo0 = 0; wo0 < a.Wo; wo0 += kGwRow) {
-            const int cw = a.Wo - wo0 < kGwRow ? a.Wo - wo0 : kGwRow;
-            for (int idx = threadIdx.x; idx < cw * 16 * e; idx += 256) {
+        grow = G + ((size_t)half * Bhg + ((size_t)pair * a.Ho + ho) * a.Wo) * gw_;
+        xrow = X + ((size_t)half * Bhx + ((size_t)pair * a.H + hi) * a.W) * xw;
+        wo0 = (t % nseg) * kGwRow;
+        cw = a.Wo - wo0 < kGwRow ? a.Wo - wo0 : kGwRow;
+        return true;
+    };
+
+    if constexpr (VEC) {
+        constexpr int NV = ((2 * kGwRow + R - 1) * 8 + 63) / 64;   // 16-byte pieces per thread and step, at most
+        const int vs = real ? 2 : 3;                                // pieces per pixel: 4 (real) or 8 (complex), as a shift
+        float4 v[NV];
+        auto fetch = [&](int t) -> bool {
+            if (!locate(t)) return false;
+            const int ng = cw << vs, nx = (cw + R - 1) << vs;
+#pragma unroll
+            for (int tt = 0; tt < NV; ++tt) {
+                const int idx = threadIdx.x + tt * 64;
+                const float* src = nullptr;
+                if (idx < ng) {
+                    const int px = idx >> vs, off = (idx & ((1 << vs) - 1)) * 4;
+                    if (i0 * e + off < gw_) src = grow + (size_t)(wo0 + px) * gw_ + i0 * e + off;
+                } else if (idx < ng + nx) {
+                    const int id2 = idx - ng, px = id2 >> vs, off = (id2 & ((1 << vs) - 1)) * 4;
+                    const int wi = wo0 + px - a.pad;
+                    if (wi >= 0 && wi < a.W && j0 * e + off < xw) src = xrow + (size_t)wi * xw + j0 * e + off;
+                }
+                v[tt] = src ? __ldg(reinterpret_cast<const float4*>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            return true;
+        };
+        bool cur = nstep > 0 && fetch(0);
+        int cur_cw = cw;
+        for (int t = 0; t < nstep; ++t) {
+            if (cur) {
+                const int ng = cur_cw << vs, nx = (cur_cw + R - 1) << vs;
+#pragma unroll
+                for (int tt = 0; tt < NV; ++tt) {
+                    const int idx = threadIdx.x + tt * 64;
+                    if (idx < ng)
+                        *reinterpret_cast<float4*>(&gs[idx >> vs][(idx & ((1 << vs) - 1)) * 4]) = v[tt];
+                    else if (idx < ng + nx)
+                        *reinterpret_cast<float4*>(&xs[(idx - ng) >> vs][((idx - ng) & ((1 << vs) - 1)) * 4]) = v[tt];
+                }
+            }
+            __syncthreads();
+            const int this_cw = cur_cw;
+            const bool was = cur;
+            cur = t + 1 < nstep && fetch(t + 1);   // next step's loads fly during the arithmetic
+            cur_cw = cw;
+            if (was) grad_w_accumulate<R>(real, this_cw, gs, xs, ti, tj, ar, ai);
+            __syncthreads();
+        }
+    } else {
+        for (int t = 0; t < nstep; ++t) {
+            if (!locate(t)) continue;
+            for (int idx = threadIdx.x; idx < cw * 16 * e; idx += 64) {
                 const int w_in = idx % (16 * e), px = idx / (16 * e);
                 const int blk = i0 + w_in / e;
                 gs[px][w_in] = blk < a.p ? __ldg(grow + (size_t)(wo0 + px) * gw_ + (size_t)blk * e + w_in % e) : 0.f;
             }
-            for (int idx = threadIdx.x; idx < (cw + R - 1) * 16 * e; idx += 256) {
+            for (int idx = threadIdx.x; idx < (cw + R - 1) * 16 * e; idx += 64) {
                 const int w_in = idx % (16 * e), px = idx / (16 * e);
                 const int wi = wo0 + px - a.pad, blk = j0 + w_in / e;
                 xs[px][w_in] = (wi >= 0 && wi < a.W && blk < a.q) ? __ldg(xrow + (size_t)wi * xw + (size_t)blk * e + w_in % e) : 0.f;
             }
             __syncthreads();
-            if (real) {
-                for (int px = 0; px < cw; ++px) {
-                    const float g = gs[px][ti];
-#pragma unroll
-                    for (int b = 0; b < R; ++b) ar[b] = fmaf(g, xs[px + b][tj], ar[b]);
-                }
-            } else {
-                for (int px = 0; px < cw; ++px) {
-                    const float2 g = *reinterpret_cast<const float2*>(&gs[px][2 * ti]);
-#pragma unroll
-                    for (int b = 0; b < R; ++b) {
-                        const float2 x = *reinterpret_cast<const float2*>(&xs[px + b][2 * tj]);
-                        // (gr + i gi) * (xr - i xi)
-                        ar[b] = fmaf(g.x, x.x, fmaf(g.y, x.y, ar[b]));
-                        ai[b] = fmaf(g.y, x.x, fmaf(-g.x, x.y, ai[b]));
-                    }
-                }
-            }
+            grad_w_accumulate<R>(real, cw, gs, xs, ti, tj, ar, ai);
             __syncthreads();
         }
     }
 
-    const int i = i0 + ti, j = j0 + tj;
-    if (i >= a.p || j >= a.q) return;
-    float* Y = a.yop + problem_offset(prob, (size_t)2 * a.St * a.q, (size_t)2 * a.St * 2 * a.q);
+    const int taps = a.r * a.r;
+    float2* P = a.part + ((size_t)slice * gridDim.z + prob) * taps * a.p * a.q;
 #pragma unroll
-    for (int b = 0; b < R; ++b) {
-        const int s = (fa * R + b) * a.p + i;
-        const bool upper = s >= a.St;                 // imaginary part V of column s - St
-        const int c = upper ? s - a.St : s;
-        if (real) {
-            atomicAdd(Y + ((size_t)(upper ? a.St : 0) + c) * a.q + j, a.scale * ar[b]);
-        } else {
-            const float sc = 0.5f * a.scale;
-            const float vr = sc * ar[b], vi = sc * (a.convention == 1 ? -ai[b] : ai[b]);
-            float* y0 = Y + (size_t)c * 2 * a.q + 2 * j;
-            float* y1 = Y + ((size_t)a.St + c) * 2 * a.q + 2 * j;
-            if (!upper) {      // + U in both columns
-                atomicAdd(y0, vr); atomicAdd(y0 + 1, vi);
-                atomicAdd(y1, vr); atomicAdd(y1 + 1, vi);
-            } else {           // + iV in the column, - iV in its mirror
-                atomicAdd(y0, -vi); atomicAdd(y0 + 1, vr);
-                atomicAdd(y1, vi);  atomicAdd(y1 + 1, -vr);
+    for (int b = 0; b < R; ++b)
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = i0 + 2 * ti + u, j = j0 + 2 * tj;
+            if (i >= a.p || j >= a.q) continue;
+            float2* dst = P + ((size_t)(fa * R + b) * a.p + i) * a.q + j;
+            dst[0] = make_float2(ar[b][u][0], ai[b][u][0]);
+            if (j + 1 < a.q) dst[1] = make_float2(ar[b][u][1], ai[b][u][1]);
+        }
+}
+
+// Adds the slices up (fixed order) and writes the gradient spectra in the input layout of the inverse-transform
+// kernel with "sample" s = tap * p + i: samples s < St (St = ceil(taps / 2) * p) are the real parts U of column s,
+// samples s + St the imaginary parts V; the kernel wants U + iV in column c and U - iV in the mirror column St + c.
+__global__ void __launch_bounds__(256) conv_grad_w_reduce_kernel(ConvGradWArgs a) {
+    // block = 32 columns j x 8 slice groups; one sample pair c per block
+    const int prob = blockIdx.z, nprob = gridDim.z;
+    const int lane = threadIdx.x % 32, grp = threadIdx.x / 32;
+    const int j = blockIdx.x * 32 + lane, c = blockIdx.y;
+    const int taps = a.r * a.r;
+    const size_t per_prob = (size_t)taps * a.p * a.q;
+    const bool has_v = c + a.St < taps * a.p;
+    __shared__ float4 red[8][32];
+    float ur = 0.f, ui = 0.f, vr = 0.f, vi = 0.f;
+    if (j < a.q) {
+        const float2* pu = a.part + (size_t)prob * per_prob + (size_t)c * a.q + j;            // sample c = (tap, i) in order
+        const float2* pv = a.part + (size_t)prob * per_prob + (size_t)(c + a.St) * a.q + j;
+        const int nslice = problem_is_real(prob) ? a.slices_real : a.slices;
+        for (int sl = grp; sl < nslice; sl += 8) {
+            const float2 u = __ldg(pu + (size_t)sl * nprob * per_prob);
+            ur += u.x; ui += u.y;
+            if (has_v) {
+                const float2 v = __ldg(pv + (size_t)sl * nprob * per_prob);
+                vr += v.x; vi += v.y;
             }
         }
+    }
+    red[grp][lane] = make_float4(ur, ui, vr, vi);
+    __syncthreads();
+    if (grp != 0 || j >= a.q) return;
+    for (int g = 1; g < 8; ++g) {
+        const float4 t = red[g][lane];
+        ur += t.x; ui += t.y; vr += t.z; vi += t.w;
+    }
+    if (problem_is_real(prob)) {
+        float* Y = a.yop + (size_t)prob * 2 * a.St * a.q;
+        Y[(size_t)c * a.q + j] = a.scale * ur;
+        Y[((size_t)a.St + c) * a.q + j] = a.scale * vr;
+    } else {
+        float* Y = a.yop + problem_offset(prob, (size_t)2 * a.St * a.q, (size_t)2 * a.St * 2 * a.q);
+        const float s = 0.5f * a.scale;
+        if (a.convention == 1) {  // correlation layer: the conjugate spectrum
+            ui = -ui;
+            vi = -vi;
+        }
+        *reinterpret_cast<float2*>(Y + (size_t)c * 2 * a.q + 2 * j) = make_float2(s * (ur - vi), s * (ui + vr));
+        *reinterpret_cast<float2*>(Y + ((size_t)a.St + c) * 2 * a.q + 2 * j) = make_float2(s * (ur + vi), s * (ui - vr));
     }
 }
 
 template <int R>
 static void launch_conv_grad_w(const ConvGradWArgs& a, dim3 grid, cudaStream_t s) {
-    conv_grad_w_kernel<R><<<grid, 256, 0, s>>>(a);
+    if (a.p % 4 == 0 && a.q % 4 == 0)
+        conv_grad_w_kernel<R, true><<<grid, 64, 0, s>>>(a);
+    else
+        conv_grad_w_kernel<R, false><<<grid, 64, 0, s>>>(a);
+}
+
+// CTAs of conv_grad_w_kernel<R, .> that fit on the device at once (one wave); the slower variant's count is used for both
+template <int R>
+static int conv_grad_w_wave() {
+    static int wave = 0;
+    if (wave == 0) {
+        int dev = 0, sms = 148, b1 = 1, b2 = 1;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b1, conv_grad_w_kernel<R, true>, 64, 0) != cudaSuccess) b1 = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b2, conv_grad_w_kernel<R, false>, 64, 0) != cudaSuccess) b2 = 1;
+        cudaGetLastError();
+        const int b = b1 < b2 ? b1 : b2;
+        wave = sms * (b > 0 ? b : 1);
+    }
+    return wave;
 }
 
 static int build_transposed(Layer* L) {
@@ -524,27 +685,44 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
     const size_t x_floats = ((size_t)2 * ex.Bh * L->n + 63) & ~(size_t)63;
     const size_t g_floats = ((size_t)2 * eg.Bh * L->m + 63) & ~(size_t)63;
     const size_t y_floats = ((size_t)2 * St * L->n + 63) & ~(size_t)63;
-    if ((rc = ensure_workspace(L, (x_floats + g_floats + y_floats) * sizeof(float) + 1024)) != CIRC_OK) return rc;
+    const int tiles = ((p + 15) / 16) * ((q + 15) / 16), nprob = num_problems(k);
+    const int rows = 2 * ex.Nh * Ho;
+    // split the pixel sum so that the grid is one full wave of CTAs (a few CTAs more would cost a second wave)
+    int wave;
+    switch (r) {
+        case 1: wave = conv_grad_w_wave<1>(); break;
+        case 2: wave = conv_grad_w_wave<2>(); break;
+        case 3: wave = conv_grad_w_wave<3>(); break;
+        case 4: wave = conv_grad_w_wave<4>(); break;
+        case 5: wave = conv_grad_w_wave<5>(); break;
+        case 6: wave = conv_grad_w_wave<6>(); break;
+        default: wave = conv_grad_w_wave<7>(); break;
+    }
+    // (giving the cheaper real problems fewer slices, to even out CTA run times, measured slower: their CTAs come
+    // first in launch order and the early finishers make room for nothing in a one-wave grid either way)
+    const long unit = (long)tiles * r;
+    long slices = wave / (unit * nprob);
+    if (slices > rows) slices = rows;
+    if (slices * r > 65535) slices = 65535 / r;
+    if (slices < 1) slices = 1;
+    const long slices_real = slices;
+    const size_t part_floats = ((size_t)slices * nprob * taps * p * q * 2 + 63) & ~(size_t)63;
+    if ((rc = ensure_workspace(L, (x_floats + g_floats + y_floats + part_floats) * sizeof(float) + 1024)) != CIRC_OK) return rc;
     float* xop = static_cast<float*>(L->ws);
     float* gop = xop + x_floats;
     float* yop = gop + g_floats;
+    float* part = yop + y_floats;
     T->x_dtype = L->y_dtype;
     if ((rc = launch_input_fft(L, x, xop, 0, ex, s)) != CIRC_OK) return rc;
     if ((rc = launch_input_fft(T, grad_y, gop, 0, eg, s)) != CIRC_OK) return rc;
-    CIRC_CUDA_TRY(cudaMemsetAsync(yop, 0, y_floats * sizeof(float), s), CIRC_ERR_CUDA);
 
     ConvGradWArgs a;
     a.gop = gop; a.xop = xop; a.yop = yop;
+    a.part = reinterpret_cast<float2*>(part);
     a.p = p; a.q = q; a.k = k; a.r = r; a.pad = pad; a.H = H; a.W = W; a.Ho = Ho; a.Wo = Wo;
-    a.Nh = ex.Nh; a.St = St; a.convention = L->convention;
-    a.rows = 2 * ex.Nh * Ho;
+    a.Nh = ex.Nh; a.St = St; a.convention = L->convention; a.slices = (int)slices; a.slices_real = (int)slices_real;
+    a.rows = rows;
     a.scale = 1.0f / (float)k;
-    const int tiles = ((p + 15) / 16) * ((q + 15) / 16), nprob = num_problems(k);
-    // split the pixel sum so that about four CTAs per SM are in flight
-    long slices = (4L * 148 + (long)tiles * nprob * r - 1) / ((long)tiles * nprob * r);
-    if (slices > a.rows) slices = a.rows;
-    if (slices < 1) slices = 1;
-    if (slices * r > 65535) slices = 65535 / r;
     const dim3 grid((unsigned)tiles, (unsigned)(slices * r), (unsigned)nprob);
     switch (r) {
         case 1: launch_conv_grad_w<1>(a, grid, s); break;
@@ -555,7 +733,9 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
         case 6: launch_conv_grad_w<6>(a, grid, s); break;
         default: launch_conv_grad_w<7>(a, grid, s); break;
     }
-    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    conv_grad_w_reduce_kernel<<<dim3((q + 31) / 32, St, nprob), 256, 0, s>>>(a);
+    count_launches(2);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
 
     // inverse transforms: "samples" are (tap, row block i), paired s with s + St; "row blocks" are the q column
