@@ -65,16 +65,17 @@ class Workload:
     sx: int
     sy: int
     contraction_flops: float = 0.0   # p q B (4k - 4) (x taps): flops of the per-frequency products
+    spectra_bf16: bool = False       # the streaming kernel reads bfloat16 weight spectra (workload suffix _w16)
 
 
 def workload(name: str) -> Workload:
-    """Named workloads: cfg1, cfg2_b{B}, cfg3_l{0,1,2}, cfg4, sweep_n{n}_k{k}_b{B}[_bf16]."""
-    def fc(case, desc):
+    """Named workloads: cfg1, cfg2_b{B}, cfg3_l{0,1,2}, cfg4, sweep_n{n}_k{k}_b{B}[_bf16][_w16]."""
+    def fc(case, desc, w16=False):
         s = 2 if case.bf16_io else 4
-        alg = 4 * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
+        alg = (2 if w16 else 4) * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
         p, q = case.m // case.k, case.n // case.k
         return Workload(name, desc, "fc", case, case.batch, alg, 2.0 * case.m * case.n * case.batch, s, s,
-                        float(p) * q * case.batch * (4 * case.k - 4))
+                        float(p) * q * case.batch * (4 * case.k - 4), w16)
 
     if name == "cfg1":
         return fc(synth.config1(), "FC 256x256 k=16 fp32 batch 1")
@@ -88,10 +89,13 @@ def workload(name: str) -> Workload:
         if c.x.shape[0] != 128:
             c.x = synth.normal((128, c.n), 1.0, synth.stream_id(c.name, "x"), absolute=True)
         return fc(c, f"FC {c.n}->{c.m} k=128 fp32 batch 128 (AlexNet-FC stack layer {m.group(1)})")
-    m = re.fullmatch(r"sweep_n(\d+)_k(\d+)_b(\d+)(_bf16)?", name)
+    m = re.fullmatch(r"sweep_n(\d+)_k(\d+)_b(\d+)(_bf16)?(_w16)?", name)
     if m:
-        n, k, b, bf = int(m.group(1)), int(m.group(2)), int(m.group(3)), bool(m.group(4))
-        return fc(synth.sweep_point(n, k, b, bf), f"FC {n}x{n} k={k} {'bf16' if bf else 'fp32'} batch {b}")
+        n, k, b, bf, w16 = int(m.group(1)), int(m.group(2)), int(m.group(3)), bool(m.group(4)), bool(m.group(5))
+        if w16 and b > 8:
+            raise SystemExit("_w16 (bfloat16 weight spectra) applies to the small-batch streaming kernel: batch <= 8")
+        return fc(synth.sweep_point(n, k, b, bf),
+                  f"FC {n}x{n} k={k} {'bf16' if bf else 'fp32'} batch {b}" + (", bf16 weight spectra" if w16 else ""), w16)
     if name == "cfg4":
         c = synth.config4()
         pix = c.N * c.H * c.W
@@ -291,6 +295,8 @@ def run_ours(args) -> int:
         circ.circ_set_activation(h, int(c.relu))
         code = circ.CIRC_BF16 if c.bf16_io else circ.CIRC_F32
         circ.circ_set_io_dtype(h, code, code)
+        if wl.spectra_bf16:
+            circ.circ_set_spectrum_dtype(h, circ.CIRC_BF16)
         if args.variant:
             circ.circ_set_variant(h, args.variant)
         handles.append(h)

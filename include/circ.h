@@ -210,6 +210,18 @@ CIRC_API int circ_set_io_dtype(circ_handle h, int x_dtype, int y_dtype);
  * vector x).  Recomputes the spectra from the retained copy of w; synchronises. */
 CIRC_API int circ_set_convention(circ_handle h, int convention);
 
+/*
+ * circ_set_spectrum_dtype -- storage type of the weight spectra that the small-batch streaming kernel reads
+ * (Sec. 4.3 keeps FFT(w_ij) in 16-bit words; here the reduced type is bfloat16, round to nearest even).
+ *   dtype : CIRC_F32 (default) or CIRC_BF16.
+ * With CIRC_BF16 the fused kernel (batch <= 8), which is bound by reading the spectra once, reads half the bytes;
+ * arithmetic stays float32.  The result is then the exact layer of the rounded spectra: expect the accuracy class
+ * of the bfloat16-activation path (relative error to the output scale ~1e-3, bound 2e-2), not 1e-4.  The larger
+ * batch paths are unaffected (the tensor path with bfloat16 activations uses bfloat16 spectra by itself).
+ * The first switch to CIRC_BF16 allocates m*n/k*2 bytes and synchronises.
+ */
+CIRC_API int circ_set_spectrum_dtype(circ_handle h, int dtype);
+
 /* circ_set_variant -- force a kernel variant (CIRC_VARIANT_*); AUTO restores the planner. */
 CIRC_API int circ_set_variant(circ_handle h, int variant);
 

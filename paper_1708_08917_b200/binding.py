@@ -43,6 +43,7 @@ SIGNATURES = {
     "circ_set_activation": (_ci, [_vp, _ci]),
     "circ_set_io_dtype": (_ci, [_vp, _ci, _ci]),
     "circ_set_convention": (_ci, [_vp, _ci]),
+    "circ_set_spectrum_dtype": (_ci, [_vp, _ci]),
     "circ_set_variant": (_ci, [_vp, _ci]),
     "circ_reserve": (_ci, [_vp, _cl]),
     "circ_workspace_bytes": (_cl, [_vp]),
@@ -225,6 +226,11 @@ def circ_set_io_dtype(h: int, x_dtype: int, y_dtype: int) -> None:
 
 def circ_set_convention(h: int, convention: int) -> None:
     _check(load().circ_set_convention(h, convention))
+
+
+def circ_set_spectrum_dtype(h: int, dtype: int) -> None:
+    """CIRC_BF16: the small-batch streaming kernel reads bfloat16 weight spectra (half the bytes)."""
+    _check(load().circ_set_spectrum_dtype(h, dtype))
 
 
 def circ_set_variant(h: int, variant: int) -> None:

@@ -92,6 +92,7 @@ void free_layer(Layer* L) {
     cudaFree(L->w_dev);
     cudaFree(L->bias_dev);
     cudaFree(L->w_stream);
+    cudaFree(L->w_stream_bf16);
     cudaFree(L->a_f32);
     cudaFree(L->a_bf16);
     cudaFree(L->ws);
@@ -534,6 +535,29 @@ int circ_set_convention(circ_handle h, int convention) {
     int rc = launch_precompute(L, 0);
     if (rc != CIRC_OK) return rc;
     CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int circ_set_spectrum_dtype(circ_handle h, int dtype) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (dtype != CIRC_F32 && dtype != CIRC_BF16)) {
+        set_error(CIRC_ERR_ARG, "bad handle or spectrum dtype %d", dtype);
+        return CIRC_ERR_ARG;
+    }
+    if (dtype == CIRC_BF16 && !L->w_stream_bf16) {
+        const size_t count = (size_t)L->geo.taps * L->geo.p * L->geo.q * L->geo.k;
+        CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+        if (cudaMalloc(&L->w_stream_bf16, count * sizeof(__nv_bfloat16)) != cudaSuccess) {
+            cudaGetLastError();
+            L->w_stream_bf16 = nullptr;
+            set_error(CIRC_ERR_ALLOC, "allocation of the bfloat16 spectra (%zu bytes) failed", count * sizeof(__nv_bfloat16));
+            return CIRC_ERR_ALLOC;
+        }
+        int rc = launch_round_stream(L, 0);
+        if (rc != CIRC_OK) return rc;
+        CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
+    }
+    L->w_dtype = dtype;
     return CIRC_OK;
 }
 

@@ -78,6 +78,8 @@ struct Layer {
     float* w_dev;       // retained copy of the defining vectors [taps][p][q][k]
     float* bias_dev;    // [m] or nullptr
     float* w_stream;    // spectra for the fused kernel: [taps][p][q][k] packed half spectra
+    __nv_bfloat16* w_stream_bf16;  // the same rounded to bfloat16 (only after circ_set_spectrum_dtype), or nullptr
+    int w_dtype;        // CIRC_F32 or CIRC_BF16: which stream the fused kernel reads
     float* a_f32;       // embedded float32 operand for the staged FMA contraction
     __nv_bfloat16* a_bf16;  // embedded bfloat16 operand (hi | lo split) for the tensor-core contraction
     size_t a_elems;     // elements of a_f32
@@ -148,6 +150,8 @@ inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KArgs...), dim3 
 
 // S0: spectra of the defining vectors, in every stored layout.
 int launch_precompute(Layer* L, cudaStream_t stream);
+// Rounds w_stream into w_stream_bf16 (which must be allocated).
+int launch_round_stream(Layer* L, cudaStream_t stream);
 
 // S1 / C1: forward transforms of the input -> operand X.  xmode 0: float32 [problem][col][Kq];
 // 1: bfloat16 [problem][col][hi | lo][Kq] (split of float32 values); 2: bfloat16 [problem][col][Kq].

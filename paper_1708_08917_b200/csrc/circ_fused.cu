@@ -27,7 +27,7 @@ constexpr int kMaxFusedSmem = 200 * 1024;
 struct FusedArgs {
     const void* x;
     void* y;
-    const float* w_stream;
+    const void* w_stream;   // float or __nv_bfloat16, the kernel's WT
     const float* bias;
     int relu, x_bf16, y_bf16;
     int m, n, p, q, batch, Bh;
@@ -39,7 +39,28 @@ __host__ __device__ inline size_t fused_smem_bytes(int k, int q, int pairs, int 
     return sizeof(float2) * ((size_t)k + (size_t)pairs * q * k + (size_t)jsplit * rows_per_cta * pairs * k);
 }
 
-template <int K, int PAIRS>
+// Four consecutive packed spectrum values (two slots) as stored and as float4.
+template <typename WT>
+struct WeightVec;
+template <>
+struct WeightVec<float> {
+    using raw = float4;
+    static __device__ __forceinline__ raw load(const float* blk, int idx) { return __ldg(reinterpret_cast<const float4*>(blk) + idx); }
+    static __device__ __forceinline__ raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ float4 widen(raw r) { return r; }
+};
+template <>
+struct WeightVec<__nv_bfloat16> {
+    using raw = uint2;
+    static __device__ __forceinline__ raw load(const __nv_bfloat16* blk, int idx) { return __ldg(reinterpret_cast<const uint2*>(blk) + idx); }
+    static __device__ __forceinline__ raw zero() { return make_uint2(0u, 0u); }
+    static __device__ __forceinline__ float4 widen(raw r) {   // a bfloat16 is the upper half of a float
+        return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xffff0000u), __uint_as_float(r.y << 16),
+                           __uint_as_float(r.y & 0xffff0000u));
+    }
+};
+
+template <int K, int PAIRS, typename WT>
 __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a) {
     // transforms here are latency, not throughput: few points per lane keep every thread's chain short
     constexpr int EMAX = K <= 8 ? 16 : (K <= 128 ? 4 : 8);
@@ -48,7 +69,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
     constexpr int G = K / 4;                    // threads that cover one block with 16-byte loads
     constexpr int NU = G > 32 ? G / 32 : 1;     // 16-byte loads per thread and block
     constexpr int BPW = G >= 32 ? 1 : 32 / G;   // blocks per warp-wide load
-    constexpr int UNROLL = (PAIRS == 1 ? 8 : PAIRS == 2 ? 4 : 2) / (NU > 1 ? 2 : 1);  // weight loads in flight per thread
+    // weight loads in flight per thread (the same bytes in flight for either storage type)
+    constexpr int UNROLL = (PAIRS == 1 ? 8 : PAIRS == 2 ? 4 : 2) / (NU > 1 ? 2 : 1) * (int)(sizeof(float) / sizeof(WT));
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2* zlo = tw + K;                                      // [PAIRS][q][H]  Z[s]
@@ -113,7 +135,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
         const int per_slice = ((q + JS * BPW - 1) / (JS * BPW)) * BPW;
         const int jb = slice * per_slice, je = min(q, jb + per_slice);
         for (int row = row_first; row < rows; row += row_step) {
-            const float* wrow = a.w_stream + (size_t)(i0 + row) * q * K;
+            const WT* wrow = static_cast<const WT*>(a.w_stream) + (size_t)(i0 + row) * q * K;
             float2 acc[PAIRS][NU][4];
 #pragma unroll
             for (int c = 0; c < PAIRS; ++c)
@@ -123,14 +145,13 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
                     for (int e = 0; e < 4; ++e) acc[c][t][e] = make_float2(0.f, 0.f);
 
             for (int j = jb + jsub; j < je; j += BPW * UNROLL) {
-                float4 wv[UNROLL][NU];
+                typename WeightVec<WT>::raw wv[UNROLL][NU];
 #pragma unroll
                 for (int s = 0; s < UNROLL; ++s) {
                     const int jj = j + s * BPW;
 #pragma unroll
                     for (int t = 0; t < NU; ++t)
-                        wv[s][t] = jj < je ? __ldg(reinterpret_cast<const float4*>(wrow + (size_t)jj * K) + u0 + 32 * t)
-                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                        wv[s][t] = jj < je ? WeightVec<WT>::load(wrow + (size_t)jj * K, u0 + 32 * t) : WeightVec<WT>::zero();
                 }
 #pragma unroll
                 for (int s = 0; s < UNROLL; ++s) {
@@ -139,7 +160,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
                     for (int t = 0; t < NU; ++t) {
                         const int u = u0 + 32 * t;
                         const bool dc = (u == 0);
-                        const float4 w = wv[s][t];
+                        const float4 w = WeightVec<WT>::widen(wv[s][t]);
                         // slot 2u: (a0, b0); slot 2u+1: (a1, b1).  The first slot of a block packs the two real bins.
                         const float a0 = w.x, b0 = dc ? 0.f : w.y, h0 = dc ? w.y : w.x;
                         const float a1 = w.z, b1 = w.w;
@@ -267,28 +288,33 @@ bool fused_fc_supported(const Layer* L, int batch) {
     return fused_smem_bytes(L->geo.k, L->geo.q, pairs, rows, js) <= (size_t)kMaxFusedSmem;
 }
 
-template <int K, int PAIRS>
+template <int K, int PAIRS, typename WT>
 static int launch_one(const FusedArgs& a, unsigned grid, size_t smem, cudaStream_t stream) {
     static thread_local int configured_device = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured_device != dev) {
-        CIRC_CUDA_TRY(cudaFuncSetAttribute(fused_fc_kernel<K, PAIRS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        CIRC_CUDA_TRY(cudaFuncSetAttribute(fused_fc_kernel<K, PAIRS, WT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            kMaxFusedSmem),
                       CIRC_ERR_CUDA);
         configured_device = dev;
     }
-    launch_kernel(true, fused_fc_kernel<K, PAIRS>, dim3(grid), dim3(kFusedThreads), smem, stream, a);
+    launch_kernel(true, fused_fc_kernel<K, PAIRS, WT>, dim3(grid), dim3(kFusedThreads), smem, stream, a);
     return CIRC_OK;
 }
 
-template <int K>
-static int launch_k(const FusedArgs& a, int pairs, unsigned grid, size_t smem, cudaStream_t stream) {
+template <int K, typename WT>
+static int launch_w(const FusedArgs& a, int pairs, unsigned grid, size_t smem, cudaStream_t stream) {
     switch (pairs) {
-        case 1: return launch_one<K, 1>(a, grid, smem, stream);
-        case 2: return launch_one<K, 2>(a, grid, smem, stream);
-        default: return launch_one<K, 4>(a, grid, smem, stream);
+        case 1: return launch_one<K, 1, WT>(a, grid, smem, stream);
+        case 2: return launch_one<K, 2, WT>(a, grid, smem, stream);
+        default: return launch_one<K, 4, WT>(a, grid, smem, stream);
     }
+}
+
+template <int K>
+static int launch_k(const FusedArgs& a, bool bf16_spectra, int pairs, unsigned grid, size_t smem, cudaStream_t stream) {
+    return bf16_spectra ? launch_w<K, __nv_bfloat16>(a, pairs, grid, smem, stream) : launch_w<K, float>(a, pairs, grid, smem, stream);
 }
 
 int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStream_t stream) {
@@ -296,7 +322,8 @@ int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStrea
     FusedArgs a;
     a.x = x;
     a.y = y;
-    a.w_stream = L->w_stream;
+    const bool wb = L->w_dtype == CIRC_BF16 && L->w_stream_bf16;
+    a.w_stream = wb ? static_cast<const void*>(L->w_stream_bf16) : static_cast<const void*>(L->w_stream);
     a.bias = L->bias_dev;
     a.relu = L->relu;
     a.x_bf16 = L->x_dtype == CIRC_BF16;
@@ -309,13 +336,13 @@ int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStrea
     const size_t smem = fused_smem_bytes(L->geo.k, a.q, pairs, a.rows_per_cta, a.jsplit);
     int rc;
     switch (L->geo.k) {
-        case 4: rc = launch_k<4>(a, pairs, grid, smem, stream); break;
-        case 8: rc = launch_k<8>(a, pairs, grid, smem, stream); break;
-        case 16: rc = launch_k<16>(a, pairs, grid, smem, stream); break;
-        case 32: rc = launch_k<32>(a, pairs, grid, smem, stream); break;
-        case 64: rc = launch_k<64>(a, pairs, grid, smem, stream); break;
-        case 128: rc = launch_k<128>(a, pairs, grid, smem, stream); break;
-        case 256: rc = launch_k<256>(a, pairs, grid, smem, stream); break;
+        case 4: rc = launch_k<4>(a, wb, pairs, grid, smem, stream); break;
+        case 8: rc = launch_k<8>(a, wb, pairs, grid, smem, stream); break;
+        case 16: rc = launch_k<16>(a, wb, pairs, grid, smem, stream); break;
+        case 32: rc = launch_k<32>(a, wb, pairs, grid, smem, stream); break;
+        case 64: rc = launch_k<64>(a, wb, pairs, grid, smem, stream); break;
+        case 128: rc = launch_k<128>(a, wb, pairs, grid, smem, stream); break;
+        case 256: rc = launch_k<256>(a, wb, pairs, grid, smem, stream); break;
         default: set_error(CIRC_ERR_SHAPE, "block size %d not supported", L->geo.k); return CIRC_ERR_SHAPE;
     }
     if (rc != CIRC_OK) return rc;

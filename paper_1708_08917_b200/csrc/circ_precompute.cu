@@ -93,6 +93,22 @@ __global__ void precompute_spectra_kernel(const float* __restrict__ w, float* __
     }
 }
 
+// Reduced-precision copy of the streamed spectra (Sec. 4.3 stores 16-bit spectra; here bfloat16, round to nearest even).
+__global__ void round_stream_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t count) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x)
+        dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+int launch_round_stream(Layer* L, cudaStream_t stream) {
+    const size_t count = (size_t)L->geo.taps * L->geo.p * L->geo.q * L->geo.k;
+    size_t blocks = (count + 255) / 256;
+    if (blocks > 148 * 32) blocks = 148 * 32;
+    round_stream_kernel<<<(unsigned)blocks, 256, 0, stream>>>(L->w_stream, L->w_stream_bf16, count);
+    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
 int launch_precompute(Layer* L, cudaStream_t stream) {
     const Geometry& g = L->geo;
     const long total = (long)g.taps * g.p * g.q * (g.k / 2 + 1);
@@ -103,6 +119,7 @@ int launch_precompute(Layer* L, cudaStream_t stream) {
                                                                        L->convention, total);
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    if (L->w_stream_bf16) return launch_round_stream(L, stream);
     return CIRC_OK;
 }
 
