@@ -69,7 +69,7 @@ class Workload:
 
 
 def workload(name: str) -> Workload:
-    """Named workloads: cfg1, cfg2_b{B}, cfg3_l{0,1,2}, cfg4, sweep_n{n}_k{k}_b{B}[_bf16][_w16]."""
+    """Named workloads: cfg1, cfg2_b{B}, cfg3_l{0,1,2}, cfg3_stack, cfg4, sweep_n{n}_k{k}_b{B}[_bf16][_w16]."""
     def fc(case, desc, w16=False):
         s = 2 if case.bf16_io else 4
         alg = (2 if w16 else 4) * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
@@ -96,6 +96,17 @@ def workload(name: str) -> Workload:
             raise SystemExit("_w16 (bfloat16 weight spectra) applies to the small-batch streaming kernel: batch <= 8")
         return fc(synth.sweep_point(n, k, b, bf),
                   f"FC {n}x{n} k={k} {'bf16' if bf else 'fp32'} batch {b}" + (", bf16 weight spectra" if w16 else ""), w16)
+    if name == "cfg3_stack":
+        layers = synth.config3_layers(128)
+        first, last = layers[0], layers[-1]
+        # what the stack must move: every layer's defining vectors once, the input and the final output;
+        # the activations between the layers need not touch memory
+        alg = sum(4 * l.m * l.n // l.k for l in layers) + 4 * 128 * (first.n + last.m)
+        stack = synth.FcCase("cfg3_stack", last.m, first.n, first.k, 128, None, first.x, None, False, False)
+        stack.layers = layers
+        return Workload(name, "FC stack 9216->4096->4096->1024 k=128 fp32 batch 128, ReLU between layers, one circ_stack_forward",
+                        "stack", stack, 128, alg, sum(2.0 * l.m * l.n * 128 for l in layers), 4, 4,
+                        sum(float(l.m // l.k) * (l.n // l.k) * 128 * (4 * l.k - 4) for l in layers))
     if name == "cfg4":
         c = synth.config4()
         pix = c.N * c.H * c.W
@@ -168,6 +179,11 @@ def oracle_forward(wl: Workload, units: int):
     import oracle
     c = wl.case
     bias = None if c.bias is None else c.bias.astype(np.float64)
+    if wl.kind == "stack":
+        a = c.x[:units].astype(np.float64)
+        for l in c.layers:
+            a = oracle.fc(l.w.astype(np.float64), a, relu=l.relu)
+        return a
     if wl.kind == "fc":
         return oracle.fc(c.w.astype(np.float64), c.x[:units].astype(np.float64), bias=bias, relu=c.relu)
     return oracle.conv(c.w.astype(np.float64), c.x[:units].astype(np.float64), c.pad, bias=bias, relu=c.relu)
@@ -187,7 +203,7 @@ def oracle_rate(wl: Workload, budget_s: float = 12.0):
         dt = time.perf_counter() - t0
         if dt >= budget_s or done >= 50 * wl.samples:
             break
-    what = "batch rows" if wl.kind == "fc" else "images"
+    what = "images" if wl.kind == "conv" else "batch rows"
     return done / dt, f"{units} of {wl.samples} {what} per pass, {done // units} passes, all outputs, {dt:.1f} s", oracle.threads()
 
 
@@ -209,7 +225,7 @@ def run_reference(args) -> int:
         oracle_forward(wl, units)
     dt = time.perf_counter() - t0
     value = units * args.steps / dt
-    sample = f"{units} of {wl.samples} {'batch rows' if wl.kind == 'fc' else 'images'} per step, all outputs"
+    sample = f"{units} of {wl.samples} {'images' if wl.kind == 'conv' else 'batch rows'} per step, all outputs"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
@@ -265,6 +281,10 @@ def run_ours(args) -> int:
         x_shape, y_shape = (c.batch, c.n), (c.batch, c.m)
         weight_store = 3 * 4 * c.m * c.n // c.k + 4 * c.m * c.n // c.k      # stream + embedded f32 + embedded bf16 hi/lo
         workspace = 4 * (c.batch + 1) * (c.m + c.n)
+    elif wl.kind == "stack":
+        x_shape, y_shape = (c.batch, c.n), (c.batch, c.m)
+        weight_store = sum(16 * l.m * l.n // l.k for l in c.layers)
+        workspace = sum(4 * (c.batch + 1) * (l.m + l.n) for l in c.layers)
     else:
         Ho, Wo = c.H + 2 * c.pad - c.r + 1, c.W + 2 * c.pad - c.r + 1
         x_shape, y_shape = (c.N, c.H, c.W, c.c_in), (c.N, Ho, Wo, c.c_out)
@@ -278,12 +298,27 @@ def run_ours(args) -> int:
     def draw_x(tag):
         if wl.kind == "fc":
             a = synth.uniform(x_shape, -1.0, 1.0, synth.stream_id(c.name, tag))
-        else:
+        else:   # CONV and the FC stack take post-ReLU-like activations
             a = synth.normal(x_shape, 1.0, synth.stream_id(c.name, tag), absolute=True)
         return torch.from_numpy(a)
 
-    handles, xs, ys = [], [], []
+    handles, xs, ys, stacks, stack_layers = [], [], [], [], []
     for s in range(sets):
+        if wl.kind == "stack":
+            hs = []
+            for l in c.layers:
+                hl = circ.circ_fc_create(l.m, l.n, l.k, l.w)
+                circ.circ_set_activation(hl, int(l.relu))
+                if args.variant:
+                    circ.circ_set_variant(hl, args.variant)
+                hs.append(hl)
+            st_h = circ.circ_stack_create(hs)
+            circ.circ_stack_reserve(st_h, c.batch)
+            stack_layers.append(hs)
+            stacks.append(st_h)
+            xs.append(draw_x(f"x{rank}_{s}").cuda().to(tdt))
+            ys.append(torch.empty(y_shape, device="cuda", dtype=tdt))
+            continue
         if wl.kind == "fc":
             h = circ.circ_fc_create(c.m, c.n, c.k, c.w)
             circ.circ_reserve(h, c.batch)
@@ -306,7 +341,9 @@ def run_ours(args) -> int:
     torch.cuda.synchronize()
 
     def forward(s, st):
-        if wl.kind == "fc":
+        if wl.kind == "stack":
+            circ.circ_stack_forward(stacks[s], xs[s], ys[s], c.batch, st)
+        elif wl.kind == "fc":
             circ.circ_fc_forward(handles[s], xs[s], ys[s], c.batch, st)
         else:
             circ.circ_conv_forward(handles[s], xs[s], ys[s], c.N, c.H, c.W, st)
@@ -314,7 +351,7 @@ def run_ours(args) -> int:
     for i in range(max(args.warmup, 3)):
         forward(i % sets, stream)
     torch.cuda.synchronize()
-    circ.circ_device_status(handles[0])
+    circ.circ_device_status(stack_layers[0][0] if wl.kind == "stack" else handles[0])
 
     # One rotation through all sets is captured in a CUDA graph so that the GPU, not the host's
     # launch rate, sets the pace; the timed region replays it and runs the remainder eagerly.
@@ -362,7 +399,7 @@ def run_ours(args) -> int:
     ms_total = max_over_ranks(e0.elapsed_time(e1), world)
     ms_step = ms_total / args.steps
     value = world * wl.samples * args.steps / (ms_total * 1e-3)
-    variant = circ.circ_last_variant(handles[0])
+    variant = circ.circ_last_variant(stack_layers[0][0] if wl.kind == "stack" else handles[0])
 
     # Per-kernel device times, measured with the same CUDA events on the same rotating buffers: the
     # rotation is captured again with ONE stage's kernel launched 1 + R times per forward (each of
@@ -397,7 +434,7 @@ def run_ours(args) -> int:
 
     R = 3
     nrep = max(3, min(200, args.steps // sets // 4))
-    used_stages = [3] if variant == circ.CIRC_VARIANT_FUSED else [0, 1, 2]
+    used_stages = [] if wl.kind == "stack" else [3] if variant == circ.CIRC_VARIANT_FUSED else [0, 1, 2]
     base_ms = time_rotation(nrep)
     stage_ms = [0.0] * 4
     for st_i in used_stages:
@@ -409,16 +446,23 @@ def run_ours(args) -> int:
     per_launch_us = {STAGES[i]: (1e3 * stage_ms[i] if i in used_stages else None) for i in range(4)}
     # context only: the same rotation with four independent batches in flight (four graph branches)
     overlap4 = world * wl.samples / (time_rotation(nrep, 4) * 1e-3) if sets >= 4 else None
-    dom = max(used_stages, key=lambda i: stage_ms[i])
-    dom_us = max(1e3 * stage_ms[dom], 1e-3)
     peaks = measured_peaks()
+    if wl.kind == "stack":
+        # seven kernels of three kinds: the roofline is taken over the whole call (every layer's defining vectors,
+        # the input and the output once, against the HBM peak); per-kernel figures are those of the cfg3_l* workloads
+        dom, dom_us = 2, 1e3 * ms_step
+        STAGE_NAME = "whole_stack"
+    else:
+        dom = max(used_stages, key=lambda i: stage_ms[i])
+        dom_us = max(1e3 * stage_ms[dom], 1e-3)
+        STAGE_NAME = STAGES[dom]
     # Which roofline bounds the dominant kernel: the contraction is tensor-bound when its flops at the
     # tensor peak (a third of the bf16 peak for float32 inputs: three bf16 passes) take longer than the
     # forward's algorithmic bytes at the HBM peak; everything else is HBM-bound.
     tensor_peak = peaks["bf16_tflops"] / (1.0 if c.bf16_io else 3.0)
     t_hbm = wl.alg_bytes / (peaks["hbm_gbs"] * 1e9)
     t_tc = wl.contraction_flops / (tensor_peak * 1e12)
-    if STAGES[dom] == "contraction" and variant == circ.CIRC_VARIANT_TENSOR and t_tc > t_hbm:
+    if STAGE_NAME == "contraction" and variant == circ.CIRC_VARIANT_TENSOR and t_tc > t_hbm:
         achieved = wl.contraction_flops / (dom_us * 1e-6) / 1e12
         roofline = {"bound": "tensor", "kernel": STAGES[dom], "achieved": achieved, "peak": tensor_peak, "unit": "TFLOP/s",
                     "frac": achieved / tensor_peak, "peak_source": peaks["source"],
@@ -426,9 +470,10 @@ def run_ours(args) -> int:
                     "traffic": traffic_if_current(wl.name, STAGES[dom]), "algorithmic_flops_per_launch": wl.contraction_flops}
     else:
         achieved = wl.alg_bytes / (dom_us * 1e-6) / 1e9
-        roofline = {"bound": "hbm", "kernel": STAGES[dom], "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+        roofline = {"bound": "hbm", "kernel": STAGE_NAME, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": achieved / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                    "frac_of_nominal_8000": achieved / 8000.0, "traffic": traffic_if_current(wl.name, STAGES[dom]),
+                    "frac_of_nominal_8000": achieved / 8000.0,
+                    "traffic": None if wl.kind == "stack" else traffic_if_current(wl.name, STAGES[dom]),
                     "algorithmic_bytes_per_launch": wl.alg_bytes}
     roofline["kernel_us_per_launch"] = per_launch_us
     roofline["whole_forward_hbm_frac"] = wl.alg_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"]
@@ -441,7 +486,11 @@ def run_ours(args) -> int:
         yh = [torch.empty(y_shape, dtype=tdt).pin_memory() for _ in range(nh)]
 
         def forward_host(i):
-            if wl.kind == "fc":
+            if wl.kind == "stack":   # no host-pointer entry point for stacks: the same copies, issued here
+                xs[i % sets].copy_(xh[i % nh], non_blocking=True)
+                circ.circ_stack_forward(stacks[i % sets], xs[i % sets], ys[i % sets], c.batch, stream)
+                yh[i % nh].copy_(ys[i % sets], non_blocking=True)
+            elif wl.kind == "fc":
                 circ.circ_fc_forward_host(handles[i % sets], xh[i % nh], yh[i % nh], c.batch, stream)
             else:
                 circ.circ_conv_forward_host(handles[i % sets], xh[i % nh], yh[i % nh], c.N, c.H, c.W, stream)
@@ -467,7 +516,9 @@ def run_ours(args) -> int:
         rate, what, threads = oracle_rate(wl)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what}
 
-    for h in handles:
+    for st_h in stacks:
+        circ.circ_stack_destroy(st_h)
+    for h in handles + [hl for hs in stack_layers for hl in hs]:
         circ.circ_destroy(h)
     if rank == 0:
         line = {

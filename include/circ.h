@@ -189,6 +189,35 @@ CIRC_API int circ_conv_backward_input(circ_handle h, const void* grad_y, void* g
 CIRC_API int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, float* grad_w, int N, int H, int W,
                                        void* stream);
 
+/*
+ * Layer stacks -- several fully-connected layers run as one call (the paper evaluates whole networks, e.g. the
+ * FC layers of AlexNet in Sec. 5, and keeps activations on chip between layers).
+ *
+ * circ_stack_create  : layers[0..count) are fully-connected handles with layers[l].m == layers[l+1].n, on one
+ *                      device; the stack BORROWS them (the caller keeps ownership, must keep them alive and destroys
+ *                      them after the stack).  Each layer keeps its own bias / activation / variant / dtype settings.
+ *                      Returns NULL on error (circ_last_error()).
+ * circ_stack_forward : y[batch][m_last] = layer_{count-1}( ... layer_0(x) ... ); x, y DEVICE pointers, 16-byte
+ *                      aligned, element types = the first layer's x type / the last layer's y type.  Enqueues on
+ *                      `stream`.  Between two consecutive layers that both run on the staged (three-kernel) path
+ *                      with the same block size and float32 activations, the inverse transforms of the first and
+ *                      the input transforms of the second run as ONE relay kernel and the activation between them
+ *                      is never written to memory: 2*count + 1 launches instead of 3*count.  Other boundaries
+ *                      (batch <= 8 on the single-launch kernel, different k, bfloat16 in between) go through an
+ *                      intermediate buffer owned by the stack.  Results equal those of calling circ_fc_forward
+ *                      layer by layer up to float32 rounding.
+ * circ_stack_reserve : allocate every workspace for batches up to max_batch now, so that later forwards only
+ *                      enqueue (needed before stream capture).
+ * circ_stack_relayed : number of layer boundaries the last circ_stack_forward relayed.
+ * circ_stack_destroy : frees the stack (not the layers).  NULL is a no-op.
+ */
+typedef struct circ_stack* circ_stack_handle;
+CIRC_API circ_stack_handle circ_stack_create(const circ_handle* layers, int count);
+CIRC_API int circ_stack_forward(circ_stack_handle s, const void* x, void* y, int batch, void* stream);
+CIRC_API int circ_stack_reserve(circ_stack_handle s, long max_batch);
+CIRC_API int circ_stack_relayed(circ_stack_handle s);
+CIRC_API void circ_stack_destroy(circ_stack_handle s);
+
 /* circ_destroy -- free a handle and everything it owns.  NULL is a no-op. */
 CIRC_API void circ_destroy(circ_handle h);
 

@@ -37,6 +37,11 @@ SIGNATURES = {
     "circ_fc_backward": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _vp]),
     "circ_conv_backward_input": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_conv_backward_weight": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _ci, _vp]),
+    "circ_stack_create": (_vp, [_vp, _ci]),
+    "circ_stack_forward": (_ci, [_vp, _vp, _vp, _ci, _vp]),
+    "circ_stack_reserve": (_ci, [_vp, _cl]),
+    "circ_stack_relayed": (_ci, [_vp]),
+    "circ_stack_destroy": (None, [_vp]),
     "circ_device_status": (_ci, [_vp]),
     "circ_destroy": (None, [_vp]),
     "circ_set_bias": (_ci, [_vp, _vp]),
@@ -194,6 +199,32 @@ def circ_conv_backward_input(h: int, grad_y, grad_x, N: int, H: int, W: int, str
 def circ_conv_backward_weight(h: int, x, grad_y, grad_w, N: int, H: int, W: int, stream=None) -> None:
     """Enqueue ``grad_w[r][r][p][q][k]`` (float32) from the forward input ``x`` and ``grad_y``."""
     _check(load().circ_conv_backward_weight(h, _ptr(x), _ptr(grad_y), _ptr(grad_w), N, H, W, _stream(stream)))
+
+
+def circ_stack_create(layers) -> int:
+    """A stack over fully-connected layer handles (borrowed: destroy the stack first, then the layers)."""
+    arr = (ctypes.c_void_p * len(layers))(*layers)
+    s = load().circ_stack_create(ctypes.addressof(arr), len(layers))
+    if not s:
+        raise CircError(circ_last_code(), circ_last_error())
+    return s
+
+
+def circ_stack_forward(s: int, x, y, batch: int, stream=None) -> None:
+    """Enqueue all layers; boundaries between staged layers of equal block size run as one relay kernel."""
+    _check(load().circ_stack_forward(s, _ptr(x), _ptr(y), batch, _stream(stream)))
+
+
+def circ_stack_reserve(s: int, max_batch: int) -> None:
+    _check(load().circ_stack_reserve(s, max_batch))
+
+
+def circ_stack_relayed(s: int) -> int:
+    return load().circ_stack_relayed(s)
+
+
+def circ_stack_destroy(s: int | None) -> None:
+    load().circ_stack_destroy(s)
 
 
 def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:

@@ -175,6 +175,9 @@ bool tensor_batch_product_supported(int cols);
 // S3 / C3: inverse transforms + bias + activation -> y.
 int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);
 
+// S3 of layer L and S1 of the next layer (same k, its q = L's p) in one launch: Y operand -> X operand (xmode 0 or 1).
+int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, const Extent& ext, cudaStream_t stream);
+
 // S4: the whole FC forward in one launch (small batch, weight-streaming).
 int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStream_t stream);
 bool fused_fc_supported(const Layer* L, int batch);

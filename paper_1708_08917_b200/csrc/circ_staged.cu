@@ -40,46 +40,86 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
     return hi;
 }
 
-// ---- S1: x -> operand X ------------------------------------------------------------------------
-// One transform = (pair c, column block j).  A CTA takes TT = 256 / L consecutive transforms.
-// XMODE 0: float32 operand [problem][col][Kq]                      (FMA contraction, any q)
-// XMODE 1: bfloat16 operand [problem][col][hi | lo][Kq]            (tensor cores, float32 input split in two)
-// XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
-// Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
-template <int K, int EMAX, typename TIN, int XMODE>
-__global__ void __launch_bounds__(Tile<K, EMAX>::NT)
-input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
-                 int B, int Bh, long total) {
-    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW,
-                  kThreads = Tile<K, EMAX>::NT;
-    __shared__ float2 tw[K];
-    __shared__ __align__(16) float2 zs[K][ROW];
-    load_twiddles<K>(tw);
-    pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
-    pdl_trigger();
-
-    const int gi = threadIdx.x / L, l = threadIdx.x % L;
-    const long T = (long)blockIdx.x * TT + gi;
-    float2 v[E];
-    {
-        float re[E], im[E];
+// Operand Y -> tile (the first half of S3): fills zs[bin][transform] for the CTA's TT transforms.
+template <int K, int EMAX, bool VEC>
+__device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW], const float* __restrict__ yop, int p, int Bho,
+                                               long total) {
+    constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
+    const size_t cols = 2 * (size_t)Bho;
+    const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
+    if constexpr (VEC) {
+        // all loads of the tile are issued before the first one is used
+        constexpr int GROUPS = TT / 4;
+        constexpr int ITERS = GROUPS * K / kThreads;
+        static_assert(GROUPS * K % kThreads == 0, "tile must divide evenly among the threads");
+        float4 r0[ITERS], r1[ITERS];
 #pragma unroll
-        for (int r = 0; r < E; ++r) re[r] = im[r] = 0.f;
-        if (T < total) {
-            const int c = (int)(T / q), j = (int)(T % q);
-            load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
-            if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
+        for (int it = 0; it < ITERS; ++it) {
+            const int item = threadIdx.x + it * kThreads;
+            const int grp = item % GROUPS, f = item / GROUPS;
+            const long T0 = (long)blockIdx.x * TT + grp * 4;
+            r0[it] = r1[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (T0 >= total) continue;
+            const int c = (int)(T0 / p), i = (int)(T0 % p);
+            if (f == 0 || f == K / 2) {
+                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                r0[it] = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
+                r1[it] = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
+            } else {
+                const bool mirror = f > K / 2;
+                const int g = mirror ? K - f : f;
+                const float4* r = reinterpret_cast<const float4*>(yop + problem_offset(g + 1, real_sz, cplx_sz) +
+                                                                  ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i);
+                r0[it] = __ldg(r);
+                r1[it] = __ldg(r + 1);
+            }
         }
 #pragma unroll
-        for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
+        for (int it = 0; it < ITERS; ++it) {
+            const int item = threadIdx.x + it * kThreads;
+            const int grp = item % GROUPS, f = item / GROUPS;
+            float4 za, zb;
+            if (f == 0 || f == K / 2) {
+                za = make_float4(r0[it].x, r1[it].x, r0[it].y, r1[it].y);
+                zb = make_float4(r0[it].z, r1[it].z, r0[it].w, r1[it].w);
+            } else {
+                const float sgn = f > K / 2 ? -1.f : 1.f;
+                za = r0[it];
+                zb = r1[it];
+                za.y *= sgn; za.w *= sgn; zb.y *= sgn; zb.w *= sgn;
+            }
+            *reinterpret_cast<float4*>(&zs[f][grp * 4]) = za;
+            *reinterpret_cast<float4*>(&zs[f][grp * 4 + 2]) = zb;
+        }
+    } else {
+        for (int item = threadIdx.x; item < TT * K; item += kThreads) {
+            const int tl = item % TT, f = item / TT;
+            const long T2 = (long)blockIdx.x * TT + tl;
+            if (T2 >= total) continue;
+            const int c = (int)(T2 / p), i = (int)(T2 % p);
+            float2 z;
+            if (f == 0 || f == K / 2) {
+                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
+                z.x = __ldg(yg + (size_t)c * p + i);
+                z.y = __ldg(yg + ((size_t)Bho + c) * p + i);
+            } else if (f < K / 2) {
+                const float* yg = yop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * p + 2 * i;
+                z = __ldg(reinterpret_cast<const float2*>(yg));
+            } else {
+                const float* yg = yop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bho + c) * 2 * p + 2 * i;
+                z = __ldg(reinterpret_cast<const float2*>(yg));
+                z.y = -z.y;
+            }
+            zs[f][tl] = z;
+        }
     }
-    __syncthreads();  // twiddles ready
-    fft_forward<K, EMAX>(v, l, tw);
-    const int f2 = lane_residue<K, EMAX>(l);
-#pragma unroll
-    for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
-    __syncthreads();
+}
 
+// Tile -> operand X (the second half of S1): zs[bin][transform] holds the spectra of the CTA's TT transforms.
+template <int K, int EMAX, int XMODE>
+__device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>::ROW], void* __restrict__ xop, int q, int Bh,
+                                                long total) {
+    constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
     const size_t cols = 2 * (size_t)Bh;
     constexpr int NPART = XMODE == 1 ? 2 : 1;
     const size_t real_sz = cols * q * NPART, cplx_sz = 2 * real_sz;
@@ -147,6 +187,48 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     }
 }
 
+// ---- S1: x -> operand X ------------------------------------------------------------------------
+// One transform = (pair c, column block j).  A CTA takes TT = 256 / L consecutive transforms.
+// XMODE 0: float32 operand [problem][col][Kq]                      (FMA contraction, any q)
+// XMODE 1: bfloat16 operand [problem][col][hi | lo][Kq]            (tensor cores, float32 input split in two)
+// XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
+// Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
+template <int K, int EMAX, typename TIN, int XMODE>
+__global__ void __launch_bounds__(Tile<K, EMAX>::NT)
+input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
+                 int B, int Bh, long total) {
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
+    __shared__ float2 tw[K];
+    __shared__ __align__(16) float2 zs[K][ROW];
+    load_twiddles<K>(tw);
+    pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
+    pdl_trigger();
+
+    const int gi = threadIdx.x / L, l = threadIdx.x % L;
+    const long T = (long)blockIdx.x * TT + gi;
+    float2 v[E];
+    {
+        float re[E], im[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) re[r] = im[r] = 0.f;
+        if (T < total) {
+            const int c = (int)(T / q), j = (int)(T % q);
+            load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
+            if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
+        }
+#pragma unroll
+        for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
+    }
+    __syncthreads();  // twiddles ready
+    fft_forward<K, EMAX>(v, l, tw);
+    const int f2 = lane_residue<K, EMAX>(l);
+#pragma unroll
+    for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
+    __syncthreads();
+
+    scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total);
+}
+
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
 // One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
@@ -154,15 +236,12 @@ template <int K, int EMAX, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
-    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW,
-                  kThreads = Tile<K, EMAX>::NT;
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     __shared__ float2 tw[K];
     __shared__ __align__(16) float2 zs[K][ROW];
     load_twiddles<K>(tw);
     pdl_wait();     // Y is written by the contraction kernel before this one
     pdl_trigger();
-    const size_t cols = 2 * (size_t)Bho;
-    const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
 
     // the bias of this thread's outputs is fetched now, long before the epilogue needs it
     float bv[E];
@@ -173,72 +252,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         if (bias && Tb < total) load_run<E>(bias + (int)(Tb % p) * K + E * (threadIdx.x % L), bv);
     }
 
-    if constexpr (VEC) {
-        // all loads of the tile are issued before the first one is used
-        constexpr int GROUPS = TT / 4;
-        constexpr int ITERS = GROUPS * K / kThreads;
-        static_assert(GROUPS * K % kThreads == 0, "tile must divide evenly among the threads");
-        float4 r0[ITERS], r1[ITERS];
-#pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            const int item = threadIdx.x + it * kThreads;
-            const int grp = item % GROUPS, f = item / GROUPS;
-            const long T0 = (long)blockIdx.x * TT + grp * 4;
-            r0[it] = r1[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (T0 >= total) continue;
-            const int c = (int)(T0 / p), i = (int)(T0 % p);
-            if (f == 0 || f == K / 2) {
-                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                r0[it] = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
-                r1[it] = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
-            } else {
-                const bool mirror = f > K / 2;
-                const int g = mirror ? K - f : f;
-                const float4* r = reinterpret_cast<const float4*>(yop + problem_offset(g + 1, real_sz, cplx_sz) +
-                                                                  ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i);
-                r0[it] = __ldg(r);
-                r1[it] = __ldg(r + 1);
-            }
-        }
-#pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
-            const int item = threadIdx.x + it * kThreads;
-            const int grp = item % GROUPS, f = item / GROUPS;
-            float4 za, zb;
-            if (f == 0 || f == K / 2) {
-                za = make_float4(r0[it].x, r1[it].x, r0[it].y, r1[it].y);
-                zb = make_float4(r0[it].z, r1[it].z, r0[it].w, r1[it].w);
-            } else {
-                const float sgn = f > K / 2 ? -1.f : 1.f;
-                za = r0[it];
-                zb = r1[it];
-                za.y *= sgn; za.w *= sgn; zb.y *= sgn; zb.w *= sgn;
-            }
-            *reinterpret_cast<float4*>(&zs[f][grp * 4]) = za;
-            *reinterpret_cast<float4*>(&zs[f][grp * 4 + 2]) = zb;
-        }
-    } else {
-        for (int item = threadIdx.x; item < TT * K; item += kThreads) {
-            const int tl = item % TT, f = item / TT;
-            const long T2 = (long)blockIdx.x * TT + tl;
-            if (T2 >= total) continue;
-            const int c = (int)(T2 / p), i = (int)(T2 % p);
-            float2 z;
-            if (f == 0 || f == K / 2) {
-                const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                z.x = __ldg(yg + (size_t)c * p + i);
-                z.y = __ldg(yg + ((size_t)Bho + c) * p + i);
-            } else if (f < K / 2) {
-                const float* yg = yop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * p + 2 * i;
-                z = __ldg(reinterpret_cast<const float2*>(yg));
-            } else {
-                const float* yg = yop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bho + c) * 2 * p + 2 * i;
-                z = __ldg(reinterpret_cast<const float2*>(yg));
-                z.y = -z.y;
-            }
-            zs[f][tl] = z;
-        }
-    }
+    gather_operand<K, EMAX, VEC>(zs, yop, p, Bho, total);
     __syncthreads();
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
@@ -264,6 +278,57 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     }
     store_run<E>(y + (size_t)c * m + col, re);
     if (c + Bho < Bo) store_run<E>(y + (size_t)(c + Bho) * m + col, im);
+}
+
+// ---- relay: operand Y of one layer -> operand X of the next -----------------------------------------
+// Between two stacked fully-connected layers with the same block size, the activation y = psi(a + theta) is only
+// ever transformed again: this kernel is S3 of the first layer and S1 of the second in one launch, with the
+// activation kept in registers (inverse transform, bias, activation, forward transform); y never reaches memory.
+// One transform = (pair c, block i); the first layer's row blocks are the second layer's column blocks.
+template <int K, int EMAX, int XMODE, bool VEC>
+__global__ void __launch_bounds__(Tile<K, EMAX>::NT)
+relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float* __restrict__ bias, int relu, int p, int B, int Bh,
+             long total) {
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
+    __shared__ float2 tw[K];
+    __shared__ __align__(16) float2 zs[K][ROW];
+    load_twiddles<K>(tw);
+    pdl_wait();
+    pdl_trigger();
+    const int gi = threadIdx.x / L, l = threadIdx.x % L;
+    const long T = (long)blockIdx.x * TT + gi;
+    const bool live = T < total;
+    float bv[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) bv[r] = 0.f;
+    if (bias && live) load_run<E>(bias + (int)(T % p) * K + E * l, bv);
+
+    gather_operand<K, EMAX, VEC>(zs, yop, p, Bh, total);
+    __syncthreads();
+    const int f2 = lane_residue<K, EMAX>(l);
+    float2 v[E];
+#pragma unroll
+    for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[f2 + L * f1][gi] : make_float2(0.f, 0.f);
+    fft_inverse<K, EMAX>(v, l, tw);
+    {
+        // the second sample of the last pair does not exist when the batch is odd: it must enter the next layer as zero
+        const bool second = live && (int)(T / p) + Bh < B;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            float re = v[r].x + bv[r], im = v[r].y + bv[r];
+            if (relu) {
+                re = fmaxf(re, 0.f);
+                im = fmaxf(im, 0.f);
+            }
+            v[r] = make_float2(live ? re : 0.f, second ? im : 0.f);
+        }
+    }
+    fft_forward<K, EMAX>(v, l, tw);
+    __syncthreads();  // every thread has taken its bins out of the tile
+#pragma unroll
+    for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
+    __syncthreads();
+    scatter_operand<K, EMAX, XMODE>(zs, xop, p, Bh, total);
 }
 
 // ---- launchers -------------------------------------------------------------------------------------
@@ -355,6 +420,45 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
             } else {
                 if (vec) launch(float{}, std::true_type{}); else launch(float{}, std::false_type{});
             }
+        };
+        if (small) with_shape(std::integral_constant<int, SmallShape<K>::EMAX>{});
+        else with_shape(std::integral_constant<int, 16>{});
+        return CIRC_OK;
+    };
+    const int rc = dispatch_k(L->geo.k, go);
+    if (rc != CIRC_OK) return rc;
+    count_launches(1);
+    CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+    return CIRC_OK;
+}
+
+int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, const Extent& ext, cudaStream_t stream) {
+    const int p = L->geo.p;
+    const long total = (long)ext.Bho * p;
+    if (xmode != 0 && xmode != 1) {
+        set_error(CIRC_ERR_ARG, "relay operand mode %d", xmode);
+        return CIRC_ERR_ARG;
+    }
+    if (xmode == 1 && (p % 8) != 0) {
+        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need p %% 8 == 0 (p=%d)", p);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    const bool small = latency_bound(total, L->geo.k);
+    auto go = [&](auto kc) -> int {
+        constexpr int K = decltype(kc)::value;
+        auto with_shape = [&](auto ec) {
+            constexpr int EMAX = decltype(ec)::value;
+            constexpr int TT = Tile<K, EMAX>::TT;
+            const unsigned blocks = (unsigned)((total + TT - 1) / TT);
+            auto launch = [&](auto mode, auto vec) {
+                constexpr int XMODE = decltype(mode)::value;
+                constexpr bool VEC = decltype(vec)::value;
+                launch_kernel(false, relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream, yop, xop_next,
+                              static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bo, ext.Bho, total);
+            };
+            if (xmode == 1) launch(std::integral_constant<int, 1>{}, std::true_type{});
+            else if ((p % 4) == 0) launch(std::integral_constant<int, 0>{}, std::true_type{});
+            else launch(std::integral_constant<int, 0>{}, std::false_type{});
         };
         if (small) with_shape(std::integral_constant<int, SmallShape<K>::EMAX>{});
         else with_shape(std::integral_constant<int, 16>{});
