@@ -30,6 +30,8 @@ constexpr int kTileCols = 128;            // MMA M: batch columns / pixels per t
 constexpr int kKBlock = 64;               // bf16 elements per stage along K (one 128-byte swizzle row)
 constexpr int kMaxStages = 8;        // ring depth is chosen per launch (as many stages as shared memory holds)
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded wait: polls before giving up
+constexpr int kStagePitch = 36;           // floats per row of the epilogue's 32 x 32 staging tiles (16-byte aligned, conflict-free)
+constexpr int kStageOutBytes = 4 * 32 * kStagePitch * 4;   // one staging tile per epilogue warp
 
 struct TcArgs {
     float* yop;
@@ -417,9 +419,25 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             }
         }
     } else {
-        // ---- epilogue: TMEM -> registers -> Y[col][row] ------------------------------------------
+        // ---- epilogue: TMEM -> registers -> shared memory -> Y[col][row] ----------------------------
+        // A thread reads one TMEM lane = one column (pixel) of the tile, i.e. a run of rows that is
+        // contiguous in Y, but the 32 lanes of a warp then hold 32 different memory lines.  The warp
+        // therefore turns each 32 x 32 chunk around in shared memory and stores it with 8 lanes per
+        // pixel (one 128-byte line per pixel, 512 contiguous bytes per instruction when the pixels
+        // are neighbours), instead of 32 scattered 16-byte pieces per instruction.
         const int quarter = warp & 3;                 // a warp may only read its own 32 TMEM lanes
-        const int r = quarter * 32 + lane;            // row of the tile = flattened pixel index at the input pitch
+        float* stg = reinterpret_cast<float*>(ring + (size_t)g.stages * stage_bytes) + quarter * (32 * kStagePitch);
+        const int sub = lane >> 3, seg = lane & 7;    // store phase: pixel sub + 4 * it of the warp, floats 4 seg .. 4 seg + 3
+        // tile-independent position of the pixels this lane touches: row of the tile = flattened pixel
+        // index at the input pitch
+        uint32_t px_pos[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int rr = quarter * 32 + it * 4 + sub;
+            const int h2 = rr / g.pitch;
+            px_pos[it] = ((uint32_t)h2 << 16) | (uint32_t)(rr - h2 * g.pitch);
+        }
+        const int r = quarter * 32 + lane;            // the lane's own row (scalar path)
         const int hh = r / g.pitch, ww = r - hh * g.pitch;
         int buf = 0;
         uint32_t acc_par = 0;
@@ -428,36 +446,50 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], acc_par, &abort_flag));  // warp-uniform
             if (!ok) break;
             tc_fence_after();
-            const int ho = t.ho0 + hh, wo = t.wo0 + ww;
-            const bool live = hh < g.th && ww < g.tw && ho < g.Ho && wo < g.Wo;
             const size_t y_real = (size_t)g.cols_out * g.p;
-            float* yrow = g.yop + problem_offset(t.prob, y_real, 2 * y_real) +
-                          ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg + t.row0;
+            float* ytile = g.yop + problem_offset(t.prob, y_real, 2 * y_real) + t.row0;
+            const bool vec = (t.Mg & 3) == 0;         // rows come in whole float4 (row0, c0 and bn are multiples of 16)
             for (int c0 = 0; c0 < t.bn; c0 += 32) {
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)buf * acc_cols + (uint32_t)c0, acc);
-                if (live) {
-                    // columns of this chunk that belong to the tile (its row tile may be narrower than 32
-                    // columns, and the last row tile may reach past the matrix)
-                    int nvalid = t.bn - c0;
-                    if (nvalid > t.Mg - t.row0 - c0) nvalid = t.Mg - t.row0 - c0;
-                    if (nvalid >= 32 && (t.Mg & 3) == 0) {
+                if (c0 + 32 >= t.bn) {
+                    // last read of this accumulator: it may be overwritten by the tile after next
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
+                // columns of this chunk that belong to the tile (its row tile may be narrower than 32
+                // columns, and the last row tile may reach past the matrix)
+                int nvalid = t.bn - c0;
+                if (nvalid > t.Mg - t.row0 - c0) nvalid = t.Mg - t.row0 - c0;
+                if (nvalid > 32) nvalid = 32;
+                if (vec) {
+                    float* mine = stg + lane * kStagePitch;
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4)
-                            *reinterpret_cast<float4*>(yrow + c0 + e) =
-                                make_float4(__uint_as_float(acc[e]), __uint_as_float(acc[e + 1]), __uint_as_float(acc[e + 2]),
-                                            __uint_as_float(acc[e + 3]));
-                    } else {
+                    for (int e = 0; e < 32; e += 4)
+                        *reinterpret_cast<float4*>(mine + e) = make_float4(__uint_as_float(acc[e]), __uint_as_float(acc[e + 1]),
+                                                                           __uint_as_float(acc[e + 2]), __uint_as_float(acc[e + 3]));
+                    __syncwarp();
+#pragma unroll
+                    for (int it = 0; it < 8; ++it) {
+                        const int h2 = (int)(px_pos[it] >> 16), w2 = (int)(px_pos[it] & 0xffffu);
+                        const int ho = t.ho0 + h2, wo = t.wo0 + w2;
+                        if (h2 < g.th && w2 < g.tw && ho < g.Ho && wo < g.Wo && seg * 4 < nvalid) {
+                            const float4 v = *reinterpret_cast<const float4*>(stg + (it * 4 + sub) * kStagePitch + seg * 4);
+                            *reinterpret_cast<float4*>(ytile + ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg + c0 + seg * 4) = v;
+                        }
+                    }
+                    __syncwarp();
+                } else {
+                    const int ho = t.ho0 + hh, wo = t.wo0 + ww;
+                    if (hh < g.th && ww < g.tw && ho < g.Ho && wo < g.Wo) {
+                        float* yrow = ytile + ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg;
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
                             if (e < nvalid) yrow[c0 + e] = __uint_as_float(acc[e]);
                     }
                 }
             }
-            // this accumulator may be overwritten by the tile after next
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_empty[buf]);
             if (buf == 1) acc_par ^= 1u;
             buf ^= 1;
         }
@@ -529,7 +561,7 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
     // accumulators of bn_max columns per CTA keep both within the 512 columns of tensor memory.
     int ctas_per_sm = 1;
     {
-        const int fit2 = (int)((98 * 1024) / stage_bytes);   // stages per CTA when two CTAs share an SM
+        const int fit2 = (int)((93 * 1024) / stage_bytes);   // stages per CTA when two CTAs share an SM (ring + staging + reserve <= 114 KB each)
         if (ctas > 148 && iters_max <= 4 && bn_max <= 128 && fit2 >= 3) {
             ctas_per_sm = 2;                                  // only when each CTA still gets a ring of three or more
             if (g.stages > fit2) g.stages = fit2;
@@ -539,12 +571,12 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
         if (deep > kMaxStages) deep = kMaxStages;
         if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
     }
-    const size_t smem = (size_t)g.stages * stage_bytes + 1024;
+    const size_t smem = (size_t)g.stages * stage_bytes + 1024 + kStageOutBytes;
     static thread_local int configured_device = -1;
     int dev = 0;
     cudaGetDevice(&dev);
     if (configured_device != dev) {
-        CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024),
+        CIRC_CUDA_TRY(cudaFuncSetAttribute(contract_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024 + kStageOutBytes),
                       CIRC_ERR_CUDA);
         configured_device = dev;
     }
