@@ -28,6 +28,7 @@ namespace circ {
 constexpr int kTcThreads = 192;
 constexpr int kTileCols = 128;            // MMA M: batch columns / pixels per tile
 constexpr int kKBlock = 64;               // bf16 elements per stage along K (one 128-byte swizzle row)
+constexpr int kMaxAcc = 8;           // accumulators in tensor memory (chosen per launch: as many as 512 columns hold)
 constexpr int kMaxStages = 8;        // ring depth is chosen per launch (as many stages as shared memory holds)
 constexpr uint32_t kSpinLimit = 1u << 22; // bounded wait: polls before giving up
 constexpr int kStagePitch = 36;           // floats per row of the epilogue's 32 x 32 staging tiles (16-byte aligned, conflict-free)
@@ -50,6 +51,7 @@ struct TcArgs {
     int nt_real, nt_cplx;    // row tiles per problem
     int ctas_real;           // CTAs that serve the two real problems
     int stages;              // depth of the shared-memory ring (<= kMaxStages)
+    int nacc;                // accumulators in tensor memory (2 .. kMaxAcc)
     long tiles;              // output tiles in total; CTAs walk them with a grid stride
     long cols_out;           // V * Ho * Wo
 };
@@ -106,15 +108,33 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// The MMA warp runs its loop with all 32 lanes on warp-uniform values (so that descriptors and
+// addresses live in uniform registers) and only the instructions below are restricted to one
+// elected lane, by a guard predicate rather than a branch.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t leader;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(leader));
+    return leader;
+}
+__device__ __forceinline__ void tc_commit(uint64_t* bar, uint32_t leader) {
+    asm volatile(
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(smem_u32(bar)), "r"(leader) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
+                                            uint32_t leader) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -198,28 +218,28 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // start-address field (16-byte units): 8 units per tile row, a_step per tap, 2 per K step.
 template <int R, int KSTEPS>
 __device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step, uint64_t a_step,
-                                           uint32_t idesc, uint32_t& accumulate) {
+                                           uint32_t idesc, uint32_t& accumulate, uint32_t leader) {
 #pragma unroll
     for (int di = 0; di < R; ++di) {
 #pragma unroll
         for (int dj = 0; dj < R; ++dj) {
             const uint64_t x = dx + (uint64_t)di * row_step + (uint64_t)(dj * 8);
             const uint64_t w = da + (uint64_t)(di * R + dj) * a_step;
-            tc_mma_bf16(d_tmem, x, w, idesc, accumulate);
+            tc_mma_bf16(d_tmem, x, w, idesc, accumulate, leader);
 #pragma unroll
-            for (int k4 = 1; k4 < KSTEPS; ++k4) tc_mma_bf16(d_tmem, x + 2 * k4, w + 2 * k4, idesc, 1u);
+            for (int k4 = 1; k4 < KSTEPS; ++k4) tc_mma_bf16(d_tmem, x + 2 * k4, w + 2 * k4, idesc, 1u, leader);
             accumulate = 1u;
         }
     }
 }
 template <int R>
 __device__ __forceinline__ void issue_taps_k(int ksteps, uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step,
-                                             uint64_t a_step, uint32_t idesc, uint32_t& accumulate) {
+                                             uint64_t a_step, uint32_t idesc, uint32_t& accumulate, uint32_t leader) {
     switch (ksteps) {
-        case 1: issue_taps<R, 1>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
-        case 2: issue_taps<R, 2>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
-        case 3: issue_taps<R, 3>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
-        default: issue_taps<R, 4>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        case 1: issue_taps<R, 1>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
+        case 2: issue_taps<R, 2>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
+        case 3: issue_taps<R, 3>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
+        default: issue_taps<R, 4>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
     }
 }
 
@@ -233,7 +253,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                    const __grid_constant__ CUtensorMap map_xhi_cplx, const __grid_constant__ CUtensorMap map_xlo_cplx,
                    TcArgs g) {
     extern __shared__ unsigned char smem_dyn[];
-    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[kMaxAcc], acc_empty[kMaxAcc];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
@@ -247,7 +267,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     uint32_t acc_cols = 32;                      // columns of one accumulator
     while ((int)acc_cols < bn_max) acc_cols <<= 1;
-    const uint32_t tmem_cols = 2 * acc_cols;     // two accumulators (<= 512 columns)
+    const uint32_t tmem_cols = (uint32_t)g.nacc * acc_cols;   // a power of two, <= 512 columns
 
     if (warp == 0 && lane == 0) {
         // start fetching the copy descriptors now; the first TMA would otherwise wait for them
@@ -261,7 +281,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < g.nacc; ++b) {
             mbar_init(&acc_full[b], 1);
             mbar_init(&acc_empty[b], 4);         // one arrival per epilogue warp
         }
@@ -333,8 +353,9 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issuer -------------------------------------------------------------------------
-        if (lane == 0) {
+        // ---- MMA issuer (all lanes walk the loop; one elected lane issues) ---------------------------
+        {
+            const uint32_t leader = elect_one();
             int s = 0;
             uint32_t par = 0;
             int buf = 0;
@@ -362,16 +383,16 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                         if (g.taps == 1 && krem >= kKBlock) {
                             // fully-connected fast path: four K steps of 16 per product
                             const uint64_t dxh = smem_desc_sw128(xs), dah = smem_desc_sw128(as);
-                            tc_mma_bf16(d_tmem, dxh, dah, idesc, accumulate);
-                            tc_mma_bf16(d_tmem, dxh + 2, dah + 2, idesc, 1u);
-                            tc_mma_bf16(d_tmem, dxh + 4, dah + 4, idesc, 1u);
-                            tc_mma_bf16(d_tmem, dxh + 6, dah + 6, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dxh, dah, idesc, accumulate, leader);
+                            tc_mma_bf16(d_tmem, dxh + 2, dah + 2, idesc, 1u, leader);
+                            tc_mma_bf16(d_tmem, dxh + 4, dah + 4, idesc, 1u, leader);
+                            tc_mma_bf16(d_tmem, dxh + 6, dah + 6, idesc, 1u, leader);
                             if (g.npass == 3) {
                                 const uint64_t dxl = smem_desc_sw128(xs + x_bytes), dal = smem_desc_sw128(a_lo);
 #pragma unroll
-                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxh + 2 * k4, dal + 2 * k4, idesc, 1u);
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxh + 2 * k4, dal + 2 * k4, idesc, 1u, leader);
 #pragma unroll
-                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxl + 2 * k4, dah + 2 * k4, idesc, 1u);
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxl + 2 * k4, dah + 2 * k4, idesc, 1u, leader);
                             }
                             accumulate = 1u;
                         } else {
@@ -386,36 +407,36 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                                 const uint64_t dx = prod == 2 ? dx_lo : dx_hi;
                                 const uint64_t da = prod == 1 ? da_lo : da_hi;
                                 if (g.r == 3) {
-                                    issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
+                                    issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate, leader);
                                 } else if (g.r == 1) {
-                                    issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
+                                    issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate, leader);
                                 } else {
                                     uint64_t dx_row = dx, db = da;
                                     for (int di = 0; di < g.r; ++di, dx_row += row_step) {
                                         uint64_t dxx = dx_row;
                                         for (int dj = 0; dj < g.r; ++dj, dxx += 8, db += tap_step) {
-                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate);
+                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate, leader);
                                             for (int k4 = 1; k4 < ksteps; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
-                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u);
+                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u, leader);
                                             accumulate = 1u;
                                         }
                                     }
                                 }
                             }
                         }
-                        tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
+                        tc_commit(&empty_bar[s], leader);   // stage free once these MMAs have read it
                         if (++s == g.stages) {
                             s = 0;
                             par ^= 1u;
                         }
                     }
                 }
-                if (ok) tc_commit(&acc_full[buf]);  // accumulator complete
-                if (buf == 1) {
+                if (ok) tc_commit(&acc_full[buf], leader);  // accumulator complete
+                if (++buf == g.nacc) {
+                    buf = 0;
                     acc_par ^= 1u;
                     acc_wrapped = true;
                 }
-                buf ^= 1;
             }
         }
     } else {
@@ -490,8 +511,10 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                     }
                 }
             }
-            if (buf == 1) acc_par ^= 1u;
-            buf ^= 1;
+            if (++buf == g.nacc) {
+                buf = 0;
+                acc_par ^= 1u;
+            }
         }
     }
 
@@ -570,6 +593,15 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
         int deep = ctas_per_sm == 2 ? fit2 : (int)((198 * 1024) / stage_bytes);
         if (deep > kMaxStages) deep = kMaxStages;
         if (ctas > 148 * ctas_per_sm && deep > g.stages) g.stages = deep;
+    }
+    {
+        // Accumulators: as many as tensor memory holds (512 columns per SM, shared by the CTAs on it).  With
+        // small tiles the hand-over MMA -> epilogue -> MMA is a chain of barrier latencies; several
+        // accumulators in flight take it off the critical path.
+        int acc_cols = 32;
+        while (acc_cols < bn_max) acc_cols <<= 1;
+        g.nacc = (ctas_per_sm == 2 ? 256 : 512) / acc_cols;
+        if (g.nacc > kMaxAcc) g.nacc = kMaxAcc;
     }
     const size_t smem = (size_t)g.stages * stage_bytes + 1024 + kStageOutBytes;
     static thread_local int configured_device = -1;
