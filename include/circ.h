@@ -41,7 +41,7 @@ typedef struct circ_layer* circ_handle; /* opaque, owned by the library */
 enum {
     CIRC_OK = 0,
     CIRC_ERR_ARG = -1,            /* NULL / misaligned pointer, bad enum value, wrong handle kind */
-    CIRC_ERR_SHAPE = -2,          /* k not a power of two in [4,256], k does not divide m or n, batch < 1 ... */
+    CIRC_ERR_SHAPE = -2,          /* unsupported block size, k does not divide m or n, batch < 1 ... */
     CIRC_ERR_ALLOC = -3,          /* device or host allocation failed */
     CIRC_ERR_CUDA = -4,           /* a CUDA runtime call or a kernel launch failed */
     CIRC_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up */
@@ -60,9 +60,11 @@ enum {
 
 /*
  * circ_fc_create -- build a fully-connected block-circulant layer (Sec. 3.1).
- *   m, n : output / input widths; k : block size, a power of two in [4, 256]
+ *   m, n : output / input widths; k : block size, a power of two in [4, 1024]
  *          that divides both (the paper defines p = m / k, q = n / k and has no
- *          remainder rule; pad on the caller's side).
+ *          remainder rule; pad on the caller's side).  Blocks above 256 are built
+ *          from the same small transform with more butterfly levels (the recursive
+ *          construction of Sec. 4.1); they run on the three-launch paths only.
  *   w    : float32 defining vectors, layout [p][q][k]: w[(i*q + j)*k + t] is
  *          element t of w_ij.  HOST or DEVICE pointer (detected); read during
  *          the call, the caller keeps ownership.

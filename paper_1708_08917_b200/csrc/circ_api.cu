@@ -63,7 +63,7 @@ struct StageTimer {
     }
 };
 
-static bool pow2_in_range(int k) { return k >= 4 && k <= 256 && (k & (k - 1)) == 0; }
+static bool pow2_in_range(int k) { return k >= 4 && k <= 1024 && (k & (k - 1)) == 0; }
 
 // Copy `count` floats from a host or device pointer into fresh device memory.
 static int to_device(const float* src, size_t count, float** out) {
@@ -118,7 +118,7 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
         return nullptr;
     }
     if (!pow2_in_range(k)) {
-        set_error(CIRC_ERR_SHAPE, "block size k=%d must be a power of two in [4, 256]", k);
+        set_error(CIRC_ERR_SHAPE, "block size k=%d must be a power of two in [4, 1024]", k);
         return nullptr;
     }
     if (m <= 0 || n <= 0 || m % k || n % k) {

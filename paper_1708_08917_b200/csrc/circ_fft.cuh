@@ -1,4 +1,4 @@
-// Register / warp-shuffle complex FFTs of size K = 4 .. 256 (powers of two).
+// Register / warp-shuffle complex FFTs of size K = 4 .. 1024 (powers of two).
 //
 // The layer needs real transforms of real signals (Sec. 4.1: real inputs give a
 // conjugate-symmetric spectrum, so half of it is redundant).  That redundancy is
@@ -9,7 +9,8 @@
 // butterfly count per real signal is that of a half-size complex transform.
 //
 // A transform of size K is spread over L lanes of a warp, E points per lane
-// (K = L * E, E <= 16).  Lane l holds the contiguous samples z[E*l .. E*l+E-1],
+// (K = L * E, E <= 16; sizes above 512 take E = K / 32 so that L stays one warp: the larger block is
+// built from the same small in-register transform plus more cross-lane butterfly levels, Sec. 4.1).  Lane l holds the contiguous samples z[E*l .. E*l+E-1],
 // so global loads and stores are 16-byte vectors.  With f = f2 + L*f1:
 //
 //   Z[f2 + L f1] = sum_r w_E^(r f1) * [ w_K^(r f2) * ( sum_l w_L^(l f2) z[E l + r] ) ]
@@ -34,9 +35,9 @@ namespace circ {
 // too small to fill the machine (latency).
 template <int K, int EMAX = 16>
 struct FftShape {
-    static_assert(K >= 4 && K <= 256 && (K & (K - 1)) == 0, "block size must be a power of two in [4,256]");
+    static_assert(K >= 4 && K <= 1024 && (K & (K - 1)) == 0, "block size must be a power of two in [4,1024]");
     static_assert(EMAX == 4 || EMAX == 8 || EMAX == 16, "points per lane: 4, 8 or 16");
-    static constexpr int E = K < EMAX ? K : EMAX;  // points per lane
+    static constexpr int E = K / 32 > EMAX ? K / 32 : (K < EMAX ? K : EMAX);  // points per lane (at most 32 lanes)
     static constexpr int L = K / E;                // lanes per transform
     static_assert(L <= 32, "a transform must fit one warp");
     static constexpr int LOG_L = L == 1 ? 0 : L == 2 ? 1 : L == 4 ? 2 : L == 8 ? 3 : L == 16 ? 4 : 5;
@@ -76,6 +77,23 @@ __device__ __forceinline__ float2 mul_w16(float2 a) {
     }
 }
 
+// Multiply by exp(-+ 2 pi i IDX / 32), IDX in [0, 16): the last level of a 32-point in-register transform.
+template <int IDX, bool INV>
+__device__ __forceinline__ float2 mul_w32(float2 a) {
+    if constexpr ((IDX & 1) == 0) {
+        return mul_w16<IDX / 2, INV>(a);
+    } else {
+        constexpr float C[4] = {0.98078528040323044913f, 0.83146961230254523708f, 0.55557023301960222474f,
+                                0.19509032201612826785f};   // cos(pi/16), cos(3pi/16), cos(5pi/16), cos(7pi/16)
+        constexpr int h = (IDX & 7) >> 1;                   // IDX = 1,3,5,7 -> 0..3; IDX = 9,11,13,15 -> 0..3
+        // first quadrant: (cos, sin) = (C[h], C[3-h]); second quadrant (IDX > 8): (-C[3-h], C[h])
+        constexpr float c = IDX < 8 ? C[h] : -C[3 - h];
+        constexpr float s = IDX < 8 ? C[3 - h] : C[h];
+        return INV ? make_float2(fmaf(a.x, c, -a.y * s), fmaf(a.x, s, a.y * c))
+                   : make_float2(fmaf(a.x, c, a.y * s), fmaf(a.y, c, -a.x * s));
+    }
+}
+
 template <int E>
 __host__ __device__ constexpr int bitrev_const(int i) {
     int r = 0;
@@ -93,7 +111,7 @@ struct DitLevel {
 #pragma unroll
         for (int g = 0; g < E; g += 2 * HALF) {
             float2 a = t[g + J];
-            float2 b = mul_w16<J*(8 / HALF), INV>(t[g + J + HALF]);
+            float2 b = mul_w32<J*(16 / HALF), INV>(t[g + J + HALF]);
             t[g + J] = cadd(a, b);
             t[g + J + HALF] = csub(a, b);
         }

@@ -8,6 +8,8 @@
 // memory walks along a row (consecutive transforms of one bin), which is also the direction in
 // which the operand is contiguous, so those global accesses are full coalesced runs.
 #include <type_traits>
+#include <utility>
+#include <vector>
 
 #include "circ_common.cuh"
 #include "circ_fft.cuh"
@@ -22,10 +24,11 @@ namespace circ {
 template <int K, int EMAX>
 struct Tile {
     static constexpr int L = FftShape<K, EMAX>::L;
-    static constexpr int NT = (K >= 128 && EMAX == 16) ? 256 : 128;   // threads per CTA: small CTAs fill the SMs more evenly
+    static constexpr int NT = K >= 1024 ? 128 : (K >= 128 && EMAX == 16) ? 256 : 128;   // threads per CTA: small CTAs fill the SMs more evenly
     static constexpr int TT = NT / L;
     static constexpr int PAD = L == 1 ? 0 : (L >= 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
     static constexpr int ROW = TT + PAD;
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)K + (size_t)K * ROW);   // twiddle table + staging tile (dynamic shared memory)
 };
 
 __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
@@ -198,8 +201,9 @@ __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
                  int B, int Bh, long total) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
-    __shared__ float2 tw[K];
-    __shared__ __align__(16) float2 zs[K][ROW];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* tw = reinterpret_cast<float2*>(smem_raw);
+    float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
     pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
     pdl_trigger();
@@ -237,8 +241,9 @@ __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
                    const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
-    __shared__ float2 tw[K];
-    __shared__ __align__(16) float2 zs[K][ROW];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* tw = reinterpret_cast<float2*>(smem_raw);
+    float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
     pdl_wait();     // Y is written by the contraction kernel before this one
     pdl_trigger();
@@ -290,8 +295,9 @@ __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float* __restrict__ bias, int relu, int p, int B, int Bh,
              long total) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
-    __shared__ float2 tw[K];
-    __shared__ __align__(16) float2 zs[K][ROW];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* tw = reinterpret_cast<float2*>(smem_raw);
+    float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
     pdl_wait();
     pdl_trigger();
@@ -332,6 +338,21 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
 }
 
 // ---- launchers -------------------------------------------------------------------------------------
+// Kernels whose tile exceeds the default 48 KB of dynamic shared memory (k = 1024) opt in once per device.
+template <typename Kern>
+static void allow_smem(Kern kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return;
+    // remembered per (kernel, device); kernels of different block sizes share one function type, so the key is the pointer
+    static thread_local std::vector<std::pair<const void*, int>> configured;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const std::pair<const void*, int> key(reinterpret_cast<const void*>(kernel), dev);
+    for (const auto& c : configured)
+        if (c == key) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    configured.push_back(key);
+}
+
 template <typename F>
 static int dispatch_k(int k, F&& f) {
     switch (k) {
@@ -342,6 +363,8 @@ static int dispatch_k(int k, F&& f) {
         case 64: return f(std::integral_constant<int, 64>{});
         case 128: return f(std::integral_constant<int, 128>{});
         case 256: return f(std::integral_constant<int, 256>{});
+        case 512: return f(std::integral_constant<int, 512>{});
+        case 1024: return f(std::integral_constant<int, 1024>{});
     }
     set_error(CIRC_ERR_SHAPE, "block size %d not supported", k);
     return CIRC_ERR_SHAPE;
@@ -351,7 +374,7 @@ static int dispatch_k(int k, F&& f) {
 // (8 for k = 256), which quarters every thread's dependent chain for problems that are latency-bound.
 template <int K>
 struct SmallShape {
-    static constexpr int EMAX = K <= 8 ? 16 : (K <= 128 ? 4 : 8);   // k = 4, 8 already sit in one lane
+    static constexpr int EMAX = (K <= 8 || K >= 512) ? 16 : (K <= 128 ? 4 : 8);   // k = 4, 8 already sit in one lane; k >= 512 fills a warp anyway
 };
 static bool latency_bound(long transforms, int k) {
     const long warps_at_16 = transforms * (k < 16 ? 1 : k / 16) / 32;
@@ -375,7 +398,8 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
             auto launch = [&](auto tin, auto mode) {
                 using TIN = decltype(tin);
                 constexpr int XMODE = decltype(mode)::value;
-                launch_kernel(false, input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream,
+                allow_smem(input_fft_kernel<K, EMAX, TIN, XMODE>, Tile<K, EMAX>::SMEM);
+                launch_kernel(false, input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
                               static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total);
             };
             const bool bf = L->x_dtype == CIRC_BF16;
@@ -411,7 +435,8 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
             auto launch = [&](auto tout, auto vec) {
                 using TOUT = decltype(tout);
                 constexpr bool VEC = decltype(vec)::value;
-                launch_kernel(false, output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream, yop,
+                allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
+                launch_kernel(false, output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
                               static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total);
             };
             const bool vec = (p % 4) == 0;
@@ -453,7 +478,8 @@ int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, co
             auto launch = [&](auto mode, auto vec) {
                 constexpr int XMODE = decltype(mode)::value;
                 constexpr bool VEC = decltype(vec)::value;
-                launch_kernel(false, relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), 0, stream, yop, xop_next,
+                allow_smem(relay_kernel<K, EMAX, XMODE, VEC>, Tile<K, EMAX>::SMEM);
+                launch_kernel(false, relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop, xop_next,
                               static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bo, ext.Bho, total);
             };
             if (xmode == 1) launch(std::integral_constant<int, 1>{}, std::true_type{});
