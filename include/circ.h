@@ -60,11 +60,20 @@ enum {
 
 /*
  * circ_fc_create -- build a fully-connected block-circulant layer (Sec. 3.1).
- *   m, n : output / input widths; k : block size, a power of two in [4, 1024]
- *          that divides both (the paper defines p = m / k, q = n / k and has no
- *          remainder rule; pad on the caller's side).  Blocks above 256 are built
- *          from the same small transform with more butterfly levels (the recursive
- *          construction of Sec. 4.1); they run on the three-launch paths only.
+ *   m, n : output / input widths; k : block size; it must divide both (the paper
+ *          defines p = m / k, q = n / k and has no remainder rule; pad on the
+ *          caller's side).
+ *          Powers of two in [4, 1024] run on a transform of exactly k points.
+ *          Blocks above 256 are built from the same small transform with more
+ *          butterfly levels (the recursive construction of Sec. 4.1); they run
+ *          on the three-launch paths only.
+ *          Any other k in [1, 512] (k = 1 is an ordinary dense layer) is embedded:
+ *          the circular convolution of length k is the linear convolution of the
+ *          zero-padded vectors folded back, a[t] = c[t] + c[t + k], computed on
+ *          the next power-of-two transform with at least 2k - 1 points (zero
+ *          padding in the input-transform kernel, the fold in the inverse one).
+ *          Same results, about (transform size / k) times the work; three-launch
+ *          paths only; the weight-gradient calls refuse such layers.
  *   w    : float32 defining vectors, layout [p][q][k]: w[(i*q + j)*k + t] is
  *          element t of w_ij.  HOST or DEVICE pointer (detected); read during
  *          the call, the caller keeps ownership.

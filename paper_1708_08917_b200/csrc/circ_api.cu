@@ -117,8 +117,15 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
         set_error(CIRC_ERR_ARG, "w is NULL");
         return nullptr;
     }
-    if (!pow2_in_range(k)) {
-        set_error(CIRC_ERR_SHAPE, "block size k=%d must be a power of two in [4, 1024]", k);
+    // transform size: k itself for powers of two in [4, 1024]; otherwise the smallest power of two that holds the
+    // linear convolution of two length-k vectors (2k - 1 points), which the inverse-transform kernel folds back
+    int kt = k;
+    if (k >= 1 && !pow2_in_range(k)) {
+        kt = 4;
+        while (kt < 2 * k - 1 && kt <= 1024) kt <<= 1;
+    }
+    if (k < 1 || kt > 1024) {
+        set_error(CIRC_ERR_SHAPE, "block size k=%d is not supported: powers of two up to 1024, any other size up to 512", k);
         return nullptr;
     }
     if (m <= 0 || n <= 0 || m % k || n % k) {
@@ -134,7 +141,7 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
     L->kind = kind;
     L->m = m;
     L->n = n;
-    L->geo = Geometry{m / k, n / k, k, taps, r, pad};
+    L->geo = Geometry{m / k, n / k, kt, taps, r, pad, k};
     L->x_dtype = L->y_dtype = (kind == 1 ? CIRC_BF16 : CIRC_F32);
     L->variant = CIRC_VARIANT_AUTO;
     for (int st = 0; st < 4; ++st) L->repeat[st] = 1;
@@ -143,13 +150,13 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
         delete L;
         return nullptr;
     }
-    const size_t wcount = (size_t)taps * (m / k) * (n / k) * k;
-    if (to_device(w, wcount, &L->w_dev) != CIRC_OK) {
+    const size_t wcount = (size_t)taps * (m / k) * (n / k) * kt;   // spectra are stored at the transform size
+    if (to_device(w, (size_t)taps * (m / k) * (n / k) * k, &L->w_dev) != CIRC_OK) {
         free_layer(L);
         return nullptr;
     }
     const size_t a_real = (size_t)taps * (m / k) * (n / k);
-    L->a_elems = 2 * a_real + (size_t)(k / 2 - 1) * 4 * a_real;
+    L->a_elems = 2 * a_real + (size_t)(kt / 2 - 1) * 4 * a_real;
     bool ok = cudaMalloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
               cudaMalloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
               cudaMalloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&

@@ -28,7 +28,7 @@ __global__ void transpose_reverse_kernel(const float* __restrict__ w, float* __r
         const int t = (int)(idx % k);
         const long blk = idx / k;  // j * p + i
         const int i = (int)(blk % p), j = (int)(blk / p);
-        wt[idx] = w[((size_t)i * q + j) * k + ((k - t) & (k - 1))];
+        wt[idx] = w[((size_t)i * q + j) * k + (t ? k - t : 0)];
     }
 }
 
@@ -44,7 +44,7 @@ __global__ void transpose_reverse_conv_kernel(const float* __restrict__ w, float
         rest /= q;
         const int tj = (int)(rest % r), ti = (int)(rest / r);     // destination tap
         const int si = r - 1 - ti, sj = r - 1 - tj;               // source tap
-        wt[idx] = w[((((size_t)si * r + sj) * p + i) * q + j) * k + ((k - t) & (k - 1))];
+        wt[idx] = w[((((size_t)si * r + sj) * p + i) * q + j) * k + (t ? k - t : 0)];
     }
 }
 
@@ -488,8 +488,8 @@ static int conv_grad_w_wave() {
 
 static int build_transposed(Layer* L) {
     if (L->transposed) return CIRC_OK;
-    const int p = L->geo.p, q = L->geo.q, k = L->geo.k, r = L->geo.r, taps = L->geo.taps;
-    float* wt = nullptr;
+    const int p = L->geo.p, q = L->geo.q, k = L->geo.ku, r = L->geo.r, taps = L->geo.taps;   // the caller's block size: W^T is
+    float* wt = nullptr;                                                                       // built from the defining vectors
     const size_t count = (size_t)taps * p * q * k;
     if (cudaMalloc(&wt, count * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
@@ -548,6 +548,10 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
     }
     if (L->x_dtype != CIRC_F32 || L->y_dtype != CIRC_F32) {
         set_error(CIRC_ERR_UNSUPPORTED, "the backward pass takes float32 tensors only");
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    if (grad_w && embedded(L->geo)) {
+        set_error(CIRC_ERR_UNSUPPORTED, "the weight gradient is implemented for power-of-two block sizes only (k=%d)", L->geo.ku);
         return CIRC_ERR_UNSUPPORTED;
     }
     int rc = build_transposed(L);  // first call: allocates and synchronises
@@ -665,6 +669,10 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
     }
     if (r > 7) {
         set_error(CIRC_ERR_UNSUPPORTED, "weight gradients are built for filters up to 7 x 7 (r=%d)", r);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    if (embedded(L->geo)) {
+        set_error(CIRC_ERR_UNSUPPORTED, "the weight gradient is implemented for power-of-two block sizes only (k=%d)", L->geo.ku);
         return CIRC_ERR_UNSUPPORTED;
     }
     int rc = build_transposed(L);  // first call: allocates and synchronises

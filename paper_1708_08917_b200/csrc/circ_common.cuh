@@ -35,10 +35,16 @@ namespace circ {
 // ---------------------------------------------------------------------------------------------
 
 struct Geometry {
-    int p, q, k;      // block grid and block size
+    int p, q, k;      // block grid and transform size (a power of two)
     int taps;         // 1 for FC, r*r for CONV
     int r, pad;       // CONV filter size and zero padding (r = 1, pad = 0 for FC)
+    int ku;           // the caller's block size.  ku == k for powers of two in [4, 1024].  Any other block size is
+                      // embedded: a circular convolution of length ku is the linear convolution of the zero-padded
+                      // vectors folded back, y[t] = c[t] + c[t + ku], and the linear convolution is a circular one of
+                      // any length k >= 2 ku - 1.  S0 and S1 zero-pad w_ij and x_j to k, S3 folds; everything in
+                      // between works on k-point spectra and does not know.
 };
+__host__ __device__ inline bool embedded(const Geometry& g) { return g.ku != g.k; }
 
 __host__ __device__ inline int problem_of_bin(int g, int k) { return g == 0 ? 0 : (g == k / 2 ? 1 : g + 1); }
 __host__ __device__ inline int num_problems(int k) { return k / 2 + 1; }

@@ -281,7 +281,7 @@ static void plan(const Layer* L, int pairs, int* rows, int* jsplit) {
 }
 
 bool fused_fc_supported(const Layer* L, int batch) {
-    if (L->kind != 0 || batch < 1 || batch > 8 || L->geo.k > 256) return false;   // larger blocks: the staged path
+    if (L->kind != 0 || batch < 1 || batch > 8 || L->geo.k > 256 || embedded(L->geo)) return false;   // larger or embedded blocks: the staged path
     const int pairs = pairs_for(batch);
     int rows, js;
     plan(L, pairs, &rows, &js);

@@ -55,5 +55,10 @@ __device__ __forceinline__ void store_run(__nv_bfloat16* dst, const float (&v)[E
     }
 }
 
+// Single elements (the unaligned paths of embedded block sizes).
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ void store_one(float* dst, float v) { *dst = v; }
+__device__ __forceinline__ void store_one(__nv_bfloat16* dst, float v) { *dst = __float2bfloat16_rn(v); }
 
 }  // namespace circ

@@ -77,8 +77,8 @@ int circ_fc_forward_noalloc(circ_handle h, const void* x, void* y, int batch, vo
     e.W = e.Wo = batch;
     e.Nh = e.Bh;
     // operand X: 2*Bh columns x n floats; operand Y: 2*Bh columns x m floats (all frequencies together)
-    const size_t x_floats = ((size_t)2 * e.Bh * L->n + 63) & ~(size_t)63;
-    const size_t y_floats = (size_t)2 * e.Bh * L->m;
+    const size_t x_floats = ((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63;
+    const size_t y_floats = (size_t)2 * e.Bh * L->geo.p * L->geo.k;
     const size_t need = (x_floats + y_floats) * sizeof(float);
     if (need > kNoAllocScratchBytes) {
         set_error(CIRC_ERR_SHAPE,

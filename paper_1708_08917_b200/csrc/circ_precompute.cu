@@ -24,18 +24,22 @@ __global__ void precompute_spectra_kernel(const float* __restrict__ w, float* __
         const int j = (int)(blk % q);
         const int i = (int)((blk / q) % p);
         const int tap = (int)(blk / ((long)p * q));
-        const float* wv = w + blk * k;
+        const float* wv = w + blk * geo.ku;     // defining vectors are stored at the caller's block size
         double re = 0.0, im = 0.0;
-        for (int t = 0; t < k; ++t) {
+        // Convention 1 is W[r][c] = w[(c - r) mod ku] = w'[(r - c) mod ku] with w' the index-reversed vector.  At
+        // ku == k the reversal is the conjugate spectrum; an embedded block must be reversed before it is padded.
+        const bool reverse = convention == 1 && geo.ku != k;
+        for (int t = 0; t < geo.ku; ++t) {      // (zero padding up to k adds nothing)
             const int ph = (g * t) & (k - 1);  // exact reduction of g t / k
             double s, c;
             sincospi(-2.0 * (double)ph / (double)k, &s, &c);
-            re += (double)wv[t] * c;
-            im += (double)wv[t] * s;
+            const double wt = (double)wv[reverse && t ? geo.ku - t : t];
+            re += wt * c;
+            im += wt * s;
         }
         re /= (double)k;
         im /= (double)k;
-        if (convention == 1) im = -im;
+        if (convention == 1 && !reverse) im = -im;
         if (g == 0 || g == k / 2) im = 0.0;
         const float fre = (float)re, fim = (float)im;
 

@@ -155,7 +155,7 @@ int circ_stack_forward(circ_stack_handle s, const void* x, void* y, int batch, v
     for (int l = 0; l + 1 < D; ++l) {
         const Layer* A = S->layers[l];
         const Layer* Bn = S->layers[l + 1];
-        relay[l] = staged(variant[l]) && staged(variant[l + 1]) && A->geo.k == Bn->geo.k && A->y_dtype == CIRC_F32 &&
+        relay[l] = staged(variant[l]) && staged(variant[l + 1]) && A->geo.k == Bn->geo.k && !embedded(A->geo) && !embedded(Bn->geo) && A->y_dtype == CIRC_F32 &&
                    Bn->x_dtype == CIRC_F32;
         if (!relay[l]) {
             const size_t bytes = (size_t)batch * A->m * (A->y_dtype == CIRC_BF16 ? 2 : 4);

@@ -199,7 +199,7 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
 template <int K, int EMAX, typename TIN, int XMODE>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
-                 int B, int Bh, long total) {
+                 int B, int Bh, long total, int ku) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
@@ -217,8 +217,23 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
         for (int r = 0; r < E; ++r) re[r] = im[r] = 0.f;
         if (T < total) {
             const int c = (int)(T / q), j = (int)(T % q);
-            load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
-            if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
+            if (ku == K) {
+                load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
+                if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
+            } else {
+                // embedded block size: the block has ku samples (any alignment), the rest of the transform is zero
+                const TIN* x0 = x + (size_t)c * n + (size_t)j * ku;
+                const TIN* x1 = x + (size_t)(c + Bh) * n + (size_t)j * ku;
+                const bool second = c + Bh < B;
+#pragma unroll
+                for (int r = 0; r < E; ++r) {
+                    const int t = E * l + r;
+                    if (t < ku) {
+                        re[r] = to_float(x0[t]);
+                        if (second) im[r] = to_float(x1[t]);
+                    }
+                }
+            }
         }
 #pragma unroll
         for (int r = 0; r < E; ++r) v[r] = make_float2(re[r], im[r]);
@@ -239,7 +254,7 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
 template <int K, int EMAX, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
-                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total) {
+                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
@@ -254,7 +269,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         const long Tb = (long)blockIdx.x * TT + threadIdx.x / L;
 #pragma unroll
         for (int r = 0; r < E; ++r) bv[r] = 0.f;
-        if (bias && Tb < total) load_run<E>(bias + (int)(Tb % p) * K + E * (threadIdx.x % L), bv);
+        if (bias && Tb < total && ku == K) load_run<E>(bias + (int)(Tb % p) * K + E * (threadIdx.x % L), bv);
     }
 
     gather_operand<K, EMAX, VEC>(zs, yop, p, Bho, total);
@@ -268,6 +283,38 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[f2 + L * f1][gi] : make_float2(0.f, 0.f);
     fft_inverse<K, EMAX>(v, l, tw);
+    if (ku != K) {
+        // embedded block size: v is the linear convolution (2 ku - 1 points) of the zero-padded blocks; the
+        // circular one folds it, a[t] = c[t] + c[t + ku].  The fold crosses lanes, so it goes through the tile.
+        __syncthreads();   // every thread has taken its bins out of the tile
+#pragma unroll
+        for (int r = 0; r < E; ++r) zs[E * l + r][gi] = v[r];
+        __syncthreads();
+        if (!live) return;
+        const int c = (int)(T / p), i = (int)(T % p);
+        const bool second = c + Bho < Bo;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int t = E * l + r;
+            if (t >= ku) continue;
+            float2 a = zs[t][gi];
+            if (t + ku < K) {
+                const float2 b2 = zs[t + ku][gi];
+                a.x += b2.x;
+                a.y += b2.y;
+            }
+            const float bb = bias ? __ldg(bias + i * ku + t) : 0.f;
+            a.x += bb;
+            a.y += bb;
+            if (relu) {
+                a.x = fmaxf(a.x, 0.f);
+                a.y = fmaxf(a.y, 0.f);
+            }
+            store_one(y + (size_t)c * m + (size_t)i * ku + t, a.x);
+            if (second) store_one(y + (size_t)(c + Bho) * m + (size_t)i * ku + t, a.y);
+        }
+        return;
+    }
     if (!live) return;
     const int c = (int)(T / p), i = (int)(T % p);
     const int col = i * K + E * l;
@@ -400,7 +447,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
                 constexpr int XMODE = decltype(mode)::value;
                 allow_smem(input_fft_kernel<K, EMAX, TIN, XMODE>, Tile<K, EMAX>::SMEM);
                 launch_kernel(false, input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
-                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total);
+                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku);
             };
             const bool bf = L->x_dtype == CIRC_BF16;
             if (xmode == 0) {
@@ -437,7 +484,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
                 launch_kernel(false, output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
-                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total);
+                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku);
             };
             const bool vec = (p % 4) == 0;
             if (L->y_dtype == CIRC_BF16) {
