@@ -243,6 +243,12 @@ static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStr
     if (rc != CIRC_OK) return rc;
     float* xop = static_cast<float*>(L->ws);
     float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
+    // small forwards (none of the three kernels fills the machine) overlap each kernel's launch and set-up with
+    // its predecessor; reset on every exit path by the guard
+    struct DependentGuard {
+        DependentGuard(bool on) { dependent_launches() = on; }
+        ~DependentGuard() { dependent_launches() = false; }
+    } guard(!L->prof && (long)e.Bh * (L->geo.p > L->geo.q ? L->geo.p : L->geo.q) * L->geo.k <= 32768);
     {
         StageTimer t(L, 0, stream);
         // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16

@@ -123,17 +123,26 @@ void count_launches(long n);
 // Programmatic dependent launch.  A kernel launched with the "programmatic stream serialization"
 // attribute may be scheduled while its predecessor in the stream still runs, so that its launch
 // latency and set-up overlap the predecessor's work.  The contract every forward kernel keeps:
+//   pdl_trigger()  first thing: lets the next kernel's thread blocks be scheduled as soon as every block of
+//                  this kernel has started, so that its launch latency and set-up (twiddle tables, barriers,
+//                  tensor memory) overlap this kernel's work;
 //   pdl_wait()     before the first access to global memory: blocks until all earlier kernels have
-//                  finished and their writes are visible;
-//   pdl_trigger()  right after that wait: lets the next kernel be scheduled.  Triggering only after
-//                  the wait keeps at most one kernel queued behind the running one.
-// Both are no-ops when the kernel was launched without the attribute.  Measured on B200: the
-// attribute shortens back-to-back one-kernel forwards (the fused path) by about 5 %, but moves the
-// three-kernel path by -7 % .. +35 % depending on the shape, so only the fused kernel asks for it
-// (`dependent` = true below).
+//                  finished and their writes are visible.
+// Both are no-ops when the kernel was launched without the attribute.  Waiting blocks hold registers and
+// shared memory, so the attribute only pays when the kernels involved do not fill the machine.  Measured on
+// B200 for the three-kernel path: 10 - 14 % faster at 32 Ki transform points per forward (4096 x 4096, k = 64,
+// batch 16: 9.3 -> 8.3 us; 1024 x 1024, k = 16, batch 64: 8.4 -> 7.2 us), 4 - 40 % slower from 128 Ki points up.
+// The forward pass therefore asks for it (`dependent_launches()`) below 32 Ki points only; the one-launch
+// fused kernel always does.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Whether the staged kernels launched by this thread ask for programmatic dependent launch (set by the forward pass).
+inline bool& dependent_launches() {
+    static thread_local bool on = false;
+    return on;
+}
 
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {

@@ -24,8 +24,8 @@ struct ContractArgs {
 
 template <bool CONV>
 __global__ void __launch_bounds__(256) contract_fma_kernel(ContractArgs g) {
-    pdl_wait();     // X is written by the transform kernel before this one
     pdl_trigger();
+    pdl_wait();     // X is written by the transform kernel before this one
     const int prob = blockIdx.z;
     const bool real = problem_is_real(prob);
     const int M = real ? g.p : 2 * g.p;
@@ -135,9 +135,9 @@ int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Exte
     g.H = ext.H; g.W = ext.W; g.Ho = ext.Ho; g.Wo = ext.Wo;
     dim3 grid((g.cols_out + BN - 1) / BN, (2 * g.p + BM - 1) / BM, num_problems(g.k));
     if (L->kind == 1)
-        launch_kernel(false, contract_fma_kernel<true>, grid, dim3(256), 0, stream, g);
+        launch_kernel(dependent_launches(), contract_fma_kernel<true>, grid, dim3(256), 0, stream, g);
     else
-        launch_kernel(false, contract_fma_kernel<false>, grid, dim3(256), 0, stream, g);
+        launch_kernel(dependent_launches(), contract_fma_kernel<false>, grid, dim3(256), 0, stream, g);
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
     return CIRC_OK;

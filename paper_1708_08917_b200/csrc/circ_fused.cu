@@ -80,8 +80,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) fused_fc_kernel(FusedArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int q = a.q;
     load_twiddles<K>(tw);
-    pdl_wait();     // x may come from the kernel before
     pdl_trigger();
+    pdl_wait();     // x may come from the kernel before
     __syncthreads();
 
     // ---- phase A: Z_j for all column blocks ----------------------------------------------------

@@ -205,8 +205,8 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
     pdl_trigger();
+    pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
@@ -260,8 +260,8 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_wait();     // Y is written by the contraction kernel before this one
     pdl_trigger();
+    pdl_wait();     // Y is written by the contraction kernel before this one
 
     // the bias of this thread's outputs is fetched now, long before the epilogue needs it
     float bv[E];
@@ -346,8 +346,8 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_wait();
     pdl_trigger();
+    pdl_wait();
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
     const bool live = T < total;
@@ -446,7 +446,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
                 using TIN = decltype(tin);
                 constexpr int XMODE = decltype(mode)::value;
                 allow_smem(input_fft_kernel<K, EMAX, TIN, XMODE>, Tile<K, EMAX>::SMEM);
-                launch_kernel(false, input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
+                launch_kernel(dependent_launches(), input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
                               static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku);
             };
             const bool bf = L->x_dtype == CIRC_BF16;
@@ -483,7 +483,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
                 using TOUT = decltype(tout);
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
-                launch_kernel(false, output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
+                launch_kernel(dependent_launches(), output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
                               static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku);
             };
             const bool vec = (p % 4) == 0;
@@ -526,7 +526,7 @@ int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, co
                 constexpr int XMODE = decltype(mode)::value;
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(relay_kernel<K, EMAX, XMODE, VEC>, Tile<K, EMAX>::SMEM);
-                launch_kernel(false, relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop, xop_next,
+                launch_kernel(dependent_launches(), relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop, xop_next,
                               static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bo, ext.Bho, total);
             };
             if (xmode == 1) launch(std::integral_constant<int, 1>{}, std::true_type{});

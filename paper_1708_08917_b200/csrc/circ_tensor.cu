@@ -293,8 +293,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    pdl_wait();     // X is written by the transform kernel before this one; Y may still be read by an earlier one
     pdl_trigger();
+    pdl_wait();     // X is written by the transform kernel before this one; Y may still be read by an earlier one
 
     if (warp == 0) {
         // ---- TMA producer -----------------------------------------------------------------------
@@ -618,7 +618,7 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
     }
     g.tiles = ctas;
     const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
-    launch_kernel(false, contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, maps[0], maps[1], maps[2], maps[3], maps[4],
+    launch_kernel(dependent_launches(), contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, maps[0], maps[1], maps[2], maps[3], maps[4],
                   maps[5], g);
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
