@@ -109,8 +109,8 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // The MMA warp runs its loop with all 32 lanes on warp-uniform values (so that descriptors and
-// addresses live in uniform registers) and only the instructions below are restricted to one
-// elected lane, by a guard predicate rather than a branch.
+// addresses live in uniform registers); one elected lane enters the short branch that issues a
+// K block's MMAs and its commit.
 __device__ __forceinline__ uint32_t elect_one() {
     uint32_t leader;
     asm volatile(
@@ -120,21 +120,15 @@ __device__ __forceinline__ uint32_t elect_one() {
         : "=r"(leader));
     return leader;
 }
-__device__ __forceinline__ void tc_commit(uint64_t* bar, uint32_t leader) {
-    asm volatile(
-        "{\n\t.reg .pred q;\n\t"
-        "setp.ne.b32 q, %1, 0;\n\t"
-        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(smem_u32(bar)), "r"(leader) : "memory");
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate,
-                                            uint32_t leader) {
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p, q;\n\t"
+        "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "setp.ne.b32 q, %5, 0;\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(leader)
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -218,28 +212,28 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 // start-address field (16-byte units): 8 units per tile row, a_step per tap, 2 per K step.
 template <int R, int KSTEPS>
 __device__ __forceinline__ void issue_taps(uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step, uint64_t a_step,
-                                           uint32_t idesc, uint32_t& accumulate, uint32_t leader) {
+                                           uint32_t idesc, uint32_t& accumulate) {
 #pragma unroll
     for (int di = 0; di < R; ++di) {
 #pragma unroll
         for (int dj = 0; dj < R; ++dj) {
             const uint64_t x = dx + (uint64_t)di * row_step + (uint64_t)(dj * 8);
             const uint64_t w = da + (uint64_t)(di * R + dj) * a_step;
-            tc_mma_bf16(d_tmem, x, w, idesc, accumulate, leader);
+            tc_mma_bf16(d_tmem, x, w, idesc, accumulate);
 #pragma unroll
-            for (int k4 = 1; k4 < KSTEPS; ++k4) tc_mma_bf16(d_tmem, x + 2 * k4, w + 2 * k4, idesc, 1u, leader);
+            for (int k4 = 1; k4 < KSTEPS; ++k4) tc_mma_bf16(d_tmem, x + 2 * k4, w + 2 * k4, idesc, 1u);
             accumulate = 1u;
         }
     }
 }
 template <int R>
 __device__ __forceinline__ void issue_taps_k(int ksteps, uint32_t d_tmem, uint64_t dx, uint64_t da, uint64_t row_step,
-                                             uint64_t a_step, uint32_t idesc, uint32_t& accumulate, uint32_t leader) {
+                                             uint64_t a_step, uint32_t idesc, uint32_t& accumulate) {
     switch (ksteps) {
-        case 1: issue_taps<R, 1>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
-        case 2: issue_taps<R, 2>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
-        case 3: issue_taps<R, 3>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
-        default: issue_taps<R, 4>(d_tmem, dx, da, row_step, a_step, idesc, accumulate, leader); break;
+        case 1: issue_taps<R, 1>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        case 2: issue_taps<R, 2>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        case 3: issue_taps<R, 3>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
+        default: issue_taps<R, 4>(d_tmem, dx, da, row_step, a_step, idesc, accumulate); break;
     }
 }
 
@@ -380,19 +374,20 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                         const uint32_t as = xs + (uint32_t)g.nsplit * x_bytes;
                         const uint32_t a_lo = as + (uint32_t)g.taps * a_bytes;   // lo parts of the weight tiles
                         const int krem = t.Kq - kb * kKBlock;                    // valid contraction entries in this block
+                        if (leader) {
                         if (g.taps == 1 && krem >= kKBlock) {
                             // fully-connected fast path: four K steps of 16 per product
                             const uint64_t dxh = smem_desc_sw128(xs), dah = smem_desc_sw128(as);
-                            tc_mma_bf16(d_tmem, dxh, dah, idesc, accumulate, leader);
-                            tc_mma_bf16(d_tmem, dxh + 2, dah + 2, idesc, 1u, leader);
-                            tc_mma_bf16(d_tmem, dxh + 4, dah + 4, idesc, 1u, leader);
-                            tc_mma_bf16(d_tmem, dxh + 6, dah + 6, idesc, 1u, leader);
+                            tc_mma_bf16(d_tmem, dxh, dah, idesc, accumulate);
+                            tc_mma_bf16(d_tmem, dxh + 2, dah + 2, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dxh + 4, dah + 4, idesc, 1u);
+                            tc_mma_bf16(d_tmem, dxh + 6, dah + 6, idesc, 1u);
                             if (g.npass == 3) {
                                 const uint64_t dxl = smem_desc_sw128(xs + x_bytes), dal = smem_desc_sw128(a_lo);
 #pragma unroll
-                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxh + 2 * k4, dal + 2 * k4, idesc, 1u, leader);
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxh + 2 * k4, dal + 2 * k4, idesc, 1u);
 #pragma unroll
-                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxl + 2 * k4, dah + 2 * k4, idesc, 1u, leader);
+                                for (int k4 = 0; k4 < 4; ++k4) tc_mma_bf16(d_tmem, dxl + 2 * k4, dah + 2 * k4, idesc, 1u);
                             }
                             accumulate = 1u;
                         } else {
@@ -407,31 +402,33 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                                 const uint64_t dx = prod == 2 ? dx_lo : dx_hi;
                                 const uint64_t da = prod == 1 ? da_lo : da_hi;
                                 if (g.r == 3) {
-                                    issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate, leader);
+                                    issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
                                 } else if (g.r == 1) {
-                                    issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate, leader);
+                                    issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
                                 } else {
                                     uint64_t dx_row = dx, db = da;
                                     for (int di = 0; di < g.r; ++di, dx_row += row_step) {
                                         uint64_t dxx = dx_row;
                                         for (int dj = 0; dj < g.r; ++dj, dxx += 8, db += tap_step) {
-                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate, leader);
+                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate);
                                             for (int k4 = 1; k4 < ksteps; ++k4)   // 16 bf16 = 32 bytes per MMA step along K
-                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u, leader);
+                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u);
                                             accumulate = 1u;
                                         }
                                     }
                                 }
                             }
                         }
-                        tc_commit(&empty_bar[s], leader);   // stage free once these MMAs have read it
+                        tc_commit(&empty_bar[s]);   // stage free once these MMAs have read it
+                        if (kb + 1 == kblocks) tc_commit(&acc_full[buf]);   // accumulator complete
+                        }
+                        accumulate = 1u;
                         if (++s == g.stages) {
                             s = 0;
                             par ^= 1u;
                         }
                     }
                 }
-                if (ok) tc_commit(&acc_full[buf], leader);  // accumulator complete
                 if (++buf == g.nacc) {
                     buf = 0;
                     acc_par ^= 1u;
