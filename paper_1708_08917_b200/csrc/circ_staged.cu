@@ -28,7 +28,7 @@ struct Tile {
     static constexpr int TT = NT / L;
     static constexpr int PAD = L == 1 ? 0 : (L >= 16 ? 2 : 16 / L);  // even, so that rows stay 16-byte aligned
     static constexpr int ROW = TT + PAD;
-    static constexpr size_t SMEM = sizeof(float2) * ((size_t)K + (size_t)K * ROW);   // twiddle table + staging tile (dynamic shared memory)
+    static constexpr size_t SMEM = sizeof(float2) * ((size_t)K + (size_t)K * ROW) + (size_t)TT * 16;   // twiddle table + staging tile + per-transform output offsets (dynamic shared memory)
 };
 
 __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
@@ -315,21 +315,72 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         }
         return;
     }
-    if (!live) return;
-    const int c = (int)(T / p), i = (int)(T % p);
-    const int col = i * K + E * l;
-    float re[E], im[E];
+    if constexpr (E < 16 || !std::is_same<TOUT, float>::value) {
+        // a lane's outputs are at most 32 bytes: direct stores are already (nearly) whole lines per instruction
+        if (!live) return;
+        const int c = (int)(T / p), i = (int)(T % p);
+        const int col = i * K + E * l;
+        float re[E], im[E];
 #pragma unroll
-    for (int r = 0; r < E; ++r) {
-        re[r] = v[r].x + bv[r];
-        im[r] = v[r].y + bv[r];
-        if (relu) {
-            re[r] = fmaxf(re[r], 0.f);
-            im[r] = fmaxf(im[r], 0.f);
+        for (int r = 0; r < E; ++r) {
+            re[r] = v[r].x + bv[r];
+            im[r] = v[r].y + bv[r];
+            if (relu) {
+                re[r] = fmaxf(re[r], 0.f);
+                im[r] = fmaxf(im[r], 0.f);
+            }
         }
+        store_run<E>(y + (size_t)c * m + col, re);
+        if (c + Bho < Bo) store_run<E>(y + (size_t)(c + Bho) * m + col, im);
+        return;
+    } else {
+    // A lane holds E consecutive outputs (64 bytes at E = 16), so storing them directly makes every store
+    // instruction write 16-byte pieces 64 bytes apart.  The outputs are instead handed over through the tile
+    // (free once every thread has taken its bins) in 16-byte pieces, and stored with consecutive lanes on
+    // consecutive pieces: whole lines per instruction.  A lane's pieces are permuted (slot = r xor f(thread)) so
+    // that both the writes and the reads of the hand-over are free of bank conflicts.
+    constexpr int PPL = E / 4;                                  // pieces per lane and sample
+    constexpr int NT = Tile<K, EMAX>::NT;
+    float4* ot = reinterpret_cast<float4*>(&zs[0][0]);          // [sample][thread][PPL] pieces; K * ROW * 8 >= 2 * NT * E * 4 bytes
+    long long* offs = reinterpret_cast<long long*>(&zs[0][0] + (size_t)K * ROW);   // [TT] first output element, or -1
+    int* both = reinterpret_cast<int*>(offs + TT);             // [TT] does the pair's second sample exist
+    auto slot = [](int t, int r) { return PPL == 4 ? (r ^ ((t >> 1) & 3)) : PPL == 8 ? (r ^ (t & 7)) : r; };
+    __syncthreads();   // every thread has taken its bins out of the tile
+#pragma unroll
+    for (int r = 0; r < PPL; ++r) {
+        float o[2][4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            o[0][e] = v[4 * r + e].x + bv[4 * r + e];
+            o[1][e] = v[4 * r + e].y + bv[4 * r + e];
+            if (relu) {
+                o[0][e] = fmaxf(o[0][e], 0.f);
+                o[1][e] = fmaxf(o[1][e], 0.f);
+            }
+        }
+        const int sl = slot((int)threadIdx.x, r);
+        ot[(size_t)threadIdx.x * PPL + sl] = make_float4(o[0][0], o[0][1], o[0][2], o[0][3]);
+        ot[(size_t)(NT + threadIdx.x) * PPL + sl] = make_float4(o[1][0], o[1][1], o[1][2], o[1][3]);
     }
-    store_run<E>(y + (size_t)c * m + col, re);
-    if (c + Bho < Bo) store_run<E>(y + (size_t)(c + Bho) * m + col, im);
+    if (l == 0) {
+        const int c = (int)(T / p), i = (int)(T % p);
+        offs[gi] = live ? (long long)c * m + (long long)i * K : -1;
+        both[gi] = live && c + Bho < Bo;
+    }
+    __syncthreads();
+    constexpr int PPT = K / 4;                                  // pieces per transform
+#pragma unroll
+    for (int it = 0; it < 2 * PPL; ++it) {
+        const int w = it * NT + (int)threadIdx.x;               // (sample, transform, piece), piece fastest
+        const int pi = w % PPT, g2 = (w / PPT) % TT, smp = w / (PPT * TT);
+        const long long off = offs[g2];
+        if (off < 0 || (smp == 1 && !both[g2])) continue;
+        const int t = g2 * L + pi / PPL;                        // the thread that produced the piece
+        const float4 o = ot[(size_t)(smp * NT + t) * PPL + slot(t, pi % PPL)];
+        const float r4[4] = {o.x, o.y, o.z, o.w};
+        store_run<4>(y + (size_t)off + (smp ? (size_t)Bho * m : 0) + 4 * pi, r4);
+    }
+    }
 }
 
 // ---- relay: operand Y of one layer -> operand X of the next -----------------------------------------
