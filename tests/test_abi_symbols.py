@@ -43,8 +43,10 @@ def test_argument_errors_need_no_gpu(lib):
     lib.circ_fc_create.restype = ctypes.c_void_p
     lib.circ_last_error.restype = ctypes.c_char_p
     buf = (ctypes.c_float * 64)()
-    assert lib.circ_fc_create(8, 8, 3, buf) is None and lib.circ_last_code() == -2       # k not a power of two
+    assert lib.circ_fc_create(8, 8, 3, buf) is None and lib.circ_last_code() == -2       # k does not divide m
     assert lib.circ_fc_create(8, 8, 2048, buf) is None and lib.circ_last_code() == -2     # k out of range
+    assert lib.circ_fc_create(513, 513, 513, buf) is None and lib.circ_last_code() == -2  # 2k - 1 points exceed the largest transform
+    assert lib.circ_fc_create(8, 8, 0, buf) is None and lib.circ_last_code() == -2        # k < 1
     assert lib.circ_fc_create(10, 8, 4, buf) is None and lib.circ_last_code() == -2      # k does not divide m
     assert lib.circ_fc_create(8, 8, 4, None) is None and lib.circ_last_code() == -1      # NULL weights
     assert b"k=" in lib.circ_last_error() or b"NULL" in lib.circ_last_error()
