@@ -73,7 +73,8 @@ enum {
  *          the next power-of-two transform with at least 2k - 1 points (zero
  *          padding in the input-transform kernel, the fold in the inverse one).
  *          Same results, about (transform size / k) times the work; three-launch
- *          paths only; the weight-gradient calls refuse such layers.
+ *          paths only.  The backward calls serve such layers too (the weight
+ *          gradient is a circular correlation: it folds as g[t] = c[t] + c[t - k]).
  *   w    : float32 defining vectors, layout [p][q][k]: w[(i*q + j)*k + t] is
  *          element t of w_ij.  HOST or DEVICE pointer (detected); read during
  *          the call, the caller keeps ownership.

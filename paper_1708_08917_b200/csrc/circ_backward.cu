@@ -550,10 +550,6 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
         set_error(CIRC_ERR_UNSUPPORTED, "the backward pass takes float32 tensors only");
         return CIRC_ERR_UNSUPPORTED;
     }
-    if (grad_w && embedded(L->geo)) {
-        set_error(CIRC_ERR_UNSUPPORTED, "the weight gradient is implemented for power-of-two block sizes only (k=%d)", L->geo.ku);
-        return CIRC_ERR_UNSUPPORTED;
-    }
     int rc = build_transposed(L);  // first call: allocates and synchronises
     if (rc != CIRC_OK) return rc;
     Layer* T = L->transposed;
@@ -573,12 +569,13 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
         const int Ph = (p + 1) / 2;
         const int cols = 2 * e.Bh, cols_padded = (cols + 7) & ~7;
         const bool tensor = batch >= 32 && tensor_batch_product_supported(cols);
-        const size_t x_floats = ((size_t)cols * L->n + 63) & ~(size_t)63;
-        const size_t g_floats = ((size_t)cols * L->m + 63) & ~(size_t)63;
-        const size_t y_floats = ((size_t)2 * Ph * L->n + 63) & ~(size_t)63;
+        const size_t nk = (size_t)q * k, mk = (size_t)p * k;   // widths at the transform size (= n, m unless embedded)
+        const size_t x_floats = ((size_t)cols * nk + 63) & ~(size_t)63;
+        const size_t g_floats = ((size_t)cols * mk + 63) & ~(size_t)63;
+        const size_t y_floats = ((size_t)2 * Ph * nk + 63) & ~(size_t)63;
         // tensor route only: transposed split operands (bfloat16) and the raw products (float32)
-        const size_t xt_halves = tensor ? (((size_t)L->n * 2 * cols_padded + 127) & ~(size_t)127) : 0;
-        const size_t gt_halves = tensor ? (((size_t)L->m * 2 * cols_padded + 127) & ~(size_t)127) : 0;
+        const size_t xt_halves = tensor ? ((nk * 2 * cols_padded + 127) & ~(size_t)127) : 0;
+        const size_t gt_halves = tensor ? ((mk * 2 * cols_padded + 127) & ~(size_t)127) : 0;
         const size_t pt_floats = tensor ? (size_t)2 * p * q + (size_t)(k / 2 - 1) * 4 * p * q : 0;
         const size_t need = (x_floats + g_floats + y_floats + pt_floats) * sizeof(float) + (xt_halves + gt_halves) * 2 + 1024;
         if ((rc = ensure_workspace(L, need)) != CIRC_OK) return rc;
@@ -626,7 +623,7 @@ int circ_fc_backward(circ_handle h, const void* x, const void* grad_a, void* gra
         ew.H = ew.Ho = 1;
         ew.W = ew.Wo = p;
         ew.Nh = Ph;
-        if ((rc = launch_output_ifft(T, yop, grad_w, ew, s)) != CIRC_OK) return rc;
+        if ((rc = launch_output_ifft(T, yop, grad_w, ew, s, true)) != CIRC_OK) return rc;
     }
     return CIRC_OK;
 }
@@ -671,10 +668,6 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
         set_error(CIRC_ERR_UNSUPPORTED, "weight gradients are built for filters up to 7 x 7 (r=%d)", r);
         return CIRC_ERR_UNSUPPORTED;
     }
-    if (embedded(L->geo)) {
-        set_error(CIRC_ERR_UNSUPPORTED, "the weight gradient is implemented for power-of-two block sizes only (k=%d)", L->geo.ku);
-        return CIRC_ERR_UNSUPPORTED;
-    }
     int rc = build_transposed(L);  // first call: allocates and synchronises
     if (rc != CIRC_OK) return rc;
     Layer* T = L->transposed;
@@ -690,9 +683,10 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
     eg.B = eg.Bo = N * Ho * Wo;
     eg.Bh = eg.Bho = eg.Nh * Ho * Wo;
     const int NhT = (taps + 1) / 2, St = NhT * p;
-    const size_t x_floats = ((size_t)2 * ex.Bh * L->n + 63) & ~(size_t)63;
-    const size_t g_floats = ((size_t)2 * eg.Bh * L->m + 63) & ~(size_t)63;
-    const size_t y_floats = ((size_t)2 * St * L->n + 63) & ~(size_t)63;
+    const size_t nk = (size_t)q * k, mk = (size_t)p * k;   // channel counts at the transform size (= c_in, c_out unless embedded)
+    const size_t x_floats = ((size_t)2 * ex.Bh * nk + 63) & ~(size_t)63;
+    const size_t g_floats = ((size_t)2 * eg.Bh * mk + 63) & ~(size_t)63;
+    const size_t y_floats = ((size_t)2 * St * nk + 63) & ~(size_t)63;
     const int tiles = ((p + 15) / 16) * ((q + 15) / 16), nprob = num_problems(k);
     const int rows = 2 * ex.Nh * Ho;
     // split the pixel sum so that the grid is one full wave of CTAs (a few CTAs more would cost a second wave)
@@ -756,7 +750,7 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
     ew.Nh = St;
     const int keep = T->y_dtype;
     T->y_dtype = CIRC_F32;
-    rc = launch_output_ifft(T, yop, grad_w, ew, s);
+    rc = launch_output_ifft(T, yop, grad_w, ew, s, true);
     T->y_dtype = keep;
     return rc;
 }

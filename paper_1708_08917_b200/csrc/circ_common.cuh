@@ -188,7 +188,10 @@ int launch_tc_batch_product(const __nv_bfloat16* xt, int q, const __nv_bfloat16*
 bool tensor_batch_product_supported(int cols);
 
 // S3 / C3: inverse transforms + bias + activation -> y.
-int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);
+// `correlation`: how an embedded block size folds.  false: a[t] = c[t] + c[t + ku] (the forward pass, a circular
+// convolution); true: a[t] = c[t] + c[t - ku] (the weight gradient, a circular correlation whose negative lags sit at
+// the top of the transform).  Ignored when the block size is the transform size.
+int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation = false);
 
 // S3 of layer L and S1 of the next layer (same k, its q = L's p) in one launch: Y operand -> X operand (xmode 0 or 1).
 int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, const Extent& ext, cudaStream_t stream);

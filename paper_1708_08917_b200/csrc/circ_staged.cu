@@ -254,7 +254,7 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
 template <int K, int EMAX, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
-                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku) {
+                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku, int corr) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
@@ -285,7 +285,9 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     fft_inverse<K, EMAX>(v, l, tw);
     if (ku != K) {
         // embedded block size: v is the linear convolution (2 ku - 1 points) of the zero-padded blocks; the
-        // circular one folds it, a[t] = c[t] + c[t + ku].  The fold crosses lanes, so it goes through the tile.
+        // circular one folds it, a[t] = c[t] + c[t + ku].  (corr: v is a linear correlation with lags -ku < s < ku,
+        // the negative ones at K + s, and the fold is a[t] = c[t] + c[t - ku].)  The fold crosses lanes, so it goes
+        // through the tile.
         __syncthreads();   // every thread has taken its bins out of the tile
 #pragma unroll
         for (int r = 0; r < E; ++r) zs[E * l + r][gi] = v[r];
@@ -298,8 +300,9 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
             const int t = E * l + r;
             if (t >= ku) continue;
             float2 a = zs[t][gi];
-            if (t + ku < K) {
-                const float2 b2 = zs[t + ku][gi];
+            const int hi = corr ? K - ku + t : t + ku;
+            if (corr ? t > 0 : hi < K) {
+                const float2 b2 = zs[hi][gi];
                 a.x += b2.x;
                 a.y += b2.y;
             }
@@ -520,7 +523,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
     return CIRC_OK;
 }
 
-int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream) {
+int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation) {
     const int p = L->geo.p, m = L->m;
     const long total = (long)ext.Bho * p;
     const bool small = latency_bound(total, L->geo.k);
@@ -535,7 +538,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
                 launch_kernel(dependent_launches(), output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
-                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku);
+                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku, (int)correlation);
             };
             const bool vec = (p % 4) == 0;
             if (L->y_dtype == CIRC_BF16) {

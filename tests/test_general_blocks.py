@@ -51,25 +51,68 @@ def test_conv_any_block_size(k, c_in, c_out):
     assert scale_rel_err(got, oracle_conv(case)) <= TOL_BF16
 
 
-@pytest.mark.parametrize("k", [6, 100])
-def test_input_gradient_any_block_size(k):
-    p, q, batch = 3, 8, 12
-    case = synth.fc_case(f"gen_bwd_{k}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal")
+@pytest.mark.parametrize("k,batch", [(6, 12), (100, 12), (12, 40), (3, 33)])
+@pytest.mark.parametrize("convention", [0, 1])
+def test_gradients_any_block_size(k, batch, convention):
+    # batch >= 32 takes the tensor-core batch product, smaller ones the fp32 FMA one
+    p, q = 3, 8
+    case = synth.fc_case(f"gen_bwd_{k}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal")
     g = synth.normal((batch, p * k), 1.0, synth.stream_id(case.name, "g"))
     h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
     try:
+        circ.circ_set_convention(h, convention)
         gd = torch.from_numpy(g).cuda()
         gx = torch.full((batch, case.n), float("nan"), device="cuda")
-        circ.circ_fc_backward(h, None, gd, gx, None, batch)
+        gw = torch.full((p, q, k), float("nan"), device="cuda")
+        circ.circ_fc_backward(h, torch.from_numpy(case.x).cuda(), gd, gx, gw, batch)
         torch.cuda.synchronize()
-        ref_x, _ = oracle.fc_backward(case.w, case.x, g, want_gw=False)
+        ref_x, ref_w = oracle.fc_backward(case.w, case.x, g, convention=convention)
         assert scale_rel_err(gx.cpu().numpy(), ref_x) <= TOL_F32
-        gw = torch.empty(p, q, k, device="cuda")
-        with pytest.raises(circ.CircError) as err:       # weight gradients: powers of two only
-            circ.circ_fc_backward(h, torch.from_numpy(case.x).cuda(), gd, None, gw, batch)
-        assert err.value.code == circ.CIRC_ERR_UNSUPPORTED
+        assert scale_rel_err(gw.cpu().numpy(), ref_w) <= TOL_F32
     finally:
         circ.circ_destroy(h)
+
+
+def test_conv_gradients_any_block_size():
+    k, c_in, c_out = 12, 48, 24
+    case = synth.conv_case("gen_conv_bwd", c_out, c_in, 3, 1, k, 2, 6, 5, w_var=1.0 / (9 * c_in), bf16_io=False)
+    g = synth.normal((case.N, case.H, case.W, c_out), 1.0, synth.stream_id(case.name, "g"))
+    h = circ.circ_conv_create(c_out, c_in, 3, 1, k, case.w)
+    try:
+        circ.circ_set_io_dtype(h, circ.CIRC_F32, circ.CIRC_F32)
+        x = torch.from_numpy(case.x).cuda()
+        gd = torch.from_numpy(g).cuda()
+        gx = torch.full(case.x.shape, float("nan"), device="cuda")
+        gw = torch.full(case.w.shape, float("nan"), device="cuda")
+        circ.circ_conv_backward_input(h, gd, gx, case.N, case.H, case.W)
+        circ.circ_conv_backward_weight(h, x, gd, gw, case.N, case.H, case.W)
+        torch.cuda.synchronize()
+        assert scale_rel_err(gx.cpu().numpy(), oracle.conv_backward_input(case.w, g, case.pad, case.H, case.W)) <= TOL_F32
+        assert scale_rel_err(gw.cpu().numpy(), oracle.conv_backward_weight(case.x, g, 3, case.pad, k)) <= TOL_F32
+    finally:
+        circ.circ_destroy(h)
+
+
+def test_stack_any_block_size():
+    # embedded layers are not relayed: the boundary goes through the stack's activation buffer
+    dims, k, batch = [96, 48, 24], 12, 20
+    cases = [synth.fc_case(f"gen_stack_{i}", dims[i + 1], dims[i], k, batch, w_var=1.0 / dims[i], x_dist="absnormal") for i in range(2)]
+    hs = [circ.circ_fc_create(c.m, c.n, c.k, c.w) for c in cases]
+    try:
+        circ.circ_set_activation(hs[0], 1)
+        st = circ.circ_stack_create(hs)
+        x = torch.from_numpy(cases[0].x).cuda()
+        y = torch.full((batch, dims[-1]), float("nan"), device="cuda")
+        circ.circ_stack_forward(st, x, y, batch)
+        torch.cuda.synchronize()
+        assert circ.circ_stack_relayed(st) == 0
+        a = oracle.fc(cases[0].w, cases[0].x, relu=True)
+        ref = oracle.fc(cases[1].w, a.astype(np.float32))
+        assert scale_rel_err(y.cpu().numpy(), ref) <= TOL_F32
+        circ.circ_stack_destroy(st)
+    finally:
+        for h in hs:
+            circ.circ_destroy(h)
 
 
 def test_fused_refused_and_limit():
