@@ -225,12 +225,30 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
                 const TIN* x0 = x + (size_t)c * n + (size_t)j * ku;
                 const TIN* x1 = x + (size_t)(c + Bh) * n + (size_t)j * ku;
                 const bool second = c + Bh < B;
+                if ((ku & 3) == 0) {
+                    // rows and blocks start on multiples of four elements: whole groups of four are inside or outside
 #pragma unroll
-                for (int r = 0; r < E; ++r) {
-                    const int t = E * l + r;
-                    if (t < ku) {
-                        re[r] = to_float(x0[t]);
-                        if (second) im[r] = to_float(x1[t]);
+                    for (int g4 = 0; g4 < E; g4 += 4) {
+                        const int t = E * l + g4;
+                        if (t < ku) {
+                            float t0[4], t1[4] = {0.f, 0.f, 0.f, 0.f};
+                            load_run<4>(x0 + t, t0);
+                            if (second) load_run<4>(x1 + t, t1);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                re[g4 + e] = t0[e];
+                                im[g4 + e] = t1[e];
+                            }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int r = 0; r < E; ++r) {
+                        const int t = E * l + r;
+                        if (t < ku) {
+                            re[r] = to_float(x0[t]);
+                            if (second) im[r] = to_float(x1[t]);
+                        }
                     }
                 }
             }
@@ -289,32 +307,68 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         // the negative ones at K + s, and the fold is a[t] = c[t] + c[t - ku].)  The fold crosses lanes, so it goes
         // through the tile.
         __syncthreads();   // every thread has taken its bins out of the tile
+        // time-major hand-over, one row of K points per transform; a lane's E points are rotated by the thread's
+        // index so that lanes (whose rows of E points are 8 E bytes apart) fall on different banks
+        float2* ft = &zs[0][0] + (size_t)gi * K;      // TT * K points fit: ROW >= TT
+        const int rot = l + gi * L;
 #pragma unroll
-        for (int r = 0; r < E; ++r) zs[E * l + r][gi] = v[r];
+        for (int r = 0; r < E; ++r) ft[E * l + ((r + rot) & (E - 1))] = v[r];
         __syncthreads();
         if (!live) return;
         const int c = (int)(T / p), i = (int)(T % p);
         const bool second = c + Bho < Bo;
+        float re[E], im[E];
 #pragma unroll
         for (int r = 0; r < E; ++r) {
             const int t = E * l + r;
-            if (t >= ku) continue;
-            float2 a = zs[t][gi];
+            float2 a = v[r];                          // the low part is the lane's own
             const int hi = corr ? K - ku + t : t + ku;
-            if (corr ? t > 0 : hi < K) {
-                const float2 b2 = zs[hi][gi];
+            if (t < ku && (corr ? t > 0 : hi < K)) {
+                const int lh = hi / E;
+                const float2 b2 = ft[E * lh + (((hi & (E - 1)) + lh + gi * L) & (E - 1))];
                 a.x += b2.x;
                 a.y += b2.y;
             }
-            const float bb = bias ? __ldg(bias + i * ku + t) : 0.f;
-            a.x += bb;
-            a.y += bb;
-            if (relu) {
-                a.x = fmaxf(a.x, 0.f);
-                a.y = fmaxf(a.y, 0.f);
+            re[r] = a.x;
+            im[r] = a.y;
+        }
+        TOUT* y0 = y + (size_t)c * m + (size_t)i * ku;
+        TOUT* y1 = y + (size_t)(c + Bho) * m + (size_t)i * ku;
+        if ((ku & 3) == 0) {
+            // rows and blocks start on multiples of four elements: vector loads of the bias, vector stores
+#pragma unroll
+            for (int g4 = 0; g4 < E; g4 += 4) {
+                const int t = E * l + g4;
+                if (t >= ku) continue;
+                float bb[4] = {0.f, 0.f, 0.f, 0.f};
+                if (bias) load_run<4>(bias + i * ku + t, bb);
+                float o0[4], o1[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    o0[e] = re[g4 + e] + bb[e];
+                    o1[e] = im[g4 + e] + bb[e];
+                    if (relu) {
+                        o0[e] = fmaxf(o0[e], 0.f);
+                        o1[e] = fmaxf(o1[e], 0.f);
+                    }
+                }
+                store_run<4>(y0 + t, o0);
+                if (second) store_run<4>(y1 + t, o1);
             }
-            store_one(y + (size_t)c * m + (size_t)i * ku + t, a.x);
-            if (second) store_one(y + (size_t)(c + Bho) * m + (size_t)i * ku + t, a.y);
+        } else {
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const int t = E * l + r;
+                if (t >= ku) continue;
+                const float bb = bias ? __ldg(bias + i * ku + t) : 0.f;
+                float o0 = re[r] + bb, o1 = im[r] + bb;
+                if (relu) {
+                    o0 = fmaxf(o0, 0.f);
+                    o1 = fmaxf(o1, 0.f);
+                }
+                store_one(y0 + t, o0);
+                if (second) store_one(y1 + t, o1);
+            }
         }
         return;
     }
