@@ -310,7 +310,7 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int variant = L->variant;
     if (variant == CIRC_VARIANT_AUTO)
-        variant = fused_fc_supported(L, batch) && batch <= 8 ? CIRC_VARIANT_FUSED
+        variant = fused_fc_preferred(L, batch, tensor_supported(L)) ? CIRC_VARIANT_FUSED
                   : tensor_supported(L)                       ? CIRC_VARIANT_TENSOR
                                                               : CIRC_VARIANT_STAGED;
     if (variant == CIRC_VARIANT_FUSED) {

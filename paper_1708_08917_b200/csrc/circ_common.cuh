@@ -199,5 +199,7 @@ int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, co
 // S4: the whole FC forward in one launch (small batch, weight-streaming).
 int launch_fused_fc(const Layer* L, const void* x, void* y, int batch, cudaStream_t stream);
 bool fused_fc_supported(const Layer* L, int batch);
+// The planner's choice between the one-launch kernel and the tensor-core path (`tensor_ok`: that path can serve the layer).
+bool fused_fc_preferred(const Layer* L, int batch, bool tensor_ok);
 
 }  // namespace circ

@@ -288,6 +288,16 @@ bool fused_fc_supported(const Layer* L, int batch) {
     return fused_smem_bytes(L->geo.k, L->geo.q, pairs, rows, js) <= (size_t)kMaxFusedSmem;
 }
 
+// With 5 to 8 samples every CTA transforms four sample pairs of the whole input, and for long blocks on a wide
+// layer that redundant work outweighs the single launch.  Measured (4096 x 4096, batch 8, one launch against the
+// three-launch tensor path): k = 4: 12.3 / 19.9 us, k = 16: 9.6 / 10.8, k = 64: 10.3 / 8.1, k = 256: 13.3 / 12.4;
+// 2048 x 2048, k = 64: 6.9 / 7.0; batch 4 at k = 64: 6.8 / 7.3.
+bool fused_fc_preferred(const Layer* L, int batch, bool tensor_ok) {
+    if (!fused_fc_supported(L, batch)) return false;
+    if (tensor_ok && batch >= 5 && L->geo.k >= 64 && L->n >= 4096) return false;
+    return true;
+}
+
 template <int K, int PAIRS, typename WT>
 static int launch_one(const FusedArgs& a, unsigned grid, size_t smem, cudaStream_t stream) {
     static thread_local int configured_device = -1;

@@ -24,7 +24,7 @@ struct Stack {
 
 static int variant_for(const Layer* L, int batch) {
     if (L->variant != CIRC_VARIANT_AUTO) return L->variant;
-    if (batch <= 8 && fused_fc_supported(L, batch)) return CIRC_VARIANT_FUSED;
+    if (fused_fc_preferred(L, batch, tensor_supported(L))) return CIRC_VARIANT_FUSED;
     return tensor_supported(L) ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
 }
 
