@@ -31,6 +31,32 @@ struct Tile {
     static constexpr size_t SMEM = sizeof(float2) * ((size_t)K + (size_t)K * ROW) + (size_t)TT * 16;   // twiddle table + staging tile + per-transform output offsets (dynamic shared memory)
 };
 
+// Position of a transform: T = c * rows + i (c: sample pair, i: block).  A CTA's transforms are consecutive, so the
+// one 64-bit division is done for the CTA's first transform and the others follow by small-integer arithmetic
+// (the kernels are bound by instruction issue; a 64-bit division per work item was a third of their instructions).
+struct Split {
+    int c0, i0;
+};
+__device__ __forceinline__ Split split_base(long base, int rows) {
+    const long c = base / rows;
+    return Split{(int)c, (int)(base - c * rows)};
+}
+template <int TT>
+__device__ __forceinline__ void split_at(Split s, int d, int rows, int& c, int& i) {
+    i = s.i0 + d;
+    c = s.c0;
+    if (i >= rows) {
+        if (rows >= TT) {          // at most one wrap
+            i -= rows;
+            ++c;
+        } else {                   // few rows: small 32-bit division
+            const int a = i / rows;
+            i -= a * rows;
+            c += a;
+        }
+    }
+}
+
 __device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
     const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&t);
@@ -46,7 +72,7 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
 // Operand Y -> tile (the first half of S3): fills zs[bin][transform] for the CTA's TT transforms.
 template <int K, int EMAX, bool VEC>
 __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW], const float* __restrict__ yop, int p, int Bho,
-                                               long total) {
+                                               long total, Split sp) {
     constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
     const size_t cols = 2 * (size_t)Bho;
     const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
@@ -63,7 +89,8 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
             const long T0 = (long)blockIdx.x * TT + grp * 4;
             r0[it] = r1[it] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (T0 >= total) continue;
-            const int c = (int)(T0 / p), i = (int)(T0 % p);
+            int c, i;
+            split_at<TT>(sp, grp * 4, p, c, i);
             if (f == 0 || f == K / 2) {
                 const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
                 r0[it] = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
@@ -99,7 +126,8 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
             const int tl = item % TT, f = item / TT;
             const long T2 = (long)blockIdx.x * TT + tl;
             if (T2 >= total) continue;
-            const int c = (int)(T2 / p), i = (int)(T2 % p);
+            int c, i;
+            split_at<TT>(sp, tl, p, c, i);
             float2 z;
             if (f == 0 || f == K / 2) {
                 const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
@@ -121,7 +149,7 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
 // Tile -> operand X (the second half of S1): zs[bin][transform] holds the spectra of the CTA's TT transforms.
 template <int K, int EMAX, int XMODE>
 __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>::ROW], void* __restrict__ xop, int q, int Bh,
-                                                long total) {
+                                                long total, Split sp) {
     constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
     const size_t cols = 2 * (size_t)Bh;
     constexpr int NPART = XMODE == 1 ? 2 : 1;
@@ -134,7 +162,8 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
             const int tl = item % TT, f = item / TT;
             const long T2 = (long)blockIdx.x * TT + tl;
             if (T2 >= total) continue;
-            const int c = (int)(T2 / q), j = (int)(T2 % q);
+            int c, j;
+            split_at<TT>(sp, tl, q, c, j);
             const float2 z = zs[f][tl];
             if (f == 0 || f == K / 2) {
                 float* xg = xf + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
@@ -157,7 +186,8 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
             const int grp = item % GROUPS, f = item / GROUPS;
             const long T0 = (long)blockIdx.x * TT + grp * 4;
             if (T0 >= total) continue;                 // total is a multiple of 8 (q % 8 == 0)
-            const int c = (int)(T0 / q), j = (int)(T0 % q);
+            int c, j;
+            split_at<TT>(sp, grp * 4, q, c, j);
             const float4 za = *reinterpret_cast<const float4*>(&zs[f][grp * 4]);
             const float4 zb = *reinterpret_cast<const float4*>(&zs[f][grp * 4 + 2]);
             if (f == 0 || f == K / 2) {
@@ -210,13 +240,15 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
+    const Split sp = split_base((long)blockIdx.x * TT, q);
     float2 v[E];
     {
         float re[E], im[E];
 #pragma unroll
         for (int r = 0; r < E; ++r) re[r] = im[r] = 0.f;
         if (T < total) {
-            const int c = (int)(T / q), j = (int)(T % q);
+            int c, j;
+            split_at<TT>(sp, gi, q, c, j);
             if (ku == K) {
                 load_run<E>(x + (size_t)c * n + (size_t)j * K + E * l, re);
                 if (c + Bh < B) load_run<E>(x + (size_t)(c + Bh) * n + (size_t)j * K + E * l, im);
@@ -263,7 +295,7 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
 
-    scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total);
+    scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total, sp);
 }
 
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
@@ -281,21 +313,22 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     pdl_trigger();
     pdl_wait();     // Y is written by the contraction kernel before this one
 
-    // the bias of this thread's outputs is fetched now, long before the epilogue needs it
-    float bv[E];
-    {
-        const long Tb = (long)blockIdx.x * TT + threadIdx.x / L;
-#pragma unroll
-        for (int r = 0; r < E; ++r) bv[r] = 0.f;
-        if (bias && Tb < total && ku == K) load_run<E>(bias + (int)(Tb % p) * K + E * (threadIdx.x % L), bv);
-    }
-
-    gather_operand<K, EMAX, VEC>(zs, yop, p, Bho, total);
-    __syncthreads();
-
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
     const bool live = T < total;
+    const Split sp = split_base((long)blockIdx.x * TT, p);
+    int c, i;                     // this thread's transform: sample pair c, row block i
+    split_at<TT>(sp, gi, p, c, i);
+
+    // the bias of this thread's outputs is fetched now, long before the epilogue needs it
+    float bv[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) bv[r] = 0.f;
+    if (bias && live && ku == K) load_run<E>(bias + i * K + E * l, bv);
+
+    gather_operand<K, EMAX, VEC>(zs, yop, p, Bho, total, sp);
+    __syncthreads();
+
     const int f2 = lane_residue<K, EMAX>(l);
     float2 v[E];
 #pragma unroll
@@ -315,7 +348,6 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         for (int r = 0; r < E; ++r) ft[E * l + ((r + rot) & (E - 1))] = v[r];
         __syncthreads();
         if (!live) return;
-        const int c = (int)(T / p), i = (int)(T % p);
         const bool second = c + Bho < Bo;
         float re[E], im[E];
 #pragma unroll
@@ -375,7 +407,6 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     if constexpr (E < 16 || !std::is_same<TOUT, float>::value) {
         // a lane's outputs are at most 32 bytes: direct stores are already (nearly) whole lines per instruction
         if (!live) return;
-        const int c = (int)(T / p), i = (int)(T % p);
         const int col = i * K + E * l;
         float re[E], im[E];
 #pragma unroll
@@ -420,7 +451,6 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         ot[(size_t)(NT + threadIdx.x) * PPL + sl] = make_float4(o[1][0], o[1][1], o[1][2], o[1][3]);
     }
     if (l == 0) {
-        const int c = (int)(T / p), i = (int)(T % p);
         offs[gi] = live ? (long long)c * m + (long long)i * K : -1;
         both[gi] = live && c + Bho < Bo;
     }
@@ -459,12 +489,15 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
     const bool live = T < total;
+    const Split sp = split_base((long)blockIdx.x * TT, p);
+    int c, i;
+    split_at<TT>(sp, gi, p, c, i);
     float bv[E];
 #pragma unroll
     for (int r = 0; r < E; ++r) bv[r] = 0.f;
-    if (bias && live) load_run<E>(bias + (int)(T % p) * K + E * l, bv);
+    if (bias && live) load_run<E>(bias + i * K + E * l, bv);
 
-    gather_operand<K, EMAX, VEC>(zs, yop, p, Bh, total);
+    gather_operand<K, EMAX, VEC>(zs, yop, p, Bh, total, sp);
     __syncthreads();
     const int f2 = lane_residue<K, EMAX>(l);
     float2 v[E];
@@ -473,7 +506,7 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
     fft_inverse<K, EMAX>(v, l, tw);
     {
         // the second sample of the last pair does not exist when the batch is odd: it must enter the next layer as zero
-        const bool second = live && (int)(T / p) + Bh < B;
+        const bool second = live && c + Bh < B;
 #pragma unroll
         for (int r = 0; r < E; ++r) {
             float re = v[r].x + bv[r], im = v[r].y + bv[r];
@@ -489,7 +522,7 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
-    scatter_operand<K, EMAX, XMODE>(zs, xop, p, Bh, total);
+    scatter_operand<K, EMAX, XMODE>(zs, xop, p, Bh, total, sp);
 }
 
 // ---- launchers -------------------------------------------------------------------------------------
