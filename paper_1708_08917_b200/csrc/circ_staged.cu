@@ -298,6 +298,77 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total, sp);
 }
 
+// Bias, activation and stores of one inverse-transformed tile (block size = transform size).  `tile` is the staging
+// tile the bins came from (reused for the hand-over), `offs` / `both` are TT entries of scratch behind it.
+template <int K, int EMAX, typename TOUT>
+__device__ __forceinline__ void store_outputs(const float2 (&v)[FftShape<K, EMAX>::E], const float (&bv)[FftShape<K, EMAX>::E],
+                                              float2 (*zs)[Tile<K, EMAX>::ROW], long long* offs, int* both, int gi, int l, bool live,
+                                              int c, int i, TOUT* __restrict__ y, int relu, int m, int Bo, int Bho) {
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT;
+    if constexpr (E < 16 || !std::is_same<TOUT, float>::value) {
+        // a lane's outputs are at most 32 bytes: direct stores are already (nearly) whole lines per instruction
+        if (!live) return;
+        const int col = i * K + E * l;
+        float re[E], im[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            re[r] = v[r].x + bv[r];
+            im[r] = v[r].y + bv[r];
+            if (relu) {
+                re[r] = fmaxf(re[r], 0.f);
+                im[r] = fmaxf(im[r], 0.f);
+            }
+        }
+        store_run<E>(y + (size_t)c * m + col, re);
+        if (c + Bho < Bo) store_run<E>(y + (size_t)(c + Bho) * m + col, im);
+        return;
+    } else {
+    // A lane holds E consecutive outputs (64 bytes at E = 16), so storing them directly makes every store
+    // instruction write 16-byte pieces 64 bytes apart.  The outputs are instead handed over through the tile
+    // (free once every thread has taken its bins) in 16-byte pieces, and stored with consecutive lanes on
+    // consecutive pieces: whole lines per instruction.  A lane's pieces are permuted (slot = r xor f(thread)) so
+    // that both the writes and the reads of the hand-over are free of bank conflicts.
+    constexpr int PPL = E / 4;                                  // pieces per lane and sample
+    constexpr int NT = Tile<K, EMAX>::NT;
+    float4* ot = reinterpret_cast<float4*>(&zs[0][0]);          // [sample][thread][PPL] pieces; K * ROW * 8 >= 2 * NT * E * 4 bytes
+    auto slot = [](int t, int r) { return PPL == 4 ? (r ^ ((t >> 1) & 3)) : PPL == 8 ? (r ^ (t & 7)) : r; };
+    __syncthreads();   // every thread has taken its bins out of the tile
+#pragma unroll
+    for (int r = 0; r < PPL; ++r) {
+        float o[2][4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            o[0][e] = v[4 * r + e].x + bv[4 * r + e];
+            o[1][e] = v[4 * r + e].y + bv[4 * r + e];
+            if (relu) {
+                o[0][e] = fmaxf(o[0][e], 0.f);
+                o[1][e] = fmaxf(o[1][e], 0.f);
+            }
+        }
+        const int sl = slot((int)threadIdx.x, r);
+        ot[(size_t)threadIdx.x * PPL + sl] = make_float4(o[0][0], o[0][1], o[0][2], o[0][3]);
+        ot[(size_t)(NT + threadIdx.x) * PPL + sl] = make_float4(o[1][0], o[1][1], o[1][2], o[1][3]);
+    }
+    if (l == 0) {
+        offs[gi] = live ? (long long)c * m + (long long)i * K : -1;
+        both[gi] = live && c + Bho < Bo;
+    }
+    __syncthreads();
+    constexpr int PPT = K / 4;                                  // pieces per transform
+#pragma unroll
+    for (int it = 0; it < 2 * PPL; ++it) {
+        const int w = it * NT + (int)threadIdx.x;               // (sample, transform, piece), piece fastest
+        const int pi = w % PPT, g2 = (w / PPT) % TT, smp = w / (PPT * TT);
+        const long long off = offs[g2];
+        if (off < 0 || (smp == 1 && !both[g2])) continue;
+        const int t = g2 * L + pi / PPL;                        // the thread that produced the piece
+        const float4 o = ot[(size_t)(smp * NT + t) * PPL + slot(t, pi % PPL)];
+        const float r4[4] = {o.x, o.y, o.z, o.w};
+        store_run<4>(y + (size_t)off + (smp ? (size_t)Bho * m : 0) + 4 * pi, r4);
+    }
+    }
+}
+
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
 // One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
@@ -404,69 +475,140 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
         }
         return;
     }
-    if constexpr (E < 16 || !std::is_same<TOUT, float>::value) {
-        // a lane's outputs are at most 32 bytes: direct stores are already (nearly) whole lines per instruction
-        if (!live) return;
-        const int col = i * K + E * l;
-        float re[E], im[E];
-#pragma unroll
-        for (int r = 0; r < E; ++r) {
-            re[r] = v[r].x + bv[r];
-            im[r] = v[r].y + bv[r];
-            if (relu) {
-                re[r] = fmaxf(re[r], 0.f);
-                im[r] = fmaxf(im[r], 0.f);
-            }
-        }
-        store_run<E>(y + (size_t)c * m + col, re);
-        if (c + Bho < Bo) store_run<E>(y + (size_t)(c + Bho) * m + col, im);
-        return;
-    } else {
-    // A lane holds E consecutive outputs (64 bytes at E = 16), so storing them directly makes every store
-    // instruction write 16-byte pieces 64 bytes apart.  The outputs are instead handed over through the tile
-    // (free once every thread has taken its bins) in 16-byte pieces, and stored with consecutive lanes on
-    // consecutive pieces: whole lines per instruction.  A lane's pieces are permuted (slot = r xor f(thread)) so
-    // that both the writes and the reads of the hand-over are free of bank conflicts.
-    constexpr int PPL = E / 4;                                  // pieces per lane and sample
-    constexpr int NT = Tile<K, EMAX>::NT;
-    float4* ot = reinterpret_cast<float4*>(&zs[0][0]);          // [sample][thread][PPL] pieces; K * ROW * 8 >= 2 * NT * E * 4 bytes
     long long* offs = reinterpret_cast<long long*>(&zs[0][0] + (size_t)K * ROW);   // [TT] first output element, or -1
-    int* both = reinterpret_cast<int*>(offs + TT);             // [TT] does the pair's second sample exist
-    auto slot = [](int t, int r) { return PPL == 4 ? (r ^ ((t >> 1) & 3)) : PPL == 8 ? (r ^ (t & 7)) : r; };
-    __syncthreads();   // every thread has taken its bins out of the tile
-#pragma unroll
-    for (int r = 0; r < PPL; ++r) {
-        float o[2][4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            o[0][e] = v[4 * r + e].x + bv[4 * r + e];
-            o[1][e] = v[4 * r + e].y + bv[4 * r + e];
-            if (relu) {
-                o[0][e] = fmaxf(o[0][e], 0.f);
-                o[1][e] = fmaxf(o[1][e], 0.f);
-            }
+    int* both = reinterpret_cast<int*>(offs + TT);                                  // [TT] does the pair's second sample exist
+    store_outputs<K, EMAX, TOUT>(v, bv, zs, offs, both, gi, l, live, c, i, y, relu, m, Bo, Bho);
+}
+
+// ---- S3 with bulk-copied tiles ------------------------------------------------------------------------
+// In the complex problems of Y the (Re, Im) pairs of consecutive transforms are consecutive in memory, so a bin's
+// row of the staging tile is one contiguous run of the operand: the tile is fetched by bulk asynchronous copies
+// (cp.async.bulk, one per bin, completion counted on an mbarrier) instead of by loads, address arithmetic and
+// shared-memory stores of every thread.  CTAs are persistent and the tile is double-buffered: while a tile is
+// transformed and stored, the copies of the CTA's next tile are in flight, which keeps enough bytes outstanding to
+// run the memory system at its rate.  Mirror bins (f > K/2) arrive un-negated and are conjugated when read; the two
+// real bins interleave two runs and are fetched with ordinary loads.  Needs 16-byte aligned runs: Bho * p even.
+constexpr uint32_t kBulkSpinLimit = 1u << 22;   // bounded wait: polls before giving up
+
+__device__ __forceinline__ uint32_t bulk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool bulk_wait(uint64_t* bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kBulkSpinLimit; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok) : "r"(bulk_smem_u32(bar)), "r"(parity) : "memory");
+        if (ok) return true;
+        if (it > 64) __nanosleep(64);
+    }
+    return false;
+}
+
+template <int K, typename TOUT>
+__global__ void __launch_bounds__(Tile<K, 16>::NT, 768 / Tile<K, 16>::NT)
+output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const float* __restrict__ bias, int relu, int m, int p,
+                        int Bo, int Bho, long total, int ntiles, int* status) {
+    constexpr int EMAX = 16;
+    constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float2* tw = reinterpret_cast<float2*>(smem_raw);
+    float2 (*z0)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
+    auto zbuf = [&](int b) { return z0 + (size_t)b * K; };      // buffer b: K rows further
+    long long* offs = reinterpret_cast<long long*>(tw + K + (size_t)2 * K * ROW);
+    int* both = reinterpret_cast<int*>(offs + TT);
+    uint64_t* full = reinterpret_cast<uint64_t*>(both + TT + (TT & 1));   // 8-byte aligned
+    load_twiddles<K>(tw);
+    if (threadIdx.x == 0) {
+        for (int b = 0; b < 2; ++b)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bulk_smem_u32(&full[b])), "r"(1));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    pdl_trigger();
+    pdl_wait();     // Y is written by the contraction kernel before this one
+
+    const size_t cols = 2 * (size_t)Bho;
+    const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
+    const int gi = threadIdx.x / L, l = threadIdx.x % L;
+    const int f2 = lane_residue<K, EMAX>(l);
+
+    // bytes of one bin's run in a tile, and the two steps of fetching a tile: thread 0 announces the bytes, then (after a
+    // CTA barrier) thread f issues the copy of bin f
+    auto run_bytes = [&](int tile) {
+        const long left = total - (long)tile * TT;
+        return (uint32_t)((left < TT ? left : TT) * 8);
+    };
+    auto announce = [&](int tile, int b) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bulk_smem_u32(&full[b])),
+                     "r"((uint32_t)(K - 2) * run_bytes(tile)) : "memory");
+    };
+    auto fetch = [&](int tile, int b) {
+        for (int f = threadIdx.x; f < K; f += Tile<K, EMAX>::NT) {
+            if (f == 0 || f == K / 2) continue;
+            const bool mirror = f > K / 2;
+            const int g = mirror ? K - f : f;
+            const float* src = yop + problem_offset(g + 1, real_sz, cplx_sz) + (mirror ? (size_t)Bho * 2 * p : 0) + 2 * (size_t)tile * TT;
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(bulk_smem_u32(&zbuf(b)[f][0])), "l"(src), "r"(run_bytes(tile)), "r"(bulk_smem_u32(&full[b])) : "memory");
         }
-        const int sl = slot((int)threadIdx.x, r);
-        ot[(size_t)threadIdx.x * PPL + sl] = make_float4(o[0][0], o[0][1], o[0][2], o[0][3]);
-        ot[(size_t)(NT + threadIdx.x) * PPL + sl] = make_float4(o[1][0], o[1][1], o[1][2], o[1][3]);
-    }
-    if (l == 0) {
-        offs[gi] = live ? (long long)c * m + (long long)i * K : -1;
-        both[gi] = live && c + Bho < Bo;
-    }
-    __syncthreads();
-    constexpr int PPT = K / 4;                                  // pieces per transform
+    };
+
+    int tile = blockIdx.x;
+    if (tile < ntiles && threadIdx.x == 0) announce(tile, 0);
+    __syncthreads();   // barriers initialised, twiddles ready, bytes announced
+    if (tile < ntiles) fetch(tile, 0);
+
+    bool ok = true;
+    int it = 0;
+    for (; tile < ntiles; tile += gridDim.x, ++it) {
+        const int b = it & 1;
+        const int next = tile + (int)gridDim.x;
+        if (next < ntiles && threadIdx.x == 0) announce(next, b ^ 1);
+
+        const long T = (long)tile * TT + gi;
+        const bool live = T < total;
+        const Split sp = split_base((long)tile * TT, p);
+        int c, i;
+        split_at<TT>(sp, gi, p, c, i);
+        float bv[E];
 #pragma unroll
-    for (int it = 0; it < 2 * PPL; ++it) {
-        const int w = it * NT + (int)threadIdx.x;               // (sample, transform, piece), piece fastest
-        const int pi = w % PPT, g2 = (w / PPT) % TT, smp = w / (PPT * TT);
-        const long long off = offs[g2];
-        if (off < 0 || (smp == 1 && !both[g2])) continue;
-        const int t = g2 * L + pi / PPL;                        // the thread that produced the piece
-        const float4 o = ot[(size_t)(smp * NT + t) * PPL + slot(t, pi % PPL)];
-        const float r4[4] = {o.x, o.y, o.z, o.w};
-        store_run<4>(y + (size_t)off + (smp ? (size_t)Bho * m : 0) + 4 * pi, r4);
+        for (int r = 0; r < E; ++r) bv[r] = 0.f;
+        if (bias && live) load_run<E>(bias + i * K + E * l, bv);
+
+        // the two real bins: (column c, column Bho + c) of problems 0 and 1
+        float4 rb = make_float4(0.f, 0.f, 0.f, 0.f);
+        const long Tr = (long)tile * TT + threadIdx.x;
+        if (threadIdx.x < TT && Tr < total) {
+            const float* y0 = yop + Tr;                   // problem 0, first column group
+            rb = make_float4(__ldg(y0), __ldg(y0 + (size_t)Bho * p), __ldg(y0 + real_sz), __ldg(y0 + real_sz + (size_t)Bho * p));
+        }
+        ok = bulk_wait(&full[b], (uint32_t)(it >> 1) & 1u);
+        if (threadIdx.x < TT) {
+            zbuf(b)[0][threadIdx.x] = make_float2(rb.x, rb.y);
+            zbuf(b)[K / 2][threadIdx.x] = make_float2(rb.z, rb.w);
+        }
+        ok = __syncthreads_and(ok);   // real bins visible; the other buffer's readers finished an iteration ago
+        if (!ok) break;
+        if (next < ntiles) fetch(next, b ^ 1);
+
+        float2 v[E];
+#pragma unroll
+        for (int f1 = 0; f1 < E; ++f1) {
+            const int f = f2 + L * f1;
+            float2 z = zbuf(b)[f][gi];
+            if (f > K / 2) z.y = -z.y;
+            v[f1] = live ? z : make_float2(0.f, 0.f);
+        }
+        fft_inverse<K, EMAX>(v, l, tw);
+        store_outputs<K, EMAX, TOUT>(v, bv, zbuf(b), offs, both, gi, l, live, c, i, y, relu, m, Bo, Bho);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic accesses to this buffer before its next bulk copies
+        __syncthreads();
     }
+    if (!ok) {
+        // a wait gave up: report it, and give the copies that are still in flight (this tile's; the next tile's
+        // have not been issued) one more bounded wait to land before the CTA's shared memory goes away
+        if (threadIdx.x == 0) atomicExch(status, 1);
+        bulk_wait(&full[it & 1], (uint32_t)(it >> 1) & 1u);
     }
 }
 
@@ -610,10 +752,66 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
     return CIRC_OK;
 }
 
+// Resident CTAs per SM of a kernel at a given launch shape, remembered per (kernel, device).
+template <typename Kern>
+static int blocks_per_sm(Kern kernel, int threads, size_t smem) {
+    static thread_local std::vector<std::pair<std::pair<const void*, int>, int>> known;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const std::pair<const void*, int> key(reinterpret_cast<const void*>(kernel), dev);
+    for (const auto& e : known)
+        if (e.first == key) return e.second;
+    int n = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        n = 1;
+    }
+    known.push_back(std::make_pair(key, n));
+    return n;
+}
+
+template <int K>
+static constexpr size_t bulk_smem() {
+    return sizeof(float2) * ((size_t)K + (size_t)2 * K * Tile<K, 16>::ROW) + (size_t)Tile<K, 16>::TT * 12 + 32;
+}
+
 int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation) {
     const int p = L->geo.p, m = L->m;
     const long total = (long)ext.Bho * p;
     const bool small = latency_bound(total, L->geo.k);
+    // large forwards of power-of-two blocks up to 256: tiles fetched by bulk copies, persistent CTAs (needs 16-byte aligned runs)
+    // (measured at 16384 x 16384, batch 1024: k = 16: 40.7 -> 35.2 us, k = 64: 33.7 -> 32.5, k = 256: no change; k = 4, whose
+    // tile has two bulk rows only, is slower this way and keeps the load-based kernel)
+    const bool bulk = !small && !embedded(L->geo) && L->geo.k >= 16 && L->geo.k <= 256 && (total & 1) == 0 && total >= 148L * 256 &&
+                      (reinterpret_cast<uintptr_t>(yop) & 15u) == 0 && L->dev_status != nullptr;
+    if (bulk) {
+        auto go = [&](auto kc) -> int {
+            constexpr int K = decltype(kc)::value;
+            if constexpr (K >= 16 && K <= 256) {
+                constexpr int TT = Tile<K, 16>::TT, NT = Tile<K, 16>::NT;
+                const long ntiles = (total + TT - 1) / TT;
+                if (ntiles >= (1L << 31)) return CIRC_ERR_SHAPE;
+                auto launch = [&](auto tout) {
+                    using TOUT = decltype(tout);
+                    allow_smem(output_ifft_bulk_kernel<K, TOUT>, bulk_smem<K>());
+                    int sms = 148;
+                    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, L->device);
+                    const long resident = (long)sms * blocks_per_sm(output_ifft_bulk_kernel<K, TOUT>, NT, bulk_smem<K>());
+                    const unsigned blocks = (unsigned)(ntiles < resident ? ntiles : resident);
+                    launch_kernel(dependent_launches(), output_ifft_bulk_kernel<K, TOUT>, dim3(blocks), dim3(NT), bulk_smem<K>(), stream, yop,
+                                  static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total,
+                                  (int)ntiles, L->dev_status);
+                };
+                if (L->y_dtype == CIRC_BF16) launch(__nv_bfloat16{}); else launch(float{});
+            }
+            return CIRC_OK;
+        };
+        const int rc = dispatch_k(L->geo.k, go);
+        if (rc != CIRC_OK) return rc;
+        count_launches(1);
+        CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
+        return CIRC_OK;
+    }
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
         auto with_shape = [&](auto ec) {
