@@ -46,12 +46,12 @@ STAGE_SOURCE = {"input_fft": "circ_staged.cu", "output_ifft": "circ_staged.cu", 
 NCU_TRAFFIC: dict = {
     # profiles/dram_traffic_cfg2_b256.md
     ("cfg2_b256", "input_fft"): {"bytes_per_launch": 4211584, "source_sha256": "2c4296cd4a497d41ba9e2d60a62486c6d2ac62b9ec2d83c1bab715597c1b48b4"},
-    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6311936, "source_sha256": "b1286aa4a1f2e6adf1ed24631818ce79970ffd6fdfca0f75a3f88b037158eb89"},
+    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6311936, "source_sha256": "498aaea78199b3c537fdee7af01a5671ff0e1fe543c51cc803d19aac3fb85d99"},
     ("cfg2_b256", "output_ifft"): {"bytes_per_launch": 4230400, "source_sha256": "2c4296cd4a497d41ba9e2d60a62486c6d2ac62b9ec2d83c1bab715597c1b48b4"},
     # profiles/fused_fc_kernel_sweep_n16384_k4_b1.md (dram read + write of one launch)
     ("sweep_n16384_k4_b1", "fused_fc"): {"bytes_per_launch": 275349504, "source_sha256": "dbc004fed09f19ed5d3f515d7ea5396d7c2822a051f4ceaeff60c43cd455ddde"},
     # profiles/contract_tc_kernel_sweep_n16384_k4_b1024.md
-    ("sweep_n16384_k4_b1024", "contraction"): {"bytes_per_launch": 647336448, "source_sha256": "b1286aa4a1f2e6adf1ed24631818ce79970ffd6fdfca0f75a3f88b037158eb89"},
+    ("sweep_n16384_k4_b1024", "contraction"): {"bytes_per_launch": 647336448, "source_sha256": "498aaea78199b3c537fdee7af01a5671ff0e1fe543c51cc803d19aac3fb85d99"},
 }
 
 

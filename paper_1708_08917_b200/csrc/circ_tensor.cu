@@ -239,8 +239,8 @@ __device__ __forceinline__ void issue_taps_k(int ksteps, uint32_t d_tmem, uint64
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The three roles run
 // ahead of one another: the producer keeps the shared-memory ring full across tile boundaries, the
-// MMA warp alternates between two accumulators in tensor memory, and the epilogue warps drain one
-// accumulator while the next tile's products are being formed in the other.
+// MMA warp cycles through the accumulators in tensor memory (2 to 8, as many as its 512 columns hold), and
+// the epilogue warps drain one accumulator while the following tiles' products are being formed in the others.
 __global__ void __launch_bounds__(kTcThreads, 1)
 contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_constant__ CUtensorMap map_a_cplx,
                    const __grid_constant__ CUtensorMap map_xhi_real, const __grid_constant__ CUtensorMap map_xlo_real,
