@@ -273,36 +273,17 @@ CIRC_API int circ_reserve(circ_handle h, long max_batch);
 /* circ_workspace_bytes -- bytes of device workspace currently held by the handle. */
 CIRC_API long circ_workspace_bytes(circ_handle h);
 
+/* circ_weight_bytes -- bytes of device memory the handle holds for the layer's weights, all stored forms
+ * together (the paper's storage figure is m*n/k values, Sec. 3.1: compare against 4*m*n/k). */
+CIRC_API long circ_weight_bytes(circ_handle h);
+
 /* circ_last_variant -- the CIRC_VARIANT_* the most recent forward on this handle used. */
 CIRC_API int circ_last_variant(circ_handle h);
-
-/*
- * circ_profile_begin / circ_profile_end -- per-kernel device times.  Between the two calls every
- * kernel the handle launches is bracketed by CUDA events on its stream.  circ_profile_end waits
- * for them and returns, per stage, the summed milliseconds and the number of launches:
- *   stage 0 = input transforms, 1 = per-frequency contraction, 2 = inverse transforms + epilogue,
- *   stage 3 = the fused one-launch kernel.  Both output arrays have 4 entries (HOST pointers).
- * Profiling adds event records between kernels; do not time whole forwards while it is on.
- */
-CIRC_API int circ_profile_begin(circ_handle h);
-CIRC_API int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage);
-
-/*
- * circ_set_stage_repeat -- timing aid: launch the kernel of `stage` (0..3, numbered as in
- * circ_profile_end) `times` times back to back in every forward of this handle (default 1).  Each of
- * these kernels overwrites its own output from unchanged inputs, so results do not change; the
- * difference in forward time between `times` = 1 + R and `times` = 1, divided by R, is that kernel's
- * duration without any per-event overhead.  Not meant for production calls.
- */
-CIRC_API int circ_set_stage_repeat(circ_handle h, int stage, int times);
 
 /* circ_device_status -- waits for the device (blocking copy of the handle's error word) and
  * returns CIRC_ERR_DEVICE_TIMEOUT if a kernel of this handle gave up on a bounded wait (TMA /
  * tensor-core pipeline barriers) since the last call; the word is cleared.  CIRC_OK otherwise. */
 CIRC_API int circ_device_status(circ_handle h);
-
-/* circ_launch_count -- kernels this library has launched in this process so far. */
-CIRC_API long circ_launch_count(void);
 
 /* circ_last_error / circ_last_code -- message and code of the calling thread's latest failure. */
 CIRC_API const char* circ_last_error(void);

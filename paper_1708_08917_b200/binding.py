@@ -19,6 +19,11 @@ CIRC_OK = 0
 CIRC_ERR_ARG, CIRC_ERR_SHAPE, CIRC_ERR_ALLOC, CIRC_ERR_CUDA, CIRC_ERR_DEVICE_TIMEOUT, CIRC_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
 CIRC_F32, CIRC_BF16 = 0, 1
 CIRC_VARIANT_AUTO, CIRC_VARIANT_FUSED, CIRC_VARIANT_STAGED, CIRC_VARIANT_TENSOR = 0, 1, 2, 3
+# include/circ_debug.h
+CIRC_STAGE_INPUT_FFT, CIRC_STAGE_CONTRACTION, CIRC_STAGE_OUTPUT_IFFT, CIRC_STAGE_FUSED = 0, 1, 2, 3
+CIRC_KERNEL_NONE, CIRC_KERNEL_S1_LOADS, CIRC_KERNEL_S1_BULK = 0, 1, 2
+CIRC_KERNEL_S2_FMA, CIRC_KERNEL_S2_TENSOR, CIRC_KERNEL_S3_LOADS, CIRC_KERNEL_S3_BULK = 10, 11, 20, 21
+CIRC_INJECT_NONE, CIRC_INJECT_TENSOR_NO_COPY, CIRC_INJECT_BULK_NO_COPY = 0, 1, 2
 
 # name -> (restype, argtypes); mirrors include/circ.h one to one
 _vp, _ci, _cl = ctypes.c_void_p, ctypes.c_int, ctypes.c_long
@@ -29,11 +34,8 @@ SIGNATURES = {
     "circ_conv_forward": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_fc_forward_host": (_ci, [_vp, _vp, _vp, _ci, _vp]),
     "circ_conv_forward_host": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
-    "circ_profile_begin": (_ci, [_vp]),
-    "circ_profile_end": (_ci, [_vp, _vp, _vp]),
     "circ_fc_forward_noalloc": (_ci, [_vp, _vp, _vp, _ci, _vp]),
     "circ_noalloc_max_bytes": (_cl, []),
-    "circ_set_stage_repeat": (_ci, [_vp, _ci, _ci]),
     "circ_fc_backward": (_ci, [_vp, _vp, _vp, _vp, _vp, _ci, _vp]),
     "circ_conv_backward_input": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _vp]),
     "circ_conv_backward_weight": (_ci, [_vp, _vp, _vp, _vp, _ci, _ci, _ci, _vp]),
@@ -53,7 +55,15 @@ SIGNATURES = {
     "circ_reserve": (_ci, [_vp, _cl]),
     "circ_workspace_bytes": (_cl, [_vp]),
     "circ_last_variant": (_ci, [_vp]),
-    "circ_launch_count": (_cl, []),
+    "circ_weight_bytes": (_cl, [_vp]),
+    # include/circ_debug.h
+    "circ_debug_forward_repeat": (_ci, [_vp, _vp, _vp, _ci, _ci, _ci, _ci, _ci, _vp]),
+    "circ_debug_last_kernels": (_ci, [_vp, _vp]),
+    "circ_debug_launch_count": (_cl, []),
+    "circ_debug_fma_burn": (_ci, [_vp, _ci, _ci, _vp, _vp]),
+    "circ_debug_empty_kernel": (_ci, [_vp]),
+    "circ_debug_inject": (_ci, [_vp, _ci]),
+    "circ_debug_fail_alloc_after": (_ci, [_cl]),
     "circ_last_error": (ctypes.c_char_p, []),
     "circ_last_code": (_ci, []),
 }
@@ -160,18 +170,6 @@ def circ_conv_forward_host(h: int, x_host, y_host, N: int, H: int, W: int, strea
     _check(load().circ_conv_forward_host(h, _ptr(x_host), _ptr(y_host), N, H, W, _stream(stream)))
 
 
-def circ_profile_begin(h: int) -> None:
-    _check(load().circ_profile_begin(h))
-
-
-def circ_profile_end(h: int):
-    """Returns (ms_by_stage[4], launches_by_stage[4]) as Python lists."""
-    ms = (ctypes.c_float * 4)()
-    cnt = (ctypes.c_int * 4)()
-    _check(load().circ_profile_end(h, ctypes.addressof(ms), ctypes.addressof(cnt)))
-    return list(ms), list(cnt)
-
-
 def circ_fc_forward_noalloc(h: int, x, y, batch: int, stream=None) -> None:
     """``circ_fc_forward`` for callers that may not allocate: scratch lives in a fixed array inside the library.
 
@@ -227,11 +225,6 @@ def circ_stack_destroy(s: int | None) -> None:
     load().circ_stack_destroy(s)
 
 
-def circ_set_stage_repeat(h: int, stage: int, times: int) -> None:
-    """Timing aid: launch the kernel of ``stage`` ``times`` times per forward (results unchanged)."""
-    _check(load().circ_set_stage_repeat(h, stage, times))
-
-
 def circ_device_status(h: int) -> None:
     """Blocks until the device is idle; raises CircError(CIRC_ERR_DEVICE_TIMEOUT) if a bounded wait expired."""
     _check(load().circ_device_status(h))
@@ -280,5 +273,43 @@ def circ_last_variant(h: int) -> int:
     return load().circ_last_variant(h)
 
 
-def circ_launch_count() -> int:
-    return load().circ_launch_count()
+def circ_weight_bytes(h: int) -> int:
+    """Bytes of device memory the handle holds for the layer's weights in all stored forms."""
+    return load().circ_weight_bytes(h)
+
+
+# ---- include/circ_debug.h: test and measurement aids ------------------------------------------------
+
+def circ_debug_forward_repeat(h: int, x, y, N: int, H: int, W: int, stage: int, times: int, stream=None) -> None:
+    """The forward pass with the kernel of ``stage`` launched ``times`` times (results unchanged): per-kernel timing."""
+    _check(load().circ_debug_forward_repeat(h, _ptr(x), _ptr(y), N, H, W, stage, times, _stream(stream)))
+
+
+def circ_debug_last_kernels(h: int) -> list[int]:
+    """CIRC_KERNEL_* ids of the S1 / S2 / S3 kernels of the handle's most recent staged forward."""
+    ids = (ctypes.c_int * 3)()
+    _check(load().circ_debug_last_kernels(h, ctypes.addressof(ids)))
+    return list(ids)
+
+
+def circ_debug_launch_count() -> int:
+    return load().circ_debug_launch_count()
+
+
+def circ_debug_fma_burn(sink, blocks: int, iters: int, stream=None) -> float:
+    """Enqueue the float32 FMA micro-benchmark kernel; returns the flops of the launch."""
+    flops = ctypes.c_double(0.0)
+    _check(load().circ_debug_fma_burn(_ptr(sink), blocks, iters, ctypes.addressof(flops), _stream(stream)))
+    return flops.value
+
+
+def circ_debug_empty_kernel(stream=None) -> None:
+    _check(load().circ_debug_empty_kernel(_stream(stream)))
+
+
+def circ_debug_inject(h: int, kind: int) -> None:
+    _check(load().circ_debug_inject(h, kind))
+
+
+def circ_debug_fail_alloc_after(n: int) -> None:
+    _check(load().circ_debug_fail_alloc_after(n))

@@ -27,7 +27,7 @@ def _stale(target: Path, deps: list[Path]) -> bool:
 def build(force: bool = False, verbose: bool = False) -> Path:
     """Compile every ``csrc/*.cu`` and link them into ``libcirc.so``; returns its path."""
     OBJ.mkdir(exist_ok=True)
-    headers = sorted(CSRC.glob("*.cuh")) + [HERE.parent / "include" / "circ.h"]
+    headers = sorted(CSRC.glob("*.cuh")) + sorted((HERE.parent / "include").glob("*.h"))
     jobs = []
     for src in sources():
         obj = OBJ / (src.stem + ".o")

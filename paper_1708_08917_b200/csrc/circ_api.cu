@@ -26,49 +26,28 @@ void set_error(int code, const char* fmt, ...) {
 }
 void count_launches(long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
-// Optional per-kernel device timing (circ_profile_begin / circ_profile_end).
-struct ProfRec {
-    cudaEvent_t start, stop;
-    int stage;
-};
-struct Profiler {
-    std::vector<ProfRec> recs;
-    std::vector<cudaEvent_t> pool;  // events made ahead of time so that recording stays cheap
-    bool take(cudaEvent_t* e) {
-        if (!pool.empty()) {
-            *e = pool.back();
-            pool.pop_back();
-            return true;
-        }
-        return cudaEventCreate(e) == cudaSuccess;
+long launches_so_far() { return g_launches.load(std::memory_order_relaxed); }
+
+// Device allocation with a test hook: fail_alloc_after(n) makes the n-th allocation from now report
+// cudaErrorMemoryAllocation without calling the runtime (n = 1: the next one; n <= 0: never).
+static std::atomic<long> g_alloc_countdown{0};
+void fail_alloc_after(long n) { g_alloc_countdown.store(n > 0 ? n : 0, std::memory_order_relaxed); }
+cudaError_t dev_alloc(void** ptr, size_t bytes) {
+    long c = g_alloc_countdown.load(std::memory_order_relaxed);
+    while (c > 0 && !g_alloc_countdown.compare_exchange_weak(c, c - 1, std::memory_order_relaxed)) {}
+    if (c == 1) {
+        *ptr = nullptr;
+        return cudaErrorMemoryAllocation;
     }
-};
-struct StageTimer {
-    Profiler* prof;
-    cudaStream_t stream;
-    ProfRec rec;
-    StageTimer(Layer* L, int stage, cudaStream_t s) : prof(static_cast<Profiler*>(L->prof)), stream(s) {
-        if (!prof) return;
-        rec.stage = stage;
-        if (!prof->take(&rec.start) || !prof->take(&rec.stop)) {
-            prof = nullptr;
-            return;
-        }
-        cudaEventRecord(rec.start, stream);
-    }
-    ~StageTimer() {
-        if (!prof) return;
-        cudaEventRecord(rec.stop, stream);
-        prof->recs.push_back(rec);
-    }
-};
+    return cudaMalloc(ptr, bytes);
+}
 
 static bool pow2_in_range(int k) { return k >= 4 && k <= 1024 && (k & (k - 1)) == 0; }
 
 // Copy `count` floats from a host or device pointer into fresh device memory.
 static int to_device(const float* src, size_t count, float** out) {
     float* d = nullptr;
-    if (cudaMalloc(&d, count * sizeof(float)) != cudaSuccess) {
+    if (dev_alloc(&d, count * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "cudaMalloc of %zu bytes failed", count * sizeof(float));
         return CIRC_ERR_ALLOC;
@@ -100,14 +79,6 @@ void free_layer(Layer* L) {
     cudaFree(L->x_stage);
     cudaFree(L->y_stage);
     if (L->transposed) free_layer(L->transposed);
-    if (L->prof) {
-        for (auto& r : static_cast<Profiler*>(L->prof)->recs) {
-            cudaEventDestroy(r.start);
-            cudaEventDestroy(r.stop);
-        }
-        for (auto& e : static_cast<Profiler*>(L->prof)->pool) cudaEventDestroy(e);
-        delete static_cast<Profiler*>(L->prof);
-    }
     if (prev != L->device && prev >= 0) cudaSetDevice(prev);
     delete L;
 }
@@ -144,7 +115,6 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
     L->geo = Geometry{m / k, n / k, kt, taps, r, pad, k};
     L->x_dtype = L->y_dtype = (kind == 1 ? CIRC_BF16 : CIRC_F32);
     L->variant = CIRC_VARIANT_AUTO;
-    for (int st = 0; st < 4; ++st) L->repeat[st] = 1;
     if (cudaGetDevice(&L->device) != cudaSuccess) {
         set_error(CIRC_ERR_CUDA, "no CUDA device: %s", cudaGetErrorString(cudaGetLastError()));
         delete L;
@@ -157,10 +127,10 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
     }
     const size_t a_real = (size_t)taps * (m / k) * (n / k);
     L->a_elems = 2 * a_real + (size_t)(kt / 2 - 1) * 4 * a_real;
-    bool ok = cudaMalloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
-              cudaMalloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
-              cudaMalloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
-              cudaMalloc(&L->dev_status, sizeof(int)) == cudaSuccess;
+    bool ok = dev_alloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
+              dev_alloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
+              dev_alloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
+              dev_alloc(&L->dev_status, sizeof(int)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "device allocation of the weight spectra failed");
@@ -187,7 +157,7 @@ int ensure_workspace(Layer* L, size_t need) {
     if (L->ws) cudaFree(L->ws);  // implicit synchronisation: earlier forwards have finished with it
     L->ws = nullptr;
     L->ws_bytes = 0;
-    if (cudaMalloc(&L->ws, need) != cudaSuccess) {
+    if (dev_alloc(&L->ws, need) != cudaSuccess) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "workspace allocation of %zu bytes failed", need);
         return CIRC_ERR_ALLOC;
@@ -196,7 +166,7 @@ int ensure_workspace(Layer* L, size_t need) {
     return CIRC_OK;
 }
 
-static Extent fc_extent(int batch) {
+Extent fc_extent(int batch) {
     Extent e;
     e.B = e.Bo = batch;
     e.Bh = e.Bho = (batch + 1) / 2;
@@ -206,7 +176,7 @@ static Extent fc_extent(int batch) {
     return e;
 }
 
-static Extent conv_extent(const Layer* L, int N, int H, int W) {
+Extent conv_extent(const Layer* L, int N, int H, int W) {
     Extent e;
     e.H = H;
     e.W = W;
@@ -238,41 +208,76 @@ static int check_io(const Layer* L, const void* x, const void* y) {
     return CIRC_OK;
 }
 
-static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
-    int rc = ensure_workspace(L, workspace_need(L, e));
+// Workspace of a staged forward: operand X, then operand Y.
+bool stream_is_capturing(cudaStream_t stream) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &st) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return st != cudaStreamCaptureStatusNone;
+}
+
+int staged_operands(Layer* L, const Extent& e, cudaStream_t stream, float** xop, float** yop) {
+    const size_t need = workspace_need(L, e);
+    if (L->ws_bytes < need && stream_is_capturing(stream)) {
+        // growing frees and allocates, which a capturing stream cannot record: say so before anything is enqueued
+        set_error(CIRC_ERR_UNSUPPORTED, "the workspace (%zu bytes) is too small for this forward (%zu bytes) and the stream is "
+                  "being captured: call circ_reserve before the capture", L->ws_bytes, need);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    const int rc = ensure_workspace(L, need);
     if (rc != CIRC_OK) return rc;
-    float* xop = static_cast<float*>(L->ws);
-    float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
-    // small forwards (none of the three kernels fills the machine) overlap each kernel's launch and set-up with
-    // its predecessor; reset on every exit path by the guard
-    struct DependentGuard {
-        DependentGuard(bool on) { dependent_launches() = on; }
-        ~DependentGuard() { dependent_launches() = false; }
-    } guard(!L->prof && (long)e.Bh * (L->geo.p > L->geo.q ? L->geo.p : L->geo.q) * L->geo.k <= 32768);
-    {
-        StageTimer t(L, 0, stream);
-        // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16
-        const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
-        for (int rep = 0; rep < L->repeat[0]; ++rep)
-            if ((rc = launch_input_fft(L, x, xop, xmode, e, stream)) != CIRC_OK) return rc;
+    *xop = static_cast<float*>(L->ws);
+    *yop = *xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
+    return CIRC_OK;
+}
+
+// Small forwards (none of the three kernels fills the machine) overlap each kernel's launch and set-up with its
+// predecessor (programmatic dependent launch).
+int staged_dependent_launches(const Layer* L, const Extent& e) {
+    return (long)e.Bh * (L->geo.p > L->geo.q ? L->geo.p : L->geo.q) * L->geo.k <= 32768 ? PDL_EARLY : PDL_LATE;
+}
+
+int stage_input(Layer* L, const void* x, float* xop, const Extent& e, cudaStream_t stream, bool tensor) {
+    // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16
+    const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
+    return launch_input_fft(L, x, xop, xmode, e, stream);
+}
+
+int stage_contract(Layer* L, const float* xop, float* yop, const Extent& e, cudaStream_t stream, bool tensor) {
+    if (tensor) {
+        L->last_kernels[1] = KERNEL_S2_TENSOR;
+        return launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
     }
-    {
-        StageTimer t(L, 1, stream);
-        for (int rep = 0; rep < L->repeat[1]; ++rep) {
-            if (tensor)
-                rc = launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
-            else
-                rc = launch_contract_fma(L, xop, yop, e, stream);
-            if (rc != CIRC_OK) return rc;
-        }
-    }
-    {
-        StageTimer t(L, 2, stream);
-        for (int rep = 0; rep < L->repeat[2]; ++rep)
-            if ((rc = launch_output_ifft(L, yop, y, e, stream)) != CIRC_OK) return rc;
-    }
+    L->last_kernels[1] = KERNEL_S2_FMA;
+    return launch_contract_fma(L, xop, yop, e, stream);
+}
+
+int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream) {
+    return launch_output_ifft(L, yop, y, e, stream);
+}
+
+static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
+    float *xop = nullptr, *yop = nullptr;
+    int rc = staged_operands(L, e, stream, &xop, &yop);
+    if (rc != CIRC_OK) return rc;
+    struct DependentGuard {   // reset on every exit path
+        DependentGuard(int mode) { dependent_launches() = mode; }
+        ~DependentGuard() { dependent_launches() = PDL_OFF; }
+    } guard(staged_dependent_launches(L, e));
+    if ((rc = stage_input(L, x, xop, e, stream, tensor)) != CIRC_OK) return rc;
+    if ((rc = stage_contract(L, xop, yop, e, stream, tensor)) != CIRC_OK) return rc;
+    if ((rc = stage_output(L, yop, y, e, stream)) != CIRC_OK) return rc;
     L->last_variant = tensor ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
     return CIRC_OK;
+}
+
+int plan_fc_variant(const Layer* L, int batch) {
+    if (L->variant != CIRC_VARIANT_AUTO) return L->variant;
+    return fused_fc_preferred(L, batch, tensor_supported(L)) ? CIRC_VARIANT_FUSED
+           : tensor_supported(L)                            ? CIRC_VARIANT_TENSOR
+                                                            : CIRC_VARIANT_STAGED;
 }
 
 }  // namespace circ
@@ -308,20 +313,13 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
         return CIRC_ERR_SHAPE;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    int variant = L->variant;
-    if (variant == CIRC_VARIANT_AUTO)
-        variant = fused_fc_preferred(L, batch, tensor_supported(L)) ? CIRC_VARIANT_FUSED
-                  : tensor_supported(L)                       ? CIRC_VARIANT_TENSOR
-                                                              : CIRC_VARIANT_STAGED;
+    const int variant = plan_fc_variant(L, batch);
     if (variant == CIRC_VARIANT_FUSED) {
         if (!fused_fc_supported(L, batch)) {
             set_error(CIRC_ERR_UNSUPPORTED, "the fused kernel does not serve batch=%d for this layer", batch);
             return CIRC_ERR_UNSUPPORTED;
         }
-        {
-            StageTimer t(L, 3, s);
-            for (int rep = 0; rep < L->repeat[3] && rc == CIRC_OK; ++rep) rc = launch_fused_fc(L, x, y, batch, s);
-        }
+        rc = launch_fused_fc(L, x, y, batch, s);
         if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
         return rc;
     }
@@ -362,7 +360,7 @@ static int ensure_stage(Layer* L, size_t xbytes, size_t ybytes) {
         cudaFree(L->x_stage);
         L->x_stage = nullptr;
         L->x_stage_bytes = 0;
-        if (cudaMalloc(&L->x_stage, xbytes) != cudaSuccess) {
+        if (dev_alloc(&L->x_stage, xbytes) != cudaSuccess) {
             cudaGetLastError();
             set_error(CIRC_ERR_ALLOC, "staging allocation of %zu bytes failed", xbytes);
             return CIRC_ERR_ALLOC;
@@ -373,7 +371,7 @@ static int ensure_stage(Layer* L, size_t xbytes, size_t ybytes) {
         cudaFree(L->y_stage);
         L->y_stage = nullptr;
         L->y_stage_bytes = 0;
-        if (cudaMalloc(&L->y_stage, ybytes) != cudaSuccess) {
+        if (dev_alloc(&L->y_stage, ybytes) != cudaSuccess) {
             cudaGetLastError();
             set_error(CIRC_ERR_ALLOC, "staging allocation of %zu bytes failed", ybytes);
             return CIRC_ERR_ALLOC;
@@ -420,66 +418,6 @@ int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int 
     if ((rc = circ_conv_forward(h, L->x_stage, L->y_stage, N, H, W, stream)) != CIRC_OK) return rc;
     CIRC_CUDA_TRY(cudaMemcpyAsync(y_host, L->y_stage, yb, cudaMemcpyDeviceToHost, s), CIRC_ERR_CUDA);
     return CIRC_OK;
-}
-
-int circ_set_stage_repeat(circ_handle h, int stage, int times) {
-    Layer* L = reinterpret_cast<Layer*>(h);
-    if (!L || stage < 0 || stage > 3 || times < 1 || times > 64) {
-        set_error(CIRC_ERR_ARG, "bad handle, stage %d not in [0,3] or times %d not in [1,64]", stage, times);
-        return CIRC_ERR_ARG;
-    }
-    L->repeat[stage] = times;
-    return CIRC_OK;
-}
-
-int circ_profile_begin(circ_handle h) {
-    Layer* L = reinterpret_cast<Layer*>(h);
-    if (!L) {
-        set_error(CIRC_ERR_ARG, "handle is NULL");
-        return CIRC_ERR_ARG;
-    }
-    if (!L->prof) L->prof = new (std::nothrow) Profiler();
-    if (!L->prof) {
-        set_error(CIRC_ERR_ALLOC, "host allocation failed");
-        return CIRC_ERR_ALLOC;
-    }
-    Profiler* P = static_cast<Profiler*>(L->prof);
-    while (P->pool.size() < 512) {
-        cudaEvent_t e;
-        if (cudaEventCreate(&e) != cudaSuccess) break;
-        P->pool.push_back(e);
-    }
-    return CIRC_OK;
-}
-
-int circ_profile_end(circ_handle h, float* ms_by_stage, int* launches_by_stage) {
-    Layer* L = reinterpret_cast<Layer*>(h);
-    if (!L || !L->prof || !ms_by_stage || !launches_by_stage) {
-        set_error(CIRC_ERR_ARG, "bad handle / profiling not started / NULL output");
-        return CIRC_ERR_ARG;
-    }
-    Profiler* P = static_cast<Profiler*>(L->prof);
-    for (int s = 0; s < 4; ++s) {
-        ms_by_stage[s] = 0.f;
-        launches_by_stage[s] = 0;
-    }
-    int rc = CIRC_OK;
-    for (auto& r : P->recs) {
-        float ms = 0.f;
-        if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) {
-            set_error(CIRC_ERR_CUDA, "event timing failed: %s", cudaGetErrorString(cudaGetLastError()));
-            rc = CIRC_ERR_CUDA;
-        } else if (r.stage >= 0 && r.stage < 4) {
-            ms_by_stage[r.stage] += ms;
-            launches_by_stage[r.stage] += 1;
-        }
-        cudaEventDestroy(r.start);
-        cudaEventDestroy(r.stop);
-    }
-    for (auto& e : P->pool) cudaEventDestroy(e);
-    delete P;
-    L->prof = nullptr;
-    return rc;
 }
 
 int circ_device_status(circ_handle h) {
@@ -560,7 +498,7 @@ int circ_set_spectrum_dtype(circ_handle h, int dtype) {
     if (dtype == CIRC_BF16 && !L->w_stream_bf16) {
         const size_t count = (size_t)L->geo.taps * L->geo.p * L->geo.q * L->geo.k;
         CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
-        if (cudaMalloc(&L->w_stream_bf16, count * sizeof(__nv_bfloat16)) != cudaSuccess) {
+        if (dev_alloc(&L->w_stream_bf16, count * sizeof(__nv_bfloat16)) != cudaSuccess) {
             cudaGetLastError();
             L->w_stream_bf16 = nullptr;
             set_error(CIRC_ERR_ALLOC, "allocation of the bfloat16 spectra (%zu bytes) failed", count * sizeof(__nv_bfloat16));
@@ -602,12 +540,25 @@ long circ_workspace_bytes(circ_handle h) {
     return L ? (long)L->ws_bytes : 0;
 }
 
+long circ_weight_bytes(circ_handle h) {
+    const Layer* L = reinterpret_cast<const Layer*>(h);
+    if (!L) return 0;
+    const size_t blocks = (size_t)L->geo.taps * L->geo.p * L->geo.q;
+    size_t b = 0;
+    if (L->w_dev) b += blocks * L->geo.ku * sizeof(float);
+    if (L->w_stream) b += blocks * L->geo.k * sizeof(float);
+    if (L->w_stream_bf16) b += blocks * L->geo.k * sizeof(__nv_bfloat16);
+    if (L->a_f32) b += L->a_elems * sizeof(float);
+    if (L->a_bf16) b += 2 * L->a_elems * sizeof(__nv_bfloat16) + 256;
+    if (L->transposed) b += (size_t)circ_weight_bytes(reinterpret_cast<circ_handle>(L->transposed));
+    return (long)b;
+}
+
 int circ_last_variant(circ_handle h) {
     Layer* L = reinterpret_cast<Layer*>(h);
     return L ? L->last_variant : 0;
 }
 
-long circ_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 const char* circ_last_error(void) { return g_err; }
 int circ_last_code(void) { return g_code; }
 

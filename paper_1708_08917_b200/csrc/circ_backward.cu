@@ -491,7 +491,7 @@ static int build_transposed(Layer* L) {
     const int p = L->geo.p, q = L->geo.q, k = L->geo.ku, r = L->geo.r, taps = L->geo.taps;   // the caller's block size: W^T is
     float* wt = nullptr;                                                                       // built from the defining vectors
     const size_t count = (size_t)taps * p * q * k;
-    if (cudaMalloc(&wt, count * sizeof(float)) != cudaSuccess) {
+    if (dev_alloc(&wt, count * sizeof(float)) != cudaSuccess) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "allocation of the transposed weights (%zu bytes) failed", count * sizeof(float));
         return CIRC_ERR_ALLOC;

@@ -96,15 +96,47 @@ struct Layer {
     void* x_stage;      // device staging buffers of the host-pointer entry points
     void* y_stage;
     size_t x_stage_bytes, y_stage_bytes;
-    void* prof;         // per-kernel timing records while profiling is on, else nullptr
-    int repeat[4];      // how many times each stage's kernel is launched per forward (1; more only for timing)
+    mutable int last_kernels[3];  // which S1 / S2 / S3 kernel served the most recent staged forward (KERNEL_* ids below)
+    int inject;           // test-only fault injection (circ_debug.h): 0 = none
     Layer* transposed;  // the n x m layer W^T (built on first use by the backward pass), or nullptr
 };
+
+// Kernel ids recorded in Layer::last_kernels (read back through circ_debug_last_kernels).
+enum {
+    KERNEL_NONE = 0,
+    KERNEL_S1_LOADS = 1,      // input transforms, per-thread vector loads
+    KERNEL_S1_BULK = 2,       // input transforms, tiles staged by bulk asynchronous copies
+    KERNEL_S2_FMA = 10,       // contraction on the float32 FMA pipes
+    KERNEL_S2_TENSOR = 11,    // contraction on the tensor cores
+    KERNEL_S3_LOADS = 20,     // inverse transforms, per-thread loads
+    KERNEL_S3_BULK = 21       // inverse transforms, tiles staged by bulk asynchronous copies
+};
+
+// Test-only fault injection (circ_debug_inject): the named producer issues no copy and every bounded wait of that
+// kernel gets a short limit, so that the consumer's wait runs out with nothing in flight.
+enum { INJECT_NONE = 0, INJECT_TENSOR_NO_COPY = 1, INJECT_BULK_NO_COPY = 2 };
 
 // Layer life cycle and workspace (circ_api.cu).
 Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const float* w);
 void free_layer(Layer* L);
 int ensure_workspace(Layer* L, size_t bytes);
+// Every device allocation of the library goes through here (tests can make the n-th one fail: circ_debug.h).
+cudaError_t dev_alloc(void** ptr, size_t bytes);
+template <typename T>
+inline cudaError_t dev_alloc(T** ptr, size_t bytes) { return dev_alloc(reinterpret_cast<void**>(ptr), bytes); }
+void fail_alloc_after(long n);
+long launches_so_far();
+
+// The three stages of the staged forward, each exactly one kernel launch (circ_api.cu).
+int staged_operands(Layer* L, const Extent& e, cudaStream_t stream, float** xop, float** yop);
+bool stream_is_capturing(cudaStream_t stream);
+int stage_input(Layer* L, const void* x, float* xop, const Extent& e, cudaStream_t stream, bool tensor);
+int stage_contract(Layer* L, const float* xop, float* yop, const Extent& e, cudaStream_t stream, bool tensor);
+int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream);
+int staged_dependent_launches(const Layer* L, const Extent& e);
+Extent fc_extent(int batch);
+Extent conv_extent(const Layer* L, int N, int H, int W);
+int plan_fc_variant(const Layer* L, int batch);     // the planner's CIRC_VARIANT_* for a fully-connected forward
 
 // Thread-local error record.
 void set_error(int code, const char* fmt, ...);
@@ -123,29 +155,28 @@ void count_launches(long n);
 // Programmatic dependent launch.  A kernel launched with the "programmatic stream serialization"
 // attribute may be scheduled while its predecessor in the stream still runs, so that its launch
 // latency and set-up overlap the predecessor's work.  The contract every forward kernel keeps:
-//   pdl_trigger()  first thing: lets the next kernel's thread blocks be scheduled as soon as every block of
-//                  this kernel has started, so that its launch latency and set-up (twiddle tables, barriers,
-//                  tensor memory) overlap this kernel's work;
+//   pdl_trigger()  lets the next kernel's thread blocks be scheduled once every block of this kernel has
+//                  issued it (or exited).  Small forwards issue it first thing (PDL_EARLY): the next kernel's
+//                  blocks become resident at once and their set-up (twiddle tables, barriers, tensor memory)
+//                  overlaps this kernel's work.  Forwards whose kernels fill the machine issue it when a block
+//                  has only its stores left (PDL_LATE): resident waiting blocks would take registers and shared
+//                  memory away from this kernel's later waves, but the next launch still overlaps the tail.
 //   pdl_wait()     before the first access to global memory: blocks until all earlier kernels have
 //                  finished and their writes are visible.
-// Both are no-ops when the kernel was launched without the attribute.  Waiting blocks hold registers and
-// shared memory, so the attribute only pays when the kernels involved do not fill the machine.  Measured on
-// B200 for the three-kernel path: 10 - 14 % faster at 32 Ki transform points per forward (4096 x 4096, k = 64,
-// batch 16: 9.3 -> 8.3 us; 1024 x 1024, k = 16, batch 64: 8.4 -> 7.2 us), 4 - 40 % slower from 128 Ki points up.
-// The forward pass therefore asks for it (`dependent_launches()`) below 32 Ki points only; the one-launch
-// fused kernel always does.
+// Both are no-ops when the kernel was launched without the attribute.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Whether the staged kernels launched by this thread ask for programmatic dependent launch (set by the forward pass).
-inline bool& dependent_launches() {
-    static thread_local bool on = false;
-    return on;
+enum { PDL_OFF = 0, PDL_EARLY = 1, PDL_LATE = 2 };
+// How the staged kernels launched by this thread use programmatic dependent launch (set by the forward pass).
+inline int& dependent_launches() {
+    static thread_local int mode = PDL_OFF;
+    return mode;
 }
 
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+inline cudaError_t launch_kernel(int dependent, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -155,7 +186,7 @@ inline cudaError_t launch_kernel(bool dependent, void (*kernel)(KArgs...), dim3 
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = dependent ? 1 : 0;
+    cfg.numAttrs = dependent != PDL_OFF ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 

@@ -20,11 +20,12 @@ struct ContractArgs {
     int p, q, k, taps, r, pad;
     int cols_in, cols_out;  // 2*Bh, 2*Bho
     int H, W, Ho, Wo;
+    int pdl_late;           // issue the dependent-launch trigger before the stores instead of first thing
 };
 
 template <bool CONV>
 __global__ void __launch_bounds__(256) contract_fma_kernel(ContractArgs g) {
-    pdl_trigger();
+    if (!g.pdl_late) pdl_trigger();
     pdl_wait();     // X is written by the transform kernel before this one
     const int prob = blockIdx.z;
     const bool real = problem_is_real(prob);
@@ -112,6 +113,7 @@ __global__ void __launch_bounds__(256) contract_fma_kernel(ContractArgs g) {
         }
         __syncthreads();
     }
+    if (g.pdl_late) pdl_trigger();
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
         const int col = n0 + ty + 16 * b;
@@ -133,6 +135,7 @@ int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Exte
     g.cols_in = 2 * ext.Bh;
     g.cols_out = 2 * ext.Bho;
     g.H = ext.H; g.W = ext.W; g.Ho = ext.Ho; g.Wo = ext.Wo;
+    g.pdl_late = dependent_launches() == PDL_LATE;
     dim3 grid((g.cols_out + BN - 1) / BN, (2 * g.p + BM - 1) / BM, num_problems(g.k));
     if (L->kind == 1)
         launch_kernel(dependent_launches(), contract_fma_kernel<true>, grid, dim3(256), 0, stream, g);

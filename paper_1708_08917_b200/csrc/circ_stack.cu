@@ -39,7 +39,7 @@ static int grow_activations(Stack* S, size_t need) {
     cudaFree(S->act[1]);
     S->act[0] = S->act[1] = nullptr;
     S->act_bytes = 0;
-    if (cudaMalloc(&S->act[0], need) != cudaSuccess || cudaMalloc(&S->act[1], need) != cudaSuccess) {
+    if (dev_alloc(&S->act[0], need) != cudaSuccess || dev_alloc(&S->act[1], need) != cudaSuccess) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "allocation of the intermediate activations (2 x %zu bytes) failed", need);
         return CIRC_ERR_ALLOC;

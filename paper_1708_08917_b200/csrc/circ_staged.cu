@@ -229,13 +229,13 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
 template <int K, int EMAX, typename TIN, int XMODE>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
-                 int B, int Bh, long total, int ku) {
+                 int B, int Bh, long total, int ku, int pdl_late) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_trigger();
+    if (!pdl_late) pdl_trigger();
     pdl_wait();     // x may come from the kernel before; the operand buffer may still be read by it
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
@@ -295,6 +295,7 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
 
+    if (pdl_late) pdl_trigger();
     scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total, sp);
 }
 
@@ -375,13 +376,13 @@ __device__ __forceinline__ void store_outputs(const float2 (&v)[FftShape<K, EMAX
 template <int K, int EMAX, typename TOUT, bool VEC>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
-                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku, int corr) {
+                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku, int corr, int pdl_late) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_trigger();
+    if (!pdl_late) pdl_trigger();
     pdl_wait();     // Y is written by the contraction kernel before this one
 
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
@@ -405,6 +406,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) v[f1] = live ? zs[f2 + L * f1][gi] : make_float2(0.f, 0.f);
     fft_inverse<K, EMAX>(v, l, tw);
+    if (pdl_late) pdl_trigger();
     if (ku != K) {
         // embedded block size: v is the linear convolution (2 ku - 1 points) of the zero-padded blocks; the
         // circular one folds it, a[t] = c[t] + c[t + ku].  (corr: v is a linear correlation with lags -ku < s < ku,
@@ -491,8 +493,8 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
 constexpr uint32_t kBulkSpinLimit = 1u << 22;   // bounded wait: polls before giving up
 
 __device__ __forceinline__ uint32_t bulk_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ bool bulk_wait(uint64_t* bar, uint32_t parity) {
-    for (uint32_t it = 0; it < kBulkSpinLimit; ++it) {
+__device__ __forceinline__ bool bulk_wait(uint64_t* bar, uint32_t parity, uint32_t limit = kBulkSpinLimit) {
+    for (uint32_t it = 0; it < limit; ++it) {
         uint32_t ok;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
@@ -508,8 +510,9 @@ __device__ __forceinline__ bool bulk_wait(uint64_t* bar, uint32_t parity) {
 template <int K, typename TOUT>
 __global__ void __launch_bounds__(Tile<K, 16>::NT, 768 / Tile<K, 16>::NT)
 output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, const float* __restrict__ bias, int relu, int m, int p,
-                        int Bo, int Bho, long total, int ntiles, int* status) {
+                        int Bo, int Bho, long total, int ntiles, int* status, int no_copy, int pdl_late) {
     constexpr int EMAX = 16;
+    const uint32_t spin_limit = no_copy ? (1u << 12) : kBulkSpinLimit;   // no_copy: fault injection (tests only)
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
@@ -524,7 +527,7 @@ output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, con
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bulk_smem_u32(&full[b])), "r"(1));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    pdl_trigger();
+    if (!pdl_late) pdl_trigger();
     pdl_wait();     // Y is written by the contraction kernel before this one
 
     const size_t cols = 2 * (size_t)Bho;
@@ -543,6 +546,7 @@ output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, con
                      "r"((uint32_t)(K - 2) * run_bytes(tile)) : "memory");
     };
     auto fetch = [&](int tile, int b) {
+        if (no_copy) return;               // the bytes were announced, nothing is in flight: the wait below runs out
         for (int f = threadIdx.x; f < K; f += Tile<K, EMAX>::NT) {
             if (f == 0 || f == K / 2) continue;
             const bool mirror = f > K / 2;
@@ -582,7 +586,7 @@ output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, con
             const float* y0 = yop + Tr;                   // problem 0, first column group
             rb = make_float4(__ldg(y0), __ldg(y0 + (size_t)Bho * p), __ldg(y0 + real_sz), __ldg(y0 + real_sz + (size_t)Bho * p));
         }
-        ok = bulk_wait(&full[b], (uint32_t)(it >> 1) & 1u);
+        ok = bulk_wait(&full[b], (uint32_t)(it >> 1) & 1u, spin_limit);
         if (threadIdx.x < TT) {
             zbuf(b)[0][threadIdx.x] = make_float2(rb.x, rb.y);
             zbuf(b)[K / 2][threadIdx.x] = make_float2(rb.z, rb.w);
@@ -604,11 +608,12 @@ output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, con
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic accesses to this buffer before its next bulk copies
         __syncthreads();
     }
+    if (pdl_late) pdl_trigger();
     if (!ok) {
         // a wait gave up: report it, and give the copies that are still in flight (this tile's; the next tile's
         // have not been issued) one more bounded wait to land before the CTA's shared memory goes away
         if (threadIdx.x == 0) atomicExch(status, 1);
-        bulk_wait(&full[it & 1], (uint32_t)(it >> 1) & 1u);
+        if (!no_copy) bulk_wait(&full[it & 1], (uint32_t)(it >> 1) & 1u, spin_limit);
     }
 }
 
@@ -620,13 +625,13 @@ output_ifft_bulk_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, con
 template <int K, int EMAX, int XMODE, bool VEC>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float* __restrict__ bias, int relu, int p, int B, int Bh,
-             long total) {
+             long total, int pdl_late) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
     float2 (*zs)[ROW] = reinterpret_cast<float2 (*)[ROW]>(tw + K);
     load_twiddles<K>(tw);
-    pdl_trigger();
+    if (!pdl_late) pdl_trigger();
     pdl_wait();
     const int gi = threadIdx.x / L, l = threadIdx.x % L;
     const long T = (long)blockIdx.x * TT + gi;
@@ -664,6 +669,7 @@ relay_kernel(const float* __restrict__ yop, void* __restrict__ xop, const float*
 #pragma unroll
     for (int f1 = 0; f1 < E; ++f1) zs[f2 + L * f1][gi] = v[f1];
     __syncthreads();
+    if (pdl_late) pdl_trigger();
     scatter_operand<K, EMAX, XMODE>(zs, xop, p, Bh, total, sp);
 }
 
@@ -730,7 +736,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
                 constexpr int XMODE = decltype(mode)::value;
                 allow_smem(input_fft_kernel<K, EMAX, TIN, XMODE>, Tile<K, EMAX>::SMEM);
                 launch_kernel(dependent_launches(), input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
-                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku);
+                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku, (int)(dependent_launches() == PDL_LATE));
             };
             const bool bf = L->x_dtype == CIRC_BF16;
             if (xmode == 0) {
@@ -747,6 +753,7 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
     };
     const int rc = dispatch_k(L->geo.k, go);
     if (rc != CIRC_OK) return rc;
+    L->last_kernels[0] = KERNEL_S1_LOADS;
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
     return CIRC_OK;
@@ -800,7 +807,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
                     const unsigned blocks = (unsigned)(ntiles < resident ? ntiles : resident);
                     launch_kernel(dependent_launches(), output_ifft_bulk_kernel<K, TOUT>, dim3(blocks), dim3(NT), bulk_smem<K>(), stream, yop,
                                   static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total,
-                                  (int)ntiles, L->dev_status);
+                                  (int)ntiles, L->dev_status, (int)(L->inject == INJECT_BULK_NO_COPY), (int)(dependent_launches() == PDL_LATE));
                 };
                 if (L->y_dtype == CIRC_BF16) launch(__nv_bfloat16{}); else launch(float{});
             }
@@ -808,6 +815,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
         };
         const int rc = dispatch_k(L->geo.k, go);
         if (rc != CIRC_OK) return rc;
+        L->last_kernels[2] = KERNEL_S3_BULK;
         count_launches(1);
         CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
         return CIRC_OK;
@@ -823,7 +831,8 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
                 launch_kernel(dependent_launches(), output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
-                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku, (int)correlation);
+                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku, (int)correlation,
+                              (int)(dependent_launches() == PDL_LATE));
             };
             const bool vec = (p % 4) == 0;
             if (L->y_dtype == CIRC_BF16) {
@@ -838,6 +847,7 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
     };
     const int rc = dispatch_k(L->geo.k, go);
     if (rc != CIRC_OK) return rc;
+    L->last_kernels[2] = KERNEL_S3_LOADS;
     count_launches(1);
     CIRC_CUDA_TRY(cudaGetLastError(), CIRC_ERR_CUDA);
     return CIRC_OK;
@@ -866,7 +876,7 @@ int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, co
                 constexpr bool VEC = decltype(vec)::value;
                 allow_smem(relay_kernel<K, EMAX, XMODE, VEC>, Tile<K, EMAX>::SMEM);
                 launch_kernel(dependent_launches(), relay_kernel<K, EMAX, XMODE, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop, xop_next,
-                              static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bo, ext.Bho, total);
+                              static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bo, ext.Bho, total, (int)(dependent_launches() == PDL_LATE));
             };
             if (xmode == 1) launch(std::integral_constant<int, 1>{}, std::true_type{});
             else if ((p % 4) == 0) launch(std::integral_constant<int, 0>{}, std::true_type{});

@@ -54,6 +54,9 @@ struct TcArgs {
     int nacc;                // accumulators in tensor memory (2 .. kMaxAcc)
     long tiles;              // output tiles in total; CTAs walk them with a grid stride
     long cols_out;           // V * Ho * Wo
+    uint32_t spin_limit;     // polls before a wait gives up (kSpinLimit; a few thousand under fault injection)
+    int pdl_late;            // issue the dependent-launch trigger after the CTA's last tile instead of first thing
+    int no_copy;             // fault injection (tests only): the producer announces its bytes but issues no copy
 };
 
 // ---- PTX wrappers ------------------------------------------------------------------------------
@@ -77,8 +80,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
         if (it > 64) __nanosleep(64);
@@ -287,7 +290,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
-    pdl_trigger();
+    if (!g.pdl_late) pdl_trigger();
     pdl_wait();     // X is written by the transform kernel before this one; Y may still be read by an earlier one
 
     if (warp == 0) {
@@ -309,11 +312,16 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 // one iteration = one K block: input tile (hi [, lo]) and all taps' weight tiles (hi [, lo])
                 {
                     for (int kb = 0; kb < kblocks; ++kb) {
-                        if (wrapped) ok = mbar_wait(&empty_bar[s], par ^ 1u, &abort_flag);
+                        if (wrapped) ok = mbar_wait(&empty_bar[s], par ^ 1u, &abort_flag, g.spin_limit);
                         if (!ok) break;
                         unsigned char* xs = ring + (size_t)s * stage_bytes;
                         unsigned char* as = xs + (size_t)g.nsplit * x_bytes;
                         mbar_expect_tx(&full_bar[s], tx_bytes);
+                        if (g.no_copy) {                 // fault injection: nothing is in flight, the consumer's wait runs out
+                            ok = false;
+                            issued = 0;
+                            break;
+                        }
                         // input tile with its halo: starts pad pixels before the output tile (negative and
                         // out-of-image coordinates read the zero fill)
                         tma_load_5d(xs, map_xhi, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v, t.prob_in_kind);
@@ -342,7 +350,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                         dpar ^= 1u;
                     }
                     --ds;
-                    for (uint32_t spin = 0; spin < kSpinLimit && !mbar_try_wait(&full_bar[ds], dpar); ++spin) __nanosleep(64);
+                    for (uint32_t spin = 0; spin < g.spin_limit && !mbar_try_wait(&full_bar[ds], dpar); ++spin) __nanosleep(64);
                 }
             }
         }
@@ -360,14 +368,14 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 const uint32_t a_bytes = (uint32_t)t.bn * 128;
                 const uint32_t idesc = instr_desc(t.bn);
                 const int kblocks = (t.Kq + kKBlock - 1) / kKBlock;
-                if (acc_wrapped) ok = mbar_wait(&acc_empty[buf], acc_par ^ 1u, &abort_flag);   // epilogue done with it
+                if (acc_wrapped) ok = mbar_wait(&acc_empty[buf], acc_par ^ 1u, &abort_flag, g.spin_limit);   // epilogue done with it
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * acc_cols;
                 uint32_t accumulate = 0;
                 {
                     for (int kb = 0; kb < kblocks; ++kb) {
-                        ok = mbar_wait(&full_bar[s], par, &abort_flag);
+                        ok = mbar_wait(&full_bar[s], par, &abort_flag, g.spin_limit);
                         if (!ok) break;
                         tc_fence_after();
                         const uint32_t xs = smem_u32(ring + (size_t)s * stage_bytes);
@@ -461,7 +469,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
         uint32_t acc_par = 0;
         for (long tile = blockIdx.x; tile < g.tiles; tile += gridDim.x) {
             const TileCoord t = decode_tile(g, tile);
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], acc_par, &abort_flag));  // warp-uniform
+            const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], acc_par, &abort_flag, g.spin_limit));  // warp-uniform
             if (!ok) break;
             tc_fence_after();
             const size_t y_real = (size_t)g.cols_out * g.p;
@@ -516,6 +524,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     }
 
     // ---- teardown ---------------------------------------------------------------------------------
+    if (g.pdl_late) pdl_trigger();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -614,6 +623,8 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
         return CIRC_ERR_SHAPE;
     }
     g.tiles = ctas;
+    g.pdl_late = dependent_launches() == PDL_LATE;
+    if (g.no_copy) g.spin_limit = 1u << 12;
     const unsigned grid = (unsigned)(ctas < 148 * ctas_per_sm ? ctas : 148 * ctas_per_sm);
     launch_kernel(dependent_launches(), contract_tc_kernel, dim3(grid), dim3(kTcThreads), smem, stream, maps[0], maps[1], maps[2], maps[3], maps[4],
                   maps[5], g);
@@ -631,6 +642,8 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     g.p = p; g.q = q; g.k = k; g.taps = taps; g.r = geo.r; g.pad = geo.pad;
     g.nsplit = nsplit;
     g.npass = nsplit == 2 ? 3 : 1;
+    g.spin_limit = kSpinLimit;
+    g.no_copy = L->inject == INJECT_TENSOR_NO_COPY;
     if (L->kind == 1) {
         g.W = ext.W; g.H = ext.H; g.V = 2 * ext.Nh; g.Wo = ext.Wo; g.Ho = ext.Ho;
     } else {
@@ -733,6 +746,8 @@ static int launch_tc_one_kind(bool real, const __nv_bfloat16* xt, int x_rows, co
     g.taps = 1; g.r = 1; g.pad = 0;
     g.nsplit = 2;
     g.npass = 3;
+    g.spin_limit = kSpinLimit;
+    g.no_copy = 0;
     g.W = g.Wo = x_rows; g.H = g.Ho = 1; g.V = 1;
     g.tw = x_rows < kTileCols ? x_rows : kTileCols;
     g.pitch = g.tw;

@@ -23,8 +23,8 @@ def to_device(a: np.ndarray, bf16: bool) -> torch.Tensor:
     return t.to(torch.bfloat16) if bf16 else t
 
 
-def run_fc(case: synth.FcCase, variant=circ.CIRC_VARIANT_AUTO, convention=0, y_bf16=None, stream=None):
-    """Returns (y as float64 numpy [B][m], variant used)."""
+def run_fc(case: synth.FcCase, variant=circ.CIRC_VARIANT_AUTO, convention=0, y_bf16=None, stream=None, kernels=None):
+    """Returns (y as float64 numpy [B][m], variant used); ``kernels``: a list that receives the S1 / S2 / S3 kernel ids."""
     y_bf16 = case.bf16_io if y_bf16 is None else y_bf16
     h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
     try:
@@ -42,6 +42,8 @@ def run_fc(case: synth.FcCase, variant=circ.CIRC_VARIANT_AUTO, convention=0, y_b
         torch.cuda.synchronize()
         circ.circ_device_status(h)
         used = circ.circ_last_variant(h)
+        if kernels is not None:
+            kernels.extend(circ.circ_debug_last_kernels(h))
         return y.float().cpu().numpy().astype(np.float64), used
     finally:
         circ.circ_destroy(h)

@@ -69,7 +69,7 @@ def test_reserve_then_forward_allocates_nothing():
 
 
 @pytest.mark.parametrize("variant,batch", [(circ.CIRC_VARIANT_FUSED, 4), (circ.CIRC_VARIANT_TENSOR, 48), (circ.CIRC_VARIANT_STAGED, 48)])
-def test_stage_repeat_and_profile_leave_results_unchanged(variant, batch):
+def test_repeated_stage_leaves_results_unchanged(variant, batch):
     case = synth.fc_case(f"repeat_{variant}", 512, 512, 64, batch, w_var=1.0 / 512, x_dist="normal", bias_var=0.01, relu=True)
     h = _fc_handle(case)
     try:
@@ -78,24 +78,46 @@ def test_stage_repeat_and_profile_leave_results_unchanged(variant, batch):
         y0 = torch.empty(batch, case.m, device="cuda")
         y1 = torch.empty(batch, case.m, device="cuda")
         s = torch.cuda.current_stream()
-        l0 = circ.circ_launch_count()
+        l0 = circ.circ_debug_launch_count()
         circ.circ_fc_forward(h, x, y0, batch, s)
-        per_forward = circ.circ_launch_count() - l0
+        per_forward = circ.circ_debug_launch_count() - l0
         assert per_forward == (1 if variant == circ.CIRC_VARIANT_FUSED else 3)
-        stages = [3] if variant == circ.CIRC_VARIANT_FUSED else [0, 1, 2]
+        stages = [circ.CIRC_STAGE_FUSED] if variant == circ.CIRC_VARIANT_FUSED else [0, 1, 2]
         for st in stages:
-            circ.circ_set_stage_repeat(h, st, 3)
-        circ.circ_profile_begin(h)
-        l0 = circ.circ_launch_count()
-        circ.circ_fc_forward(h, x, y1, batch, s)
-        assert circ.circ_launch_count() - l0 == 3 * per_forward
-        ms, cnt = circ.circ_profile_end(h)
-        torch.cuda.synchronize()
-        assert [c > 0 for c in cnt] == [i in stages for i in range(4)] and all(m >= 0 for m in ms)
-        assert torch.equal(y0, y1)                                   # bitwise: every kernel rewrites the same values
+            l0 = circ.circ_debug_launch_count()
+            circ.circ_debug_forward_repeat(h, x, y1, batch, 1, 1, st, 3, s)
+            assert circ.circ_debug_launch_count() - l0 == per_forward + 2
+            torch.cuda.synchronize()
+            assert torch.equal(y0, y1)                               # bitwise: every kernel rewrites the same values
         assert scale_rel_err(y1.cpu().numpy().astype(np.float64), oracle_fc(case)) <= TOL_F32
         with pytest.raises(circ.CircError):
-            circ.circ_set_stage_repeat(h, 7, 2)
+            circ.circ_debug_forward_repeat(h, x, y1, batch, 1, 1, 7, 2, s)
+        if variant != circ.CIRC_VARIANT_FUSED:
+            want = circ.CIRC_KERNEL_S2_TENSOR if variant == circ.CIRC_VARIANT_TENSOR else circ.CIRC_KERNEL_S2_FMA
+            assert circ.circ_debug_last_kernels(h)[1] == want
+    finally:
+        circ.circ_destroy(h)
+
+
+def test_growing_the_workspace_inside_a_capture_is_refused_up_front():
+    case = synth.fc_case("capture_grow", 256, 256, 16, 64, w_var=1.0 / 256, x_dist="uniform")
+    h = _fc_handle(case)
+    try:
+        x = torch.from_numpy(case.x).cuda()
+        y = torch.empty(64, 256, device="cuda")
+        side = torch.cuda.Stream()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            with pytest.raises(circ.CircError) as e:
+                circ.circ_fc_forward(h, x, y, 64, torch.cuda.current_stream())      # no workspace yet
+            assert e.value.code == circ.CIRC_ERR_UNSUPPORTED
+        circ.circ_reserve(h, 64)
+        g2 = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g2, stream=side):
+            circ.circ_fc_forward(h, x, y, 64, torch.cuda.current_stream())
+        g2.replay()
+        torch.cuda.synchronize()
+        assert scale_rel_err(y.cpu().numpy().astype(np.float64), oracle_fc(case)) <= TOL_F32
     finally:
         circ.circ_destroy(h)
 

@@ -44,6 +44,53 @@ def test_traffic_is_withheld_when_the_kernel_changed(monkeypatch):
     assert bench.traffic_if_current("other", "fused_fc") is None
 
 
+def test_graph_plan_times_exactly_the_requested_steps():
+    for steps in (1, 20, 256, 257, 300, 2000, 20000, 1009):
+        g, replays, rem = bench.graph_plan(steps)
+        assert g * replays + rem == steps and 1 <= g <= 256 and 0 <= rem < g
+
+
+def test_rotation_covers_twice_the_l2():
+    assert bench.sets_needed(403_000_000, 96) == 2
+    assert bench.sets_needed(9_453_568, 96) * 9_453_568 >= 2 * bench.L2_BYTES
+    assert bench.sets_needed(18_000, 96) == 96                       # capped: the flush between repeats covers the rest
+
+
+def test_table_lists_every_named_configuration_and_the_sweep_corners():
+    rows = bench.TABLE_ROWS
+    assert len(rows) >= 20 and len(set(rows)) == len(rows)
+    for must in ("cfg1", "cfg2_b1", "cfg2_b16", "cfg2_b256", "cfg3_stack", "cfg4", "sweep_n16384_k4_b1", "sweep_n16384_k256_b1024_bf16"):
+        assert must in rows
+    assert bench.HEADLINE == "sweep_n16384_k4_b1024"
+
+
+def test_whole_forward_fraction_rule():
+    class Ids:
+        CIRC_VARIANT_FUSED, CIRC_VARIANT_STAGED, CIRC_VARIANT_TENSOR = 1, 2, 3
+    peaks = {"hbm_gbs": 6500.0, "bf16_tflops": 1400.0, "source": "test"}
+    w = bench.workload("cfg2_b256")
+    # tensor path, HBM-bound by the rule: fraction = t_hbm / t
+    t_hbm_us = w.alg_bytes / 6500e9 * 1e6
+    r = bench.bound_and_fraction(w, 3, 10.0, peaks, 70.0, Ids)
+    assert r["bound"] == "hbm" and abs(r["frac"] - t_hbm_us / 10.0) < 1e-9
+    assert abs(r["achieved"] - w.alg_bytes / 10e-6 / 1e9) < 1e-6 and r["peak"] == 6500.0
+    # the same layer on the FMA pipes is bound by float32 arithmetic
+    r = bench.bound_and_fraction(w, 2, 10.0, peaks, 70.0, Ids)
+    assert r["bound"] == "alu" and r["t_alu_us"] > r["t_hbm_us"]
+    # float32 inputs take three bfloat16 products: a third of the tensor peak
+    big = bench.Workload("x", "", "fc", w.case, 1024, 403_000_000, 5.5e14, 4, 4, 2.06e11, 1e9)
+    r = bench.bound_and_fraction(big, 3, 500.0, peaks, 70.0, Ids)
+    assert r["bound"] == "tensor" and abs(r["peak"] - 1400.0 / 3) < 1e-9
+    assert abs(r["frac"] - (2.06e11 / (1400e12 / 3)) / 500e-6) < 1e-9
+
+
+def test_gpus_flag_must_match_the_launch(monkeypatch):
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    monkeypatch.setenv("RANK", "0")
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4"])
+    assert bench.main() == 2                                         # --gpus 4 inside a 2-rank launch: refused
+
+
 def _rank_main(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)

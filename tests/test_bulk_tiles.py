@@ -12,8 +12,9 @@ from gpu_helpers import TOL_BF16, TOL_F32, run_fc, scale_rel_err
 pytestmark = pytest.mark.gpu
 
 
-def _check(case, tol):
-    got, used = run_fc(case)
+def _check(case, tol, want_s3):
+    got, used = run_fc(case, kernels=(kernels := []))
+    assert kernels[2] == want_s3, kernels          # the inverse-transform kernel under test really served the call
     assert not np.isnan(got).any()
     B = case.batch
     half = (B + 1) // 2
@@ -32,20 +33,20 @@ def _check(case, tol):
 def test_bulk_tiles_float32(k, p, q, batch):
     case = synth.fc_case(f"bulk_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
                          bias_var=0.01, relu=True)
-    used = _check(case, TOL_F32)
+    used = _check(case, TOL_F32, circ.CIRC_KERNEL_S3_BULK)
     assert used == (circ.CIRC_VARIANT_TENSOR if q % 8 == 0 else circ.CIRC_VARIANT_STAGED)
 
 
 def test_bulk_tiles_bfloat16():
     case = synth.fc_case("bulk_bf16", 16 * 64, 8 * 64, 64, 6002, w_var=1.0 / 512, x_dist="uniform", bias_var=0.01, relu=True,
                          bf16_io=True)
-    _check(case, TOL_BF16)
+    _check(case, TOL_BF16, circ.CIRC_KERNEL_S3_BULK)
 
 
 def test_odd_transform_count_falls_back():
     # 3001 pairs x 15 row blocks = 45015 transforms: the runs of Y are not 16-byte aligned, the load-based kernel runs
     case = synth.fc_case("bulk_odd", 15 * 64, 8 * 64, 64, 6001, w_var=1.0 / 512, x_dist="normal", bias_var=0.01, relu=True)
-    _check(case, TOL_F32)
+    _check(case, TOL_F32, circ.CIRC_KERNEL_S3_LOADS)
 
 
 def test_repeatable_bitwise_large():
