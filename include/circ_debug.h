@@ -32,7 +32,8 @@ enum {
     CIRC_KERNEL_S2_FMA = 10,    /* contraction on the float32 FMA pipes */
     CIRC_KERNEL_S2_TENSOR = 11, /* contraction on the tensor cores */
     CIRC_KERNEL_S3_LOADS = 20,  /* inverse transforms fed by per-thread loads */
-    CIRC_KERNEL_S3_BULK = 21    /* inverse transforms fed by bulk asynchronous copies */
+    CIRC_KERNEL_S3_BULK = 21,   /* inverse transforms fed by bulk asynchronous copies */
+    CIRC_KERNEL_S4_FUSED = 30   /* the one-launch small-batch kernel */
 };
 
 /* Fault injection kinds of circ_debug_inject. */
@@ -54,7 +55,8 @@ CIRC_API int circ_debug_forward_repeat(circ_handle h, const void* x, void* y, in
                                        void* stream);
 
 /* circ_debug_last_kernels -- ids[0..2] = which S1 / S2 / S3 kernel (CIRC_KERNEL_*) the most recent staged
- * forward of this handle launched (HOST pointer to three ints). */
+ * forward of this handle launched (HOST pointer to three ints).  After a one-launch forward:
+ * ids = { CIRC_KERNEL_S4_FUSED, column slices (thread blocks per cluster), row blocks per thread block }. */
 CIRC_API int circ_debug_last_kernels(circ_handle h, int* ids);
 
 /* circ_debug_launch_count -- kernels this library has launched in this process so far. */
@@ -82,6 +84,10 @@ CIRC_API int circ_debug_empty_kernel(void* stream);
  * The outputs of such a forward are invalid.  CIRC_INJECT_NONE restores normal operation.
  */
 CIRC_API int circ_debug_inject(circ_handle h, int kind);
+
+/* circ_debug_set_fused_split -- force the one-launch kernel to split the layer's columns over `slices` thread
+ * blocks per cluster (1, 2, 4 or 8; must divide q); 0 restores the planner's choice.  For tests and tuning. */
+CIRC_API int circ_debug_set_fused_split(circ_handle h, int slices);
 
 /* circ_debug_fail_alloc_after -- the n-th device allocation the library makes from now on fails as if the
  * device were out of memory (n = 1: the next one); n <= 0 cancels.  Exercises the CIRC_ERR_ALLOC paths. */

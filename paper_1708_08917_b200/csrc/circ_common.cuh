@@ -98,6 +98,7 @@ struct Layer {
     size_t x_stage_bytes, y_stage_bytes;
     mutable int last_kernels[3];  // which S1 / S2 / S3 kernel served the most recent staged forward (KERNEL_* ids below)
     int inject;           // test-only fault injection (circ_debug.h): 0 = none
+    int fused_split;      // column slices of the one-launch kernel forced by circ_debug_set_fused_split (0 = planner's choice)
     Layer* transposed;  // the n x m layer W^T (built on first use by the backward pass), or nullptr
 };
 
@@ -109,7 +110,8 @@ enum {
     KERNEL_S2_FMA = 10,       // contraction on the float32 FMA pipes
     KERNEL_S2_TENSOR = 11,    // contraction on the tensor cores
     KERNEL_S3_LOADS = 20,     // inverse transforms, per-thread loads
-    KERNEL_S3_BULK = 21       // inverse transforms, tiles staged by bulk asynchronous copies
+    KERNEL_S3_BULK = 21,      // inverse transforms, tiles staged by bulk asynchronous copies
+    KERNEL_S4_FUSED = 30      // the one-launch kernel: last_kernels = {this id, column slices, row blocks per thread block}
 };
 
 // Test-only fault injection (circ_debug_inject): the named producer issues no copy and every bounded wait of that

@@ -7,7 +7,8 @@ namespace circ {
 
 static_assert((int)CIRC_KERNEL_S1_LOADS == (int)KERNEL_S1_LOADS && (int)CIRC_KERNEL_S1_BULK == (int)KERNEL_S1_BULK &&
                   (int)CIRC_KERNEL_S2_FMA == (int)KERNEL_S2_FMA && (int)CIRC_KERNEL_S2_TENSOR == (int)KERNEL_S2_TENSOR &&
-                  (int)CIRC_KERNEL_S3_LOADS == (int)KERNEL_S3_LOADS && (int)CIRC_KERNEL_S3_BULK == (int)KERNEL_S3_BULK,
+                  (int)CIRC_KERNEL_S3_LOADS == (int)KERNEL_S3_LOADS && (int)CIRC_KERNEL_S3_BULK == (int)KERNEL_S3_BULK &&
+                  (int)CIRC_KERNEL_S4_FUSED == (int)KERNEL_S4_FUSED,
               "public and internal kernel ids must agree");
 static_assert((int)CIRC_INJECT_TENSOR_NO_COPY == (int)INJECT_TENSOR_NO_COPY && (int)CIRC_INJECT_BULK_NO_COPY == (int)INJECT_BULK_NO_COPY,
               "public and internal injection kinds must agree");
@@ -126,6 +127,16 @@ int circ_debug_inject(circ_handle h, int kind) {
         return CIRC_ERR_ARG;
     }
     L->inject = kind;
+    return CIRC_OK;
+}
+
+int circ_debug_set_fused_split(circ_handle h, int slices) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (slices != 0 && slices != 1 && slices != 2 && slices != 4 && slices != 8) || (slices > 0 && L->geo.q % slices)) {
+        set_error(CIRC_ERR_ARG, "bad handle, or slices=%d is not 0, 1, 2, 4 or 8 or does not divide q", slices);
+        return CIRC_ERR_ARG;
+    }
+    L->fused_split = slices;
     return CIRC_OK;
 }
 

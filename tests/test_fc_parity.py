@@ -49,6 +49,53 @@ def test_convention_flag(variant):
     assert scale_rel_err(g0, oracle_fc(case, 1)) > 1e-2     # the flag is observable
 
 
+def _run_fused_split(case, slices):
+    import torch
+    from gpu_helpers import to_device
+    h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
+    try:
+        circ.circ_set_bias(h, case.bias)
+        circ.circ_set_activation(h, 1)
+        code = circ.CIRC_BF16 if case.bf16_io else circ.CIRC_F32
+        circ.circ_set_io_dtype(h, code, code)
+        circ.circ_set_variant(h, circ.CIRC_VARIANT_FUSED)
+        circ.circ_debug_set_fused_split(h, slices)
+        x = to_device(case.x, case.bf16_io)
+        y = torch.full((case.batch, case.m), float("nan"), device="cuda", dtype=torch.bfloat16 if case.bf16_io else torch.float32)
+        circ.circ_fc_forward(h, x, y, case.batch)
+        torch.cuda.synchronize()
+        return y.float().cpu().numpy().astype(np.float64), circ.circ_debug_last_kernels(h)
+    finally:
+        circ.circ_destroy(h)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("k,p,q,batch", [(64, 4, 64, 1), (256, 2, 16, 3), (16, 8, 128, 8), (4, 16, 1024, 5), (128, 64, 8, 2),
+                                         (32, 300, 24, 7), (256, 64, 64, 1), (64, 256, 256, 2), (8, 3, 40, 4)])
+def test_one_launch_kernel_with_split_columns(k, p, q, batch, bf16):
+    # the columns split over the 1, 2, 4 or 8 thread blocks of a cluster, partial spectra added up through distributed
+    # shared memory: odd row counts, all pair counts, both storage types, bias + ReLU, every split that divides q
+    case = synth.fc_case(f"split_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
+                         bias_var=0.01, relu=True, bf16_io=bf16)
+    ref = oracle_fc(case)
+    for slices in (1, 2, 4, 8):
+        if q % slices:
+            continue
+        got, kernels = _run_fused_split(case, slices)
+        assert kernels[0] == circ.CIRC_KERNEL_S4_FUSED and kernels[1] == slices
+        assert not np.isnan(got).any()
+        assert scale_rel_err(got, ref) <= (TOL_BF16 if bf16 else TOL_F32)
+        again, _ = _run_fused_split(case, slices)
+        assert np.array_equal(got, again)         # fixed-order sums: bitwise repeatable
+
+
+def test_one_launch_planner_splits_wide_layers_with_few_rows():
+    case = synth.fc_case("split_plan", 16384, 16384, 256, 1, w_var=1.0 / 16384, x_dist="uniform")
+    kernels = []
+    run_fc(case, circ.CIRC_VARIANT_FUSED, kernels=kernels)
+    assert kernels[0] == circ.CIRC_KERNEL_S4_FUSED and kernels[1] > 1 and kernels[1] * -(-64 // kernels[2]) >= 100, kernels
+
+
 def test_config1():
     case = synth.config1()
     got, _ = run_fc(case)
