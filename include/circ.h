@@ -142,11 +142,17 @@ CIRC_API int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_h
  * library; every GPU context that loads the library holds that array until it exits.
  *
  *   h, x, y, batch, stream : exactly as circ_fc_forward (x, y DEVICE pointers owned by the caller).
- *   Limit: 4 * (2 * ceil(batch / 2)) * (n + m) bytes (+ alignment) must fit in the array; larger
- *          requests fail with CIRC_ERR_SHAPE and a message that names both numbers.
- *          circ_noalloc_max_bytes() returns the array size.
- *   The first call on each device looks up the array's device address (cudaGetSymbolAddress);
- *   make that first call outside any stream capture.
+ *   Preparation, while allocation is still allowed: the staged path reads a stored form of the spectra that a handle
+ *          builds (allocates) the first time it is needed.  Call circ_set_variant(h, CIRC_VARIANT_STAGED) and
+ *          circ_reserve(h, batch) once, or run one circ_fc_forward on that path; this also loads the scratch
+ *          array (that is when its bytes are taken from the device) and looks up its address.  Without it this
+ *          call fails with CIRC_ERR_UNSUPPORTED rather than allocate.
+ *   Limit: 4 * (2 * ceil(batch / 2)) * (p + q) * kt bytes (+ alignment) must fit in the array, kt being the
+ *          transform size: k itself for powers of two in [4, 1024], else the smallest power of two >= 2k - 1
+ *          (so (p + q) * kt = n + m for power-of-two blocks).  Larger requests fail with CIRC_ERR_SHAPE and a
+ *          message that names both numbers.  circ_noalloc_max_bytes() returns the array size.
+ *   If no preparation ran on the device, the first call looks up the array's device address
+ *   (cudaGetSymbolAddress); make that first call outside any stream capture.
  *   All calls, on all handles and streams, share the one array and leave their intermediate
  *   results in it: two calls whose kernels overlap on the GPU race and corrupt each other, so
  *   issue them on one stream or order them yourself.  Nothing in the array needs clearing between

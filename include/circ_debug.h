@@ -30,7 +30,10 @@ enum {
     CIRC_KERNEL_S1_LOADS = 1,   /* input transforms fed by per-thread vector loads */
     CIRC_KERNEL_S1_BULK = 2,    /* input transforms fed by bulk asynchronous copies into shared memory */
     CIRC_KERNEL_S2_FMA = 10,    /* contraction on the float32 FMA pipes */
-    CIRC_KERNEL_S2_TENSOR = 11, /* contraction on the tensor cores */
+    CIRC_KERNEL_S2_TENSOR = 11, /* contraction on the tensor cores, weights in the embedded real form [Wr -Wi; Wi Wr] */
+    CIRC_KERNEL_S2_TENSOR_TWIN = 12, /* contraction on the tensor cores, every complex weight stored once (twin column groups of X) */
+    CIRC_KERNEL_S2_ROWS = 13,   /* row-streaming tensor-core contraction (few columns, many row blocks), embedded weights */
+    CIRC_KERNEL_S2_ROWS_TWIN = 14, /* row-streaming tensor-core contraction with twin columns */
     CIRC_KERNEL_S3_LOADS = 20,  /* inverse transforms fed by per-thread loads */
     CIRC_KERNEL_S3_BULK = 21,   /* inverse transforms fed by bulk asynchronous copies */
     CIRC_KERNEL_S4_FUSED = 30   /* the one-launch small-batch kernel */
@@ -88,6 +91,11 @@ CIRC_API int circ_debug_inject(circ_handle h, int kind);
 /* circ_debug_set_fused_split -- force the one-launch kernel to split the layer's columns over `slices` thread
  * blocks per cluster (1, 2, 4 or 8; must divide q); 0 restores the planner's choice.  For tests and tuning. */
 CIRC_API int circ_debug_set_fused_split(circ_handle h, int slices);
+
+/* circ_debug_set_contraction -- restrict the planner's choices for the tensor-core contraction of this handle, for
+ * tests and tuning that compare the forms on one shape.  allow_twin = 0: never the twin-column form (every complex
+ * weight stored once, X twice); allow_rows = 0: never the row-streaming kernel.  1 / 1 (default): the planner decides. */
+CIRC_API int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows);
 
 /* circ_debug_fail_alloc_after -- the n-th device allocation the library makes from now on fails as if the
  * device were out of memory (n = 1: the next one); n <= 0 cancels.  Exercises the CIRC_ERR_ALLOC paths. */

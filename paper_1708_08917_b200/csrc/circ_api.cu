@@ -74,6 +74,7 @@ void free_layer(Layer* L) {
     cudaFree(L->w_stream_bf16);
     cudaFree(L->a_f32);
     cudaFree(L->a_bf16);
+    cudaFree(L->a_twin);
     cudaFree(L->ws);
     cudaFree(L->dev_status);
     cudaFree(L->x_stage);
@@ -127,10 +128,9 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
     }
     const size_t a_real = (size_t)taps * (m / k) * (n / k);
     L->a_elems = 2 * a_real + (size_t)(kt / 2 - 1) * 4 * a_real;
-    bool ok = dev_alloc(&L->a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess &&
-              dev_alloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess &&
-              dev_alloc(&L->a_f32, L->a_elems * sizeof(float)) == cudaSuccess &&
-              dev_alloc(&L->dev_status, sizeof(int)) == cudaSuccess;
+    // Only the packed spectra are made now (the paper's storage figure, m n / k values); the operand layouts of the
+    // staged contractions are re-arrangements of them, built when a forward first takes that path.
+    bool ok = dev_alloc(&L->w_stream, wcount * sizeof(float)) == cudaSuccess && dev_alloc(&L->dev_status, sizeof(int)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         set_error(CIRC_ERR_ALLOC, "device allocation of the weight spectra failed");
@@ -143,12 +143,61 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
         free_layer(L);
         return nullptr;
     }
+    if (!embedded(L->geo)) {   // a power-of-two block's defining vectors can be recovered from its spectra
+        cudaFree(L->w_dev);
+        L->w_dev = nullptr;
+    }
     return L;
 }
 
+int ensure_forms(Layer* L, unsigned forms, cudaStream_t stream) {
+    const bool need_f32 = (forms & FORM_A_F32) && !L->a_f32, need_bf16 = (forms & FORM_A_BF16) && !L->a_bf16,
+               need_twin = (forms & FORM_A_TWIN) && !L->a_twin;
+    if (!need_f32 && !need_bf16 && !need_twin) return CIRC_OK;
+    if (stream_is_capturing(stream)) {
+        set_error(CIRC_ERR_UNSUPPORTED, "this forward needs a stored form of the spectra that has not been built yet, and the stream "
+                  "is being captured: call circ_reserve (or run one forward of this size) before the capture");
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    float* a_f32 = nullptr;
+    __nv_bfloat16 *a_bf16 = nullptr, *a_twin = nullptr;
+    bool ok = true;
+    if (need_f32) ok = ok && dev_alloc(&a_f32, L->a_elems * sizeof(float)) == cudaSuccess;
+    if (need_bf16) ok = ok && dev_alloc(&a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess;
+    if (need_twin) ok = ok && dev_alloc(&a_twin, twin_elems(L) * sizeof(__nv_bfloat16) + 256) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(a_f32);
+        cudaFree(a_bf16);
+        cudaFree(a_twin);
+        set_error(CIRC_ERR_ALLOC, "device allocation of a stored form of the spectra failed");
+        return CIRC_ERR_ALLOC;
+    }
+    // on the caller's stream: ordered before the forward that is about to read the new layout
+    const int rc = launch_spectrum_forms(L, a_f32, a_bf16, a_twin, stream);
+    if (a_f32) {
+        L->a_f32 = a_f32;
+        if (L->kind == 0) noalloc_warm();   // the allocation-free forward reads this form: have its scratch array resident too
+    }
+    if (a_bf16) L->a_bf16 = a_bf16;
+    if (a_twin) L->a_twin = a_twin;
+    return rc;
+}
+
+static size_t x_operand_floats(const Layer* L, const Extent& e) {
+    const size_t xin = (size_t)2 * e.Bh * L->geo.q * L->geo.k;   // all problems of X
+    return (use_twin(L, e) ? 2 * xin : xin);                     // twin columns: the complex problems twice
+}
+
+// Copies of Y: the row-streaming contraction writes one per piece of its contraction range.
+static size_t y_copies(const Layer* L, const Extent& e) {
+    const ContractionPlan pl = plan_contraction(L, e);
+    return pl.rows ? (size_t)rows_pieces(L, pl.twin).cplx : 1;
+}
+
 static size_t workspace_need(const Layer* L, const Extent& e) {
-    const size_t xin = (size_t)2 * e.Bh * L->geo.q * L->geo.k;   // floats: all problems of X
-    const size_t yout = (size_t)2 * e.Bho * L->geo.p * L->geo.k; // floats: all problems of Y
+    const size_t xin = x_operand_floats(L, e);                   // floats: all problems of X
+    const size_t yout = (size_t)2 * e.Bho * L->geo.p * L->geo.k * y_copies(L, e); // floats: all problems of Y (and its copies)
     return (xin + yout) * sizeof(float) + 512;
 }
 
@@ -229,7 +278,7 @@ int staged_operands(Layer* L, const Extent& e, cudaStream_t stream, float** xop,
     const int rc = ensure_workspace(L, need);
     if (rc != CIRC_OK) return rc;
     *xop = static_cast<float*>(L->ws);
-    *yop = *xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
+    *yop = *xop + ((x_operand_floats(L, e) + 63) & ~(size_t)63);
     return CIRC_OK;
 }
 
@@ -239,36 +288,48 @@ int staged_dependent_launches(const Layer* L, const Extent& e) {
     return (long)e.Bh * (L->geo.p > L->geo.q ? L->geo.p : L->geo.q) * L->geo.k <= 32768 ? PDL_EARLY : PDL_LATE;
 }
 
+int prepare_staged(Layer* L, const Extent& e, cudaStream_t stream, bool tensor) {
+    return ensure_forms(L, !tensor ? FORM_A_F32 : use_twin(L, e) ? FORM_A_TWIN : FORM_A_BF16, stream);
+}
+
 int stage_input(Layer* L, const void* x, float* xop, const Extent& e, cudaStream_t stream, bool tensor) {
     // tensor path: bfloat16 operands, split hi/lo unless the input itself is bfloat16
     const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
-    return launch_input_fft(L, x, xop, xmode, e, stream);
+    return launch_input_fft(L, x, xop, xmode, e, stream, tensor && use_twin(L, e));
 }
 
 int stage_contract(Layer* L, const float* xop, float* yop, const Extent& e, cudaStream_t stream, bool tensor) {
     if (tensor) {
-        L->last_kernels[1] = KERNEL_S2_TENSOR;
-        return launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, L->x_dtype == CIRC_BF16 ? 1 : 2, stream);
+        const ContractionPlan pl = plan_contraction(L, e);
+        const int nsplit = L->x_dtype == CIRC_BF16 ? 1 : 2;
+        if (pl.rows) {
+            L->last_kernels[1] = pl.twin ? KERNEL_S2_ROWS_TWIN : KERNEL_S2_ROWS;
+            return launch_contract_rows(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, nsplit, stream, pl.twin);
+        }
+        L->last_kernels[1] = pl.twin ? KERNEL_S2_TENSOR_TWIN : KERNEL_S2_TENSOR;
+        return launch_contract_tc(L, reinterpret_cast<const __nv_bfloat16*>(xop), yop, e, nsplit, stream, pl.twin);
     }
     L->last_kernels[1] = KERNEL_S2_FMA;
     return launch_contract_fma(L, xop, yop, e, stream);
 }
 
-int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream) {
-    return launch_output_ifft(L, yop, y, e, stream);
+int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
+    const ContractionPlan pl = tensor ? plan_contraction(L, e) : ContractionPlan{false, false};
+    return launch_output_ifft(L, yop, y, e, stream, false, pl.twin, pl.rows ? rows_pieces(L, pl.twin) : RowsPieces{0, 0});
 }
 
 static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
     float *xop = nullptr, *yop = nullptr;
     int rc = staged_operands(L, e, stream, &xop, &yop);
     if (rc != CIRC_OK) return rc;
+    if ((rc = prepare_staged(L, e, stream, tensor)) != CIRC_OK) return rc;
     struct DependentGuard {   // reset on every exit path
         DependentGuard(int mode) { dependent_launches() = mode; }
         ~DependentGuard() { dependent_launches() = PDL_OFF; }
     } guard(staged_dependent_launches(L, e));
     if ((rc = stage_input(L, x, xop, e, stream, tensor)) != CIRC_OK) return rc;
     if ((rc = stage_contract(L, xop, yop, e, stream, tensor)) != CIRC_OK) return rc;
-    if ((rc = stage_output(L, yop, y, e, stream)) != CIRC_OK) return rc;
+    if ((rc = stage_output(L, yop, y, e, stream, tensor)) != CIRC_OK) return rc;
     L->last_variant = tensor ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
     return CIRC_OK;
 }
@@ -483,7 +544,9 @@ int circ_set_convention(circ_handle h, int convention) {
         free_layer(L->transposed);   // rebuilt on the next backward call
         L->transposed = nullptr;
     }
-    int rc = launch_precompute(L, 0);
+    // a power-of-two block changes convention by conjugating its spectra; an embedded one is recomputed from its vectors
+    int rc = embedded(L->geo) ? launch_precompute(L, 0) : launch_conjugate_stream(L, 0);
+    if (rc == CIRC_OK && !embedded(L->geo)) rc = launch_spectrum_forms(L, L->a_f32, L->a_bf16, L->a_twin, 0);
     if (rc != CIRC_OK) return rc;
     CIRC_CUDA_TRY(cudaDeviceSynchronize(), CIRC_ERR_CUDA);
     return CIRC_OK;
@@ -532,7 +595,28 @@ int circ_reserve(circ_handle h, long max_batch) {
     // covered by sizing for max_batch pairs on each side.
     Extent e;
     e.Bh = e.Bho = (int)max_batch;
-    return ensure_workspace(L, workspace_need(L, e));
+    const size_t plain = ((size_t)2 * e.Bh * L->geo.q * L->geo.k + (size_t)2 * e.Bho * L->geo.p * L->geo.k) * sizeof(float) + 512;
+    size_t need = plain;
+    if (L->kind == 0 && max_batch <= (1L << 30) / 2) {       // what a forward of exactly this size takes (twin columns, copies of Y)
+        const size_t exact = workspace_need(L, fc_extent((int)max_batch));
+        if (exact > need) need = exact;
+    }
+    int rc = ensure_workspace(L, need);
+    if (rc != CIRC_OK) return rc;
+    // the stored form that a forward of exactly this size reads (other sizes may take another path and build theirs then)
+    if (max_batch > (1L << 30) / 2) return CIRC_OK;
+    int variant;
+    Extent ef;
+    if (L->kind == 0) {
+        variant = plan_fc_variant(L, (int)max_batch);
+        ef = fc_extent((int)max_batch);
+    } else {
+        variant = L->variant == CIRC_VARIANT_AUTO ? (tensor_supported(L) ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED) : L->variant;
+        ef = e;
+    }
+    if (variant == CIRC_VARIANT_FUSED) return CIRC_OK;
+    if (variant == CIRC_VARIANT_TENSOR && !tensor_supported(L)) return CIRC_OK;   // the forward itself reports it
+    return prepare_staged(L, ef, 0, variant == CIRC_VARIANT_TENSOR);
 }
 
 long circ_workspace_bytes(circ_handle h) {
@@ -550,6 +634,7 @@ long circ_weight_bytes(circ_handle h) {
     if (L->w_stream_bf16) b += blocks * L->geo.k * sizeof(__nv_bfloat16);
     if (L->a_f32) b += L->a_elems * sizeof(float);
     if (L->a_bf16) b += 2 * L->a_elems * sizeof(__nv_bfloat16) + 256;
+    if (L->a_twin) b += twin_elems(L) * sizeof(__nv_bfloat16) + 256;
     if (L->transposed) b += (size_t)circ_weight_bytes(reinterpret_cast<circ_handle>(L->transposed));
     return (long)b;
 }

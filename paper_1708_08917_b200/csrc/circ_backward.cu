@@ -498,22 +498,40 @@ static int build_transposed(Layer* L) {
     }
     long blocks = (long)((count + 255) / 256);
     if (blocks > 148L * 32) blocks = 148L * 32;
+    // the defining vectors: the retained copy (embedded block sizes), else recovered from the stored spectra
+    float* w_src = L->w_dev;
+    float* w_tmp = nullptr;
+    if (!w_src) {
+        if (dev_alloc(&w_tmp, count * sizeof(float)) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(wt);
+            set_error(CIRC_ERR_ALLOC, "allocation of the defining vectors (%zu bytes) failed", count * sizeof(float));
+            return CIRC_ERR_ALLOC;
+        }
+        // the spectra hold the layer's current convention; the vectors are wanted in the caller's (convention 0) form
+        if (launch_defining_vectors(L, w_tmp, 0) != CIRC_OK) {
+            cudaFree(wt);
+            cudaFree(w_tmp);
+            return CIRC_ERR_CUDA;
+        }
+        w_src = w_tmp;
+    }
     if (L->kind == 1)
-        transpose_reverse_conv_kernel<<<(unsigned)blocks, 256>>>(L->w_dev, wt, r, p, q, k);
+        transpose_reverse_conv_kernel<<<(unsigned)blocks, 256>>>(w_src, wt, r, p, q, k);
     else
-        transpose_reverse_kernel<<<(unsigned)blocks, 256>>>(L->w_dev, wt, p, q, k);
+        transpose_reverse_kernel<<<(unsigned)blocks, 256>>>(w_src, wt, p, q, k);
     count_launches(1);
     Layer* T = nullptr;
     // the transposed layer maps c_out -> c_in; a convolution's gradient is a convolution with padding r - 1 - pad
     if (cudaDeviceSynchronize() == cudaSuccess)
         T = make_layer(L->kind, L->n, L->m, k, taps, r, L->kind == 1 ? r - 1 - L->geo.pad : 0, wt);  // copies wt, computes spectra
     cudaFree(wt);
+    cudaFree(w_tmp);
     if (!T) return circ_last_code() != CIRC_OK ? circ_last_code() : CIRC_ERR_CUDA;
     T->x_dtype = L->y_dtype;   // the gradient flows from the output side to the input side
     T->y_dtype = L->x_dtype;
     if (L->convention != 0) {
-        T->convention = L->convention;
-        int rc = launch_precompute(T, 0);
+        int rc = circ_set_convention(reinterpret_cast<circ_handle>(T), L->convention);
         if (rc != CIRC_OK || cudaDeviceSynchronize() != cudaSuccess) {
             free_layer(T);
             set_error(CIRC_ERR_CUDA, "spectrum precompute of the transposed layer failed");

@@ -81,14 +81,17 @@ struct Layer {
     int variant;
     int last_variant;
 
-    float* w_dev;       // retained copy of the defining vectors [taps][p][q][k]
+    float* w_dev;       // retained copy of the defining vectors [taps][p][q][ku]: embedded block sizes only (a power-of-two
+                        // block's vectors can be recovered from its spectra), else nullptr
     float* bias_dev;    // [m] or nullptr
-    float* w_stream;    // spectra for the fused kernel: [taps][p][q][k] packed half spectra
+    float* w_stream;    // the canonical stored form, [taps][p][q][k] packed half spectra (m n / k floats); read by the
+                        // one-launch kernel.  The operand layouts below are built from it on first use (ensure_forms).
     __nv_bfloat16* w_stream_bf16;  // the same rounded to bfloat16 (only after circ_set_spectrum_dtype), or nullptr
     int w_dtype;        // CIRC_F32 or CIRC_BF16: which stream the fused kernel reads
     float* a_f32;       // embedded float32 operand for the staged FMA contraction
     __nv_bfloat16* a_bf16;  // embedded bfloat16 operand (hi | lo split) for the tensor-core contraction
-    size_t a_elems;     // elements of a_f32
+    __nv_bfloat16* a_twin;  // bfloat16 operand (hi | lo split) with every complex value once, for the twin-column contraction
+    size_t a_elems;     // elements of a_f32 (a_bf16 has twice as many, a_twin as many)
 
     void* ws;           // workspace: frequency-domain operands X and Y
     size_t ws_bytes;
@@ -98,6 +101,8 @@ struct Layer {
     size_t x_stage_bytes, y_stage_bytes;
     mutable int last_kernels[3];  // which S1 / S2 / S3 kernel served the most recent staged forward (KERNEL_* ids below)
     int inject;           // test-only fault injection (circ_debug.h): 0 = none
+    int no_rows_kernel;   // 1: never use the row-streaming tensor-core contraction (circ_debug_set_contraction)
+    int no_twin;          // 1: never use the twin-column form of the tensor contraction (circ_debug_set_twin)
     int fused_split;      // column slices of the one-launch kernel forced by circ_debug_set_fused_split (0 = planner's choice)
     Layer* transposed;  // the n x m layer W^T (built on first use by the backward pass), or nullptr
 };
@@ -108,7 +113,10 @@ enum {
     KERNEL_S1_LOADS = 1,      // input transforms, per-thread vector loads
     KERNEL_S1_BULK = 2,       // input transforms, tiles staged by bulk asynchronous copies
     KERNEL_S2_FMA = 10,       // contraction on the float32 FMA pipes
-    KERNEL_S2_TENSOR = 11,    // contraction on the tensor cores
+    KERNEL_S2_TENSOR = 11,    // contraction on the tensor cores, embedded weights [Wr -Wi; Wi Wr]
+    KERNEL_S2_TENSOR_TWIN = 12,  // contraction on the tensor cores, weights stored once, twin column groups of X
+    KERNEL_S2_ROWS = 13,      // row-streaming tensor-core contraction (weight rows on the MMA's M side), embedded weights
+    KERNEL_S2_ROWS_TWIN = 14, // the same with twin columns
     KERNEL_S3_LOADS = 20,     // inverse transforms, per-thread loads
     KERNEL_S3_BULK = 21,      // inverse transforms, tiles staged by bulk asynchronous copies
     KERNEL_S4_FUSED = 30      // the one-launch kernel: last_kernels = {this id, column slices, row blocks per thread block}
@@ -134,7 +142,8 @@ int staged_operands(Layer* L, const Extent& e, cudaStream_t stream, float** xop,
 bool stream_is_capturing(cudaStream_t stream);
 int stage_input(Layer* L, const void* x, float* xop, const Extent& e, cudaStream_t stream, bool tensor);
 int stage_contract(Layer* L, const float* xop, float* yop, const Extent& e, cudaStream_t stream, bool tensor);
-int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream);
+int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream, bool tensor);
+int prepare_staged(Layer* L, const Extent& e, cudaStream_t stream, bool tensor);   // stored form of the path, before the first launch
 int staged_dependent_launches(const Layer* L, const Extent& e);
 Extent fc_extent(int batch);
 Extent conv_extent(const Layer* L, int N, int H, int W);
@@ -196,20 +205,49 @@ inline cudaError_t launch_kernel(int dependent, void (*kernel)(KArgs...), dim3 g
 // Kernel launchers (one translation unit each).  All return a CIRC_* code and only enqueue.
 // ---------------------------------------------------------------------------------------------
 
-// S0: spectra of the defining vectors, in every stored layout.
+// S0: spectra of the defining vectors (w_dev -> w_stream), then every operand layout the layer already holds.
 int launch_precompute(Layer* L, cudaStream_t stream);
+// w_stream -> the given operand layouts (null pointers are skipped), and the bfloat16 stream if the layer has one.
+int launch_spectrum_forms(Layer* L, float* a_f32, __nv_bfloat16* a_bf16, __nv_bfloat16* a_twin, cudaStream_t stream);
+// The other circulant convention of a power-of-two block: conjugate w_stream in place.
+int launch_conjugate_stream(Layer* L, cudaStream_t stream);
+// Defining vectors [taps][p][q][k] recovered from w_stream (power-of-two blocks).
+int launch_defining_vectors(const Layer* L, float* w_out, cudaStream_t stream);
+// Stored operand layouts, built on first use.  `forms` is a mask of FORM_*; fails with CIRC_ERR_UNSUPPORTED when a
+// form is missing while `stream` is being captured (building allocates).
+enum { FORM_A_F32 = 1, FORM_A_BF16 = 2, FORM_A_TWIN = 4 };
+inline size_t twin_elems(const Layer* L) { return L->a_elems + (size_t)2 * L->geo.taps * L->geo.p * L->geo.q; }   // bfloat16 values of a_twin
+int ensure_forms(Layer* L, unsigned forms, cudaStream_t stream);
+// How the tensor-core contraction of a forward runs (circ_tensor_rows.cu): `twin`: weights stored once, X twice;
+// `rows`: the row-streaming kernel instead of the large-batch one.
+struct ContractionPlan {
+    bool twin, rows;
+};
+ContractionPlan plan_contraction(const Layer* L, const Extent& e);
+inline bool use_twin(const Layer* L, const Extent& e) { return plan_contraction(L, e).twin; }
+int launch_contract_rows(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin);
+// Copies of Y that the row-streaming contraction writes for a real / a complex problem; the inverse-transform kernel
+// adds them up.  {0, 0}: Y is a single array.
+struct RowsPieces {
+    int real, cplx;
+};
+RowsPieces rows_pieces(const Layer* L, bool twin);
+// Loads the fixed scratch array of the allocation-free entry point and caches its address (circ_noalloc.cu).
+int noalloc_warm();
 // Rounds w_stream into w_stream_bf16 (which must be allocated).
 int launch_round_stream(Layer* L, cudaStream_t stream);
 
 // S1 / C1: forward transforms of the input -> operand X.  xmode 0: float32 [problem][col][Kq];
 // 1: bfloat16 [problem][col][hi | lo][Kq] (split of float32 values); 2: bfloat16 [problem][col][Kq].
-int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream);
+// `twin` (xmode 1 / 2, fully-connected): complex problems get two column groups, (Zr, -Zi) and (Zi, Zr).
+int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream, bool twin = false);
 
 // S2 / C2 on the float32 FMA pipes: Y = A . X per problem.
 int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream);
 
 // S2 / C2 on the tensor cores (bfloat16 operands from xmode 1 or 2, float32 accumulate).
-int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream);
+// `twin`: the weights come from a_twin, complex problems have p rows and twice the columns (real parts, then imaginary parts).
+int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin = false);
 bool tensor_supported(const Layer* L);
 
 // Tensor-core batch product of the backward pass: for every frequency problem
@@ -224,7 +262,10 @@ bool tensor_batch_product_supported(int cols);
 // `correlation`: how an embedded block size folds.  false: a[t] = c[t] + c[t + ku] (the forward pass, a circular
 // convolution); true: a[t] = c[t] + c[t - ku] (the weight gradient, a circular correlation whose negative lags sit at
 // the top of the transform).  Ignored when the block size is the transform size.
-int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation = false);
+// `twin`: Y of the complex problems is [real parts of all columns][imaginary parts of all columns] instead of interleaved rows.
+// `pieces`: Y comes as that many copies per real / complex problem, to be added up ({0, 0}: a single array).
+int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation = false,
+                       bool twin = false, RowsPieces pieces = RowsPieces{0, 0});
 
 // S3 of layer L and S1 of the next layer (same k, its q = L's p) in one launch: Y operand -> X operand (xmode 0 or 1).
 int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, const Extent& ext, cudaStream_t stream);

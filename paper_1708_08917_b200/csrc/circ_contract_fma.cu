@@ -127,6 +127,10 @@ __global__ void __launch_bounds__(256) contract_fma_kernel(ContractArgs g) {
 }
 
 int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream) {
+    if (!L->a_f32) {
+        set_error(CIRC_ERR_ARG, "the float32 operand of the staged contraction has not been built");
+        return CIRC_ERR_ARG;
+    }
     ContractArgs g;
     g.a = L->a_f32;
     g.x = xop;

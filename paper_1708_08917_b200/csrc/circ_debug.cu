@@ -7,6 +7,8 @@ namespace circ {
 
 static_assert((int)CIRC_KERNEL_S1_LOADS == (int)KERNEL_S1_LOADS && (int)CIRC_KERNEL_S1_BULK == (int)KERNEL_S1_BULK &&
                   (int)CIRC_KERNEL_S2_FMA == (int)KERNEL_S2_FMA && (int)CIRC_KERNEL_S2_TENSOR == (int)KERNEL_S2_TENSOR &&
+                  (int)CIRC_KERNEL_S2_TENSOR_TWIN == (int)KERNEL_S2_TENSOR_TWIN && (int)CIRC_KERNEL_S2_ROWS == (int)KERNEL_S2_ROWS &&
+                  (int)CIRC_KERNEL_S2_ROWS_TWIN == (int)KERNEL_S2_ROWS_TWIN &&
                   (int)CIRC_KERNEL_S3_LOADS == (int)KERNEL_S3_LOADS && (int)CIRC_KERNEL_S3_BULK == (int)KERNEL_S3_BULK &&
                   (int)CIRC_KERNEL_S4_FUSED == (int)KERNEL_S4_FUSED,
               "public and internal kernel ids must agree");
@@ -75,6 +77,7 @@ int circ_debug_forward_repeat(circ_handle h, const void* x, void* y, int N, int 
     }
     float *xop = nullptr, *yop = nullptr;
     if ((rc = staged_operands(L, e, s, &xop, &yop)) != CIRC_OK) return rc;
+    if ((rc = prepare_staged(L, e, s, tensor)) != CIRC_OK) return rc;
     struct DependentGuard {
         DependentGuard(int mode) { dependent_launches() = mode; }
         ~DependentGuard() { dependent_launches() = PDL_OFF; }
@@ -84,7 +87,7 @@ int circ_debug_forward_repeat(circ_handle h, const void* x, void* y, int N, int 
     for (int rep = 0; rep < (stage == CIRC_STAGE_CONTRACTION ? times : 1); ++rep)
         if ((rc = stage_contract(L, xop, yop, e, s, tensor)) != CIRC_OK) return rc;
     for (int rep = 0; rep < (stage == CIRC_STAGE_OUTPUT_IFFT ? times : 1); ++rep)
-        if ((rc = stage_output(L, yop, y, e, s)) != CIRC_OK) return rc;
+        if ((rc = stage_output(L, yop, y, e, s, tensor)) != CIRC_OK) return rc;
     L->last_variant = variant;
     return CIRC_OK;
 }
@@ -137,6 +140,17 @@ int circ_debug_set_fused_split(circ_handle h, int slices) {
         return CIRC_ERR_ARG;
     }
     L->fused_split = slices;
+    return CIRC_OK;
+}
+
+int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (allow_twin != 0 && allow_twin != 1) || (allow_rows != 0 && allow_rows != 1)) {
+        set_error(CIRC_ERR_ARG, "bad handle or flags %d, %d", allow_twin, allow_rows);
+        return CIRC_ERR_ARG;
+    }
+    L->no_twin = !allow_twin;
+    L->no_rows_kernel = !allow_rows;
     return CIRC_OK;
 }
 

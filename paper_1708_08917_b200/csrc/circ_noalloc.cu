@@ -9,6 +9,8 @@
 // It runs the staged fully-connected path (input transforms -> per-frequency FMA contraction ->
 // inverse transforms with bias / ReLU) with the frequency-domain operands X and Y placed in the
 // fixed device array below instead of an allocated workspace.
+#include <atomic>
+
 #include "circ_common.cuh"
 
 namespace circ {
@@ -20,7 +22,7 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratch
 // In host code `g_noalloc_scratch` is only a handle for the runtime, not a device address.  The
 // address is looked up once per device (with that device current) and cached here.
 constexpr int kMaxDevices = 64;
-static void* g_scratch_addr[kMaxDevices] = {};
+static std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 static int scratch_for_current_device(void** out) {
     int dev = -1;
@@ -29,17 +31,26 @@ static int scratch_for_current_device(void** out) {
         set_error(CIRC_ERR_UNSUPPORTED, "device ordinal %d is beyond the %d devices this entry point tracks", dev, kMaxDevices);
         return CIRC_ERR_UNSUPPORTED;
     }
-    if (!g_scratch_addr[dev]) {
-        void* ptr = nullptr;
+    void* ptr = g_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
+        // first use on this device: the runtime loads the module that holds the array (this is when its 32 MiB are
+        // taken from the device) and gives its address; concurrent first calls all get the same answer
         const cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
         if (e != cudaSuccess || !ptr) {
             set_error(CIRC_ERR_CUDA, "cudaGetSymbolAddress(scratch) failed: %s", cudaGetErrorString(e));
             return CIRC_ERR_CUDA;
         }
-        g_scratch_addr[dev] = ptr;
+        g_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out = g_scratch_addr[dev];
+    *out = ptr;
     return CIRC_OK;
+}
+
+// Called where the library is allowed to allocate anyway (when the stored form that the allocation-free path reads
+// is built): the array's module is loaded and its address known before the first allocation-free forward.
+int noalloc_warm() {
+    void* p = nullptr;
+    return scratch_for_current_device(&p);
 }
 
 }  // namespace circ
@@ -86,6 +97,13 @@ int circ_fc_forward_noalloc(circ_handle h, const void* x, void* y, int batch, vo
                   "(use circ_fc_forward, or a smaller batch)",
                   batch, L->m, L->n, need, kNoAllocScratchBytes);
         return CIRC_ERR_SHAPE;
+    }
+    if (!L->a_f32) {
+        // the float32 operand of the staged path is built (allocated) on first use; this call may not allocate
+        set_error(CIRC_ERR_UNSUPPORTED,
+                  "the stored form the staged path reads has not been built yet: while allocation is still allowed, call "
+                  "circ_set_variant(h, CIRC_VARIANT_STAGED) and circ_reserve(h, batch), or run one circ_fc_forward on that path");
+        return CIRC_ERR_UNSUPPORTED;
     }
     void* scratch = nullptr;
     int rc = scratch_for_current_device(&scratch);

@@ -76,6 +76,8 @@ circ_stack_handle circ_stack_create(const circ_handle* layers, int count) {
             }
         }
     }
+    // stacked layers hand their operands to one another in the embedded layout: keep every layer on it
+    for (int l = 0; l < count; ++l) reinterpret_cast<Layer*>(layers[l])->no_twin = 1;   // (its kernels are called directly here)
     Stack* S = new (std::nothrow) Stack();
     if (!S) {
         set_error(CIRC_ERR_ALLOC, "host allocation failed");
@@ -185,6 +187,7 @@ int circ_stack_forward(circ_stack_handle s, const void* x, void* y, int batch, v
         }
         const bool tensor = variant[l] == CIRC_VARIANT_TENSOR;
         if ((rc = ensure_workspace(L, stack_workspace(L, e))) != CIRC_OK) return rc;
+        if ((rc = ensure_forms(L, tensor ? FORM_A_BF16 : FORM_A_F32, st)) != CIRC_OK) return rc;   // stacks use the embedded weights
         float* xop = static_cast<float*>(L->ws);
         float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
         if (!operand_ready) {

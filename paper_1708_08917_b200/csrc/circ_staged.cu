@@ -70,9 +70,14 @@ __device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& 
 }
 
 // Operand Y -> tile (the first half of S3): fills zs[bin][transform] for the CTA's TT transforms.
-template <int K, int EMAX, bool VEC>
+// TWIN: Y of a complex problem holds the real parts of all 2 Bho columns, then the imaginary parts (p rows each),
+// instead of 2p interleaved rows.
+// Y may come as several copies, `copy_stride` floats apart (copies_r of every real problem, copies_c of every complex
+// one), that are added here in a fixed order (the row-streaming contraction cuts its contraction range into pieces).
+__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+template <int K, int EMAX, bool VEC, bool TWIN = false>
 __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW], const float* __restrict__ yop, int p, int Bho,
-                                               long total, Split sp) {
+                                               long total, Split sp, int copies_r = 1, int copies_c = 1, size_t copy_stride = 0) {
     constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
     const size_t cols = 2 * (size_t)Bho;
     const size_t real_sz = cols * p, cplx_sz = 2 * real_sz;
@@ -93,15 +98,26 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
             split_at<TT>(sp, grp * 4, p, c, i);
             if (f == 0 || f == K / 2) {
                 const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                r0[it] = __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i));
-                r1[it] = __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i));
+                for (int s = 0; s < copies_r; ++s, yg += copy_stride) {
+                    r0[it] = add4(r0[it], __ldg(reinterpret_cast<const float4*>(yg + (size_t)c * p + i)));
+                    r1[it] = add4(r1[it], __ldg(reinterpret_cast<const float4*>(yg + ((size_t)Bho + c) * p + i)));
+                }
             } else {
                 const bool mirror = f > K / 2;
                 const int g = mirror ? K - f : f;
-                const float4* r = reinterpret_cast<const float4*>(yop + problem_offset(g + 1, real_sz, cplx_sz) +
-                                                                  ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i);
-                r0[it] = __ldg(r);
-                r1[it] = __ldg(r + 1);
+                if constexpr (TWIN) {
+                    const float* r = yop + problem_offset(g + 1, real_sz, cplx_sz) + ((size_t)(mirror ? Bho : 0) + c) * p + i;
+                    for (int s = 0; s < copies_c; ++s, r += copy_stride) {
+                        r0[it] = add4(r0[it], __ldg(reinterpret_cast<const float4*>(r)));                        // four real parts
+                        r1[it] = add4(r1[it], __ldg(reinterpret_cast<const float4*>(r + (size_t)2 * Bho * p)));  // their imaginary parts
+                    }
+                } else {
+                    const float* r = yop + problem_offset(g + 1, real_sz, cplx_sz) + ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i;
+                    for (int s = 0; s < copies_c; ++s, r += copy_stride) {
+                        r0[it] = add4(r0[it], __ldg(reinterpret_cast<const float4*>(r)));
+                        r1[it] = add4(r1[it], __ldg(reinterpret_cast<const float4*>(r) + 1));
+                    }
+                }
             }
         }
 #pragma unroll
@@ -112,6 +128,10 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
             if (f == 0 || f == K / 2) {
                 za = make_float4(r0[it].x, r1[it].x, r0[it].y, r1[it].y);
                 zb = make_float4(r0[it].z, r1[it].z, r0[it].w, r1[it].w);
+            } else if constexpr (TWIN) {
+                const float sgn = f > K / 2 ? -1.f : 1.f;
+                za = make_float4(r0[it].x, sgn * r1[it].x, r0[it].y, sgn * r1[it].y);
+                zb = make_float4(r0[it].z, sgn * r1[it].z, r0[it].w, sgn * r1[it].w);
             } else {
                 const float sgn = f > K / 2 ? -1.f : 1.f;
                 za = r0[it];
@@ -128,18 +148,30 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
             if (T2 >= total) continue;
             int c, i;
             split_at<TT>(sp, tl, p, c, i);
-            float2 z;
+            float2 z = make_float2(0.f, 0.f);
             if (f == 0 || f == K / 2) {
                 const float* yg = yop + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                z.x = __ldg(yg + (size_t)c * p + i);
-                z.y = __ldg(yg + ((size_t)Bho + c) * p + i);
-            } else if (f < K / 2) {
-                const float* yg = yop + problem_offset(f + 1, real_sz, cplx_sz) + (size_t)c * 2 * p + 2 * i;
-                z = __ldg(reinterpret_cast<const float2*>(yg));
+                for (int s = 0; s < copies_r; ++s, yg += copy_stride) {
+                    z.x += __ldg(yg + (size_t)c * p + i);
+                    z.y += __ldg(yg + ((size_t)Bho + c) * p + i);
+                }
+            } else if constexpr (TWIN) {
+                const bool mirror = f > K / 2;
+                const float* yg = yop + problem_offset((mirror ? K - f : f) + 1, real_sz, cplx_sz) + ((size_t)(mirror ? Bho : 0) + c) * p + i;
+                for (int s = 0; s < copies_c; ++s, yg += copy_stride) {
+                    z.x += __ldg(yg);
+                    z.y += __ldg(yg + (size_t)2 * Bho * p);
+                }
+                if (mirror) z.y = -z.y;
             } else {
-                const float* yg = yop + problem_offset(K - f + 1, real_sz, cplx_sz) + ((size_t)Bho + c) * 2 * p + 2 * i;
-                z = __ldg(reinterpret_cast<const float2*>(yg));
-                z.y = -z.y;
+                const bool mirror = f > K / 2;
+                const float* yg = yop + problem_offset((mirror ? K - f : f) + 1, real_sz, cplx_sz) + ((size_t)(mirror ? Bho : 0) + c) * 2 * p + 2 * i;
+                for (int s = 0; s < copies_c; ++s, yg += copy_stride) {
+                    const float2 t = __ldg(reinterpret_cast<const float2*>(yg));
+                    z.x += t.x;
+                    z.y += t.y;
+                }
+                if (mirror) z.y = -z.y;
             }
             zs[f][tl] = z;
         }
@@ -147,13 +179,15 @@ __device__ __forceinline__ void gather_operand(float2 (*zs)[Tile<K, EMAX>::ROW],
 }
 
 // Tile -> operand X (the second half of S1): zs[bin][transform] holds the spectra of the CTA's TT transforms.
-template <int K, int EMAX, int XMODE>
+// TWIN (bfloat16 modes): a complex problem gets two column groups, (Zr, -Zi) for the 2 Bh columns and then (Zi, Zr)
+// for them again; multiplied by weights stored once as (Wr, Wi) pairs they give the real and the imaginary parts.
+template <int K, int EMAX, int XMODE, bool TWIN = false>
 __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>::ROW], void* __restrict__ xop, int q, int Bh,
                                                 long total, Split sp) {
     constexpr int TT = Tile<K, EMAX>::TT, kThreads = Tile<K, EMAX>::NT;
     const size_t cols = 2 * (size_t)Bh;
     constexpr int NPART = XMODE == 1 ? 2 : 1;
-    const size_t real_sz = cols * q * NPART, cplx_sz = 2 * real_sz;
+    const size_t real_sz = cols * q * NPART, cplx_sz = (TWIN ? 4 : 2) * real_sz;
 
     if constexpr (XMODE == 0) {
         // scalar scatter (any q): one work item = (bin, transform), consecutive threads = consecutive transforms
@@ -213,8 +247,21 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
                 uint32_t l0, l1, l2, l3;
                 const uint32_t h0 = bf16_split_pair(za.x, i0, l0), h1 = bf16_split_pair(za.z, i1, l1);
                 const uint32_t h2 = bf16_split_pair(zb.x, i2, l2), h3 = bf16_split_pair(zb.z, i3, l3);
-                *reinterpret_cast<uint4*>(d) = make_uint4(h0, h1, h2, h3);
-                if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0, l1, l2, l3);
+                if constexpr (TWIN) {
+                    // a word holds (re | im << 16): negating im flips its sign bit, swapping re and im swaps the halves
+                    constexpr uint32_t S = 0x80000000u;
+                    auto swp = [](uint32_t v) { return __byte_perm(v, 0u, 0x1032); };
+                    __nv_bfloat16* d2 = d + cols * (size_t)(NPART * 2 * q);
+                    *reinterpret_cast<uint4*>(d) = make_uint4(h0 ^ S, h1 ^ S, h2 ^ S, h3 ^ S);
+                    *reinterpret_cast<uint4*>(d2) = make_uint4(swp(h0), swp(h1), swp(h2), swp(h3));
+                    if constexpr (XMODE == 1) {
+                        *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0 ^ S, l1 ^ S, l2 ^ S, l3 ^ S);
+                        *reinterpret_cast<uint4*>(d2 + 2 * q) = make_uint4(swp(l0), swp(l1), swp(l2), swp(l3));
+                    }
+                } else {
+                    *reinterpret_cast<uint4*>(d) = make_uint4(h0, h1, h2, h3);
+                    if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0, l1, l2, l3);
+                }
             }
         }
     }
@@ -226,7 +273,7 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
 // XMODE 1: bfloat16 operand [problem][col][hi | lo][Kq]            (tensor cores, float32 input split in two)
 // XMODE 2: bfloat16 operand [problem][col][Kq]                     (tensor cores, bfloat16 input)
 // Complex problems interleave (Re, Im): contraction index 2j, 2j+1.  XMODE 1 / 2 need q % 8 == 0.
-template <int K, int EMAX, typename TIN, int XMODE>
+template <int K, int EMAX, typename TIN, int XMODE, bool TWIN = false>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q,
                  int B, int Bh, long total, int ku, int pdl_late) {
@@ -296,7 +343,7 @@ input_fft_kernel(const TIN* __restrict__ x, void* __restrict__ xop, int n, int q
     __syncthreads();
 
     if (pdl_late) pdl_trigger();
-    scatter_operand<K, EMAX, XMODE>(zs, xop, q, Bh, total, sp);
+    scatter_operand<K, EMAX, XMODE, TWIN>(zs, xop, q, Bh, total, sp);
 }
 
 // Bias, activation and stores of one inverse-transformed tile (block size = transform size).  `tile` is the staging
@@ -373,10 +420,11 @@ __device__ __forceinline__ void store_outputs(const float2 (&v)[FftShape<K, EMAX
 // ---- S3: operand Y -> y --------------------------------------------------------------------------
 // One transform = (pair c, row block i).  Y[problem][col][row], complex problems with rows 2i, 2i+1 = (Re, Im).
 // VEC (p % 4 == 0): 32-byte reads of four consecutive row blocks; otherwise element by element.
-template <int K, int EMAX, typename TOUT, bool VEC>
+template <int K, int EMAX, typename TOUT, bool VEC, bool TWIN = false>
 __global__ void __launch_bounds__(Tile<K, EMAX>::NT)
 output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y, 
-                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku, int corr, int pdl_late) {
+                   const float* __restrict__ bias, int relu, int m, int p, int Bo, int Bho, long total, int ku, int corr, int pdl_late,
+                   int copies_r, int copies_c, size_t copy_stride) {
     constexpr int E = FftShape<K, EMAX>::E, L = FftShape<K, EMAX>::L, TT = Tile<K, EMAX>::TT, ROW = Tile<K, EMAX>::ROW;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float2* tw = reinterpret_cast<float2*>(smem_raw);
@@ -398,7 +446,7 @@ output_ifft_kernel(const float* __restrict__ yop, TOUT* __restrict__ y,
     for (int r = 0; r < E; ++r) bv[r] = 0.f;
     if (bias && live && ku == K) load_run<E>(bias + i * K + E * l, bv);
 
-    gather_operand<K, EMAX, VEC>(zs, yop, p, Bho, total, sp);
+    gather_operand<K, EMAX, VEC, TWIN>(zs, yop, p, Bho, total, sp, copies_r, copies_c, copy_stride);
     __syncthreads();
 
     const int f2 = lane_residue<K, EMAX>(l);
@@ -717,11 +765,15 @@ static bool latency_bound(long transforms, int k) {
     return k >= 16 && warps_at_16 < 148L * 8;
 }
 
-int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream) {
+int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream, bool twin) {
     const int q = L->geo.q, n = L->n;
     const long total = (long)ext.Bh * q;
     if (xmode != 0 && (q % 8) != 0) {
         set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need q %% 8 == 0 (q=%d)", q);
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    if (twin && (xmode == 0 || embedded(L->geo))) {
+        set_error(CIRC_ERR_UNSUPPORTED, "twin columns need a bfloat16 operand and a block size that is its transform size");
         return CIRC_ERR_UNSUPPORTED;
     }
     const bool small = latency_bound(total, L->geo.k);
@@ -734,9 +786,18 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
             auto launch = [&](auto tin, auto mode) {
                 using TIN = decltype(tin);
                 constexpr int XMODE = decltype(mode)::value;
-                allow_smem(input_fft_kernel<K, EMAX, TIN, XMODE>, Tile<K, EMAX>::SMEM);
-                launch_kernel(dependent_launches(), input_fft_kernel<K, EMAX, TIN, XMODE>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
-                              static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku, (int)(dependent_launches() == PDL_LATE));
+                auto run = [&](auto kernel) {
+                    allow_smem(kernel, Tile<K, EMAX>::SMEM);
+                    launch_kernel(dependent_launches(), kernel, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream,
+                                  static_cast<const TIN*>(x), xop, n, q, ext.B, ext.Bh, total, L->geo.ku, (int)(dependent_launches() == PDL_LATE));
+                };
+                if constexpr (XMODE != 0) {
+                    if (twin) {
+                        run(input_fft_kernel<K, EMAX, TIN, XMODE, true>);
+                        return;
+                    }
+                }
+                run(input_fft_kernel<K, EMAX, TIN, XMODE, false>);
             };
             const bool bf = L->x_dtype == CIRC_BF16;
             if (xmode == 0) {
@@ -782,14 +843,19 @@ static constexpr size_t bulk_smem() {
     return sizeof(float2) * ((size_t)K + (size_t)2 * K * Tile<K, 16>::ROW) + (size_t)Tile<K, 16>::TT * 12 + 32;
 }
 
-int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation) {
+int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream, bool correlation, bool twin, RowsPieces pieces) {
     const int p = L->geo.p, m = L->m;
     const long total = (long)ext.Bho * p;
     const bool small = latency_bound(total, L->geo.k);
     // large forwards of power-of-two blocks up to 256: tiles fetched by bulk copies, persistent CTAs (needs 16-byte aligned runs)
     // (measured at 16384 x 16384, batch 1024: k = 16: 40.7 -> 35.2 us, k = 64: 33.7 -> 32.5, k = 256: no change; k = 4, whose
     // tile has two bulk rows only, is slower this way and keeps the load-based kernel)
-    const bool bulk = !small && !embedded(L->geo) && L->geo.k >= 16 && L->geo.k <= 256 && (total & 1) == 0 && total >= 148L * 256 &&
+    if (twin && (embedded(L->geo) || correlation)) {
+        set_error(CIRC_ERR_UNSUPPORTED, "twin columns need a block size that is its transform size");
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    const size_t copy_stride = (size_t)2 * ext.Bho * p * L->geo.k;     // all problems of Y
+    const bool bulk = !twin && pieces.real == 0 && !small && !embedded(L->geo) && L->geo.k >= 16 && L->geo.k <= 256 && (total & 1) == 0 && total >= 148L * 256 &&
                       (reinterpret_cast<uintptr_t>(yop) & 15u) == 0 && L->dev_status != nullptr;
     if (bulk) {
         auto go = [&](auto kc) -> int {
@@ -829,10 +895,15 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
             auto launch = [&](auto tout, auto vec) {
                 using TOUT = decltype(tout);
                 constexpr bool VEC = decltype(vec)::value;
-                allow_smem(output_ifft_kernel<K, EMAX, TOUT, VEC>, Tile<K, EMAX>::SMEM);
-                launch_kernel(dependent_launches(), output_ifft_kernel<K, EMAX, TOUT, VEC>, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
-                              static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku, (int)correlation,
-                              (int)(dependent_launches() == PDL_LATE));
+                auto run = [&](auto kernel) {
+                    allow_smem(kernel, Tile<K, EMAX>::SMEM);
+                    launch_kernel(dependent_launches(), kernel, dim3(blocks), dim3(Tile<K, EMAX>::NT), Tile<K, EMAX>::SMEM, stream, yop,
+                                  static_cast<TOUT*>(y), static_cast<const float*>(L->bias_dev), L->relu, m, p, ext.Bo, ext.Bho, total, L->geo.ku,
+                                  (int)correlation, (int)(dependent_launches() == PDL_LATE), pieces.real > 0 ? pieces.real : 1,
+                                  pieces.cplx > 0 ? pieces.cplx : 1, copy_stride);
+                };
+                if (twin) run(output_ifft_kernel<K, EMAX, TOUT, VEC, true>);
+                else run(output_ifft_kernel<K, EMAX, TOUT, VEC, false>);
             };
             const bool vec = (p % 4) == 0;
             if (L->y_dtype == CIRC_BF16) {

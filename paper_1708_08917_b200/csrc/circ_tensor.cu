@@ -19,9 +19,7 @@
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2..5 = epilogue
 // (tcgen05.ld -> registers -> global).  Every wait is bounded: on expiry the CTA records an error
 // word, drains its copies, frees its tensor memory and returns.
-#include <cuda.h>
-
-#include "circ_common.cuh"
+#include "circ_tc.cuh"
 
 namespace circ {
 
@@ -30,7 +28,6 @@ constexpr int kTileCols = 128;            // MMA M: batch columns / pixels per t
 constexpr int kKBlock = 64;               // bf16 elements per stage along K (one 128-byte swizzle row)
 constexpr int kMaxAcc = 8;           // accumulators in tensor memory (chosen per launch: as many as 512 columns hold)
 constexpr int kMaxStages = 8;        // ring depth is chosen per launch (as many stages as shared memory holds)
-constexpr uint32_t kSpinLimit = 1u << 22; // bounded wait: polls before giving up
 constexpr int kStagePitch = 36;           // floats per row of the epilogue's 32 x 32 staging tiles (16-byte aligned, conflict-free)
 constexpr int kStageOutBytes = 4 * 32 * kStagePitch * 4;   // one staging tile per epilogue warp
 
@@ -46,7 +43,9 @@ struct TcArgs {
     int pitch;               // input tile row pitch in pixels: tw + r - 1 (halo included)
     int xrows;               // pixels of the input tile that the TMA box brings: pitch * (th + r - 1)
     int xalloc;              // pixels reserved per stage for the input tile (covers every tap's 128-row view)
-    int tiles_w, tiles_h;    // tiles per image
+    int tiles_w, tiles_h;    // tiles per image (real problems)
+    int twin;                // complex problems in twin-column form: p rows, columns [real parts | imaginary parts]
+    int Wo_c, tiles_w_c;     // output columns and column tiles of a complex problem (twice the real ones when twin)
     int bn_real, bn_cplx;    // rows per tile (multiple of 16, <= 256)
     int nt_real, nt_cplx;    // row tiles per problem
     int ctas_real;           // CTAs that serve the two real problems
@@ -59,108 +58,6 @@ struct TcArgs {
     int no_copy;             // fault injection (tests only): the producer announces its bytes but issues no copy
 };
 
-// ---- PTX wrappers ------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false (and raises the CTA's abort flag) when the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
-    for (uint32_t it = 0; it < limit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (it > 64) __nanosleep(64);
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_5d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3,
-                                            int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-// The MMA warp runs its loop with all 32 lanes on warp-uniform values (so that descriptors and
-// addresses live in uniform registers); one elected lane enters the short branch that issues a
-// K block's MMAs and its commit.
-__device__ __forceinline__ uint32_t elect_one() {
-    uint32_t leader;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "elect.sync _|p, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(leader));
-    return leader;
-}
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes with the
-// 128-byte swizzle (what the TMA copy writes): 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);        // start address, 16-byte units
-    // (row-shifted starts need no phase field: the swizzle is applied to the absolute shared-memory address)
-    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                          // descriptor version (sm_100)
-    d |= (uint64_t)2 << 61;                          // layout: 128-byte swizzle
-    return d;
-}
-
 // Instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M = 128, N = bn.
 __device__ __forceinline__ uint32_t instr_desc(int bn) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTileCols >> 4) << 24);
@@ -169,16 +66,17 @@ __device__ __forceinline__ uint32_t instr_desc(int bn) {
 // Where a tile sits: which problem, which row tile, which spatial tile.
 struct TileCoord {
     bool real;
-    int prob_in_kind, prob, row0, bn, Mg, Kq, v, ho0, wo0;
+    int prob_in_kind, prob, row0, bn, Mg, Kq, v, ho0, wo0, Wo;
 };
 // 32-bit arithmetic only: the roles that call this are single threads on the critical path
 // (the host refuses launches with 2^31 tiles or more).
 __device__ __forceinline__ TileCoord decode_tile(const TcArgs& g, long tile) {
     TileCoord t;
-    const unsigned sp_tiles = (unsigned)(g.V * g.tiles_h * g.tiles_w);
     unsigned cta = (unsigned)tile;
     t.real = cta < (unsigned)g.ctas_real;
     if (!t.real) cta -= (unsigned)g.ctas_real;
+    const unsigned tiles_w = (unsigned)(t.real ? g.tiles_w : g.tiles_w_c);
+    const unsigned sp_tiles = (unsigned)(g.V * g.tiles_h) * tiles_w;
     const unsigned nt = (unsigned)(t.real ? g.nt_real : g.nt_cplx);
     const unsigned pr = cta / sp_tiles;              // problem * nt + row tile
     unsigned sp = cta - pr * sp_tiles;
@@ -190,24 +88,22 @@ __device__ __forceinline__ TileCoord decode_tile(const TcArgs& g, long tile) {
         t.prob_in_kind = (int)(pr / nt);
         row_tile = pr - (unsigned)t.prob_in_kind * nt;
     }
-    const unsigned per_img = (unsigned)(g.tiles_h * g.tiles_w);
+    const unsigned per_img = (unsigned)g.tiles_h * tiles_w;
     t.v = (int)(sp / per_img);
     sp -= (unsigned)t.v * per_img;
-    const unsigned th_i = g.tiles_w == 1 ? sp : sp / (unsigned)g.tiles_w;
-    const unsigned tw_i = sp - th_i * (unsigned)g.tiles_w;
+    const unsigned th_i = tiles_w == 1 ? sp : sp / tiles_w;
+    const unsigned tw_i = sp - th_i * tiles_w;
     t.ho0 = (int)th_i * g.th;
     t.wo0 = (int)tw_i * g.tw;
     t.bn = t.real ? g.bn_real : g.bn_cplx;
-    t.Mg = t.real ? g.p : 2 * g.p;
+    t.Mg = (t.real || g.twin) ? g.p : 2 * g.p;
     t.Kq = t.real ? g.q : 2 * g.q;
+    t.Wo = t.real ? g.Wo : g.Wo_c;
     t.row0 = (int)row_tile * t.bn;
     t.prob = t.real ? t.prob_in_kind : 2 + t.prob_in_kind;
     return t;
 }
 
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
 
 // Issue the MMAs of one product (one X part against one A part) for all R x R taps of a K block.
 // R is a compile-time filter size so that the tap loops unroll and the single issuing thread
@@ -500,16 +396,16 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                     for (int it = 0; it < 8; ++it) {
                         const int h2 = (int)(px_pos[it] >> 16), w2 = (int)(px_pos[it] & 0xffffu);
                         const int ho = t.ho0 + h2, wo = t.wo0 + w2;
-                        if (h2 < g.th && w2 < g.tw && ho < g.Ho && wo < g.Wo && seg * 4 < nvalid) {
+                        if (h2 < g.th && w2 < g.tw && ho < g.Ho && wo < t.Wo && seg * 4 < nvalid) {
                             const float4 v = *reinterpret_cast<const float4*>(stg + (it * 4 + sub) * kStagePitch + seg * 4);
-                            *reinterpret_cast<float4*>(ytile + ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg + c0 + seg * 4) = v;
+                            *reinterpret_cast<float4*>(ytile + ((size_t)((size_t)t.v * g.Ho + ho) * t.Wo + wo) * t.Mg + c0 + seg * 4) = v;
                         }
                     }
                     __syncwarp();
                 } else {
                     const int ho = t.ho0 + hh, wo = t.wo0 + ww;
-                    if (hh < g.th && ww < g.tw && ho < g.Ho && wo < g.Wo) {
-                        float* yrow = ytile + ((size_t)((size_t)t.v * g.Ho + ho) * g.Wo + wo) * t.Mg;
+                    if (hh < g.th && ww < g.tw && ho < g.Ho && wo < t.Wo) {
+                        float* yrow = ytile + ((size_t)((size_t)t.v * g.Ho + ho) * t.Wo + wo) * t.Mg;
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
                             if (e < nvalid) yrow[c0 + e] = __uint_as_float(acc[e]);
@@ -535,43 +431,14 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
 }
 
 // ---- host side ---------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-                  const cuuint32_t* box) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) {
-        set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-        return CIRC_ERR_CUDA;
-    }
-    cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, base, dims, strides_bytes, box, ones,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) {
-        set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
-        return CIRC_ERR_CUDA;
-    }
-    return CIRC_OK;
+static EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
+static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes, const cuuint32_t* box) {
+    return encode_tensor_map(map, base, rank, dims, strides_bytes, box);
 }
 
 static int round_up16(int v) { return (v + 15) & ~15; }
 
-bool tensor_supported(const Layer* L) { return L->a_bf16 != nullptr && (L->geo.q % 8) == 0 && encode_fn() != nullptr; }
+bool tensor_supported(const Layer* L) { return (L->geo.q % 8) == 0 && encode_fn() != nullptr; }
 
 // Ring depth, CTAs per SM and grid for a planned launch; maps = {A real, A complex, X hi real, X lo real, X hi complex, X lo complex}.
 static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int taps, int kq_max, long ctas, cudaStream_t stream) {
@@ -633,7 +500,7 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
     return CIRC_OK;
 }
 
-int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream) {
+int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin) {
     const Geometry& geo = L->geo;
     const int p = geo.p, q = geo.q, k = geo.k, taps = geo.taps;
     TcArgs g;
@@ -649,8 +516,19 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     } else {
         g.W = g.Wo = 2 * ext.Bh; g.H = g.Ho = 1; g.V = 1;
     }
+    if (twin && L->kind != 0) {
+        set_error(CIRC_ERR_UNSUPPORTED, "twin columns serve fully-connected layers only");
+        return CIRC_ERR_UNSUPPORTED;
+    }
+    const __nv_bfloat16* a_op = twin ? L->a_twin : L->a_bf16;
+    if (!a_op) {
+        set_error(CIRC_ERR_ARG, "the stored form of the spectra for this contraction has not been built");
+        return CIRC_ERR_ARG;
+    }
+    g.twin = twin ? 1 : 0;
+    g.Wo_c = twin ? 2 * g.Wo : g.Wo;
     const int halo = geo.r - 1;
-    g.tw = g.Wo < kTileCols - halo ? g.Wo : kTileCols - halo;
+    g.tw = g.Wo_c < kTileCols - halo ? g.Wo_c : kTileCols - halo;   // the wider problem kind sets the tile
     g.pitch = g.tw + halo;
     g.th = (kTileCols - g.tw) / g.pitch + 1;          // (th - 1) * pitch + tw <= 128 MMA rows
     if (g.th > g.Ho) g.th = g.Ho;
@@ -661,9 +539,11 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         g.xalloc = (need + 7) & ~7;                            // whole 1024-byte swizzle groups
     }
     g.tiles_w = (g.Wo + g.tw - 1) / g.tw;
+    g.tiles_w_c = (g.Wo_c + g.tw - 1) / g.tw;
     g.tiles_h = (g.Ho + g.th - 1) / g.th;
+    const int rows_c = twin ? p : 2 * p;                // rows of a complex problem
     g.bn_real = round_up16(p) > 256 ? 256 : round_up16(p);
-    g.bn_cplx = round_up16(2 * p) > 256 ? 256 : round_up16(2 * p);
+    g.bn_cplx = round_up16(rows_c) > 256 ? 256 : round_up16(rows_c);
     {
         // all taps' weight tiles of one K block share a stage with the input tile: narrow the row
         // tile until a stage fits half of the shared memory (two stages), or all of it at worst
@@ -676,13 +556,13 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         if (g.bn_cplx > cap) g.bn_cplx = cap;
     }
     g.cols_out = (long)g.V * g.Ho * g.Wo;
-    const int sp_tiles = g.V * g.tiles_h * g.tiles_w;
+    const int sp_tiles = g.V * g.tiles_h * g.tiles_w, sp_tiles_c = g.V * g.tiles_h * g.tiles_w_c;
     long ctas = 0;
     for (;;) {
         g.nt_real = (p + g.bn_real - 1) / g.bn_real;
-        g.nt_cplx = (2 * p + g.bn_cplx - 1) / g.bn_cplx;
+        g.nt_cplx = (rows_c + g.bn_cplx - 1) / g.bn_cplx;
         g.ctas_real = 2 * g.nt_real * sp_tiles;
-        ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles;
+        ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles_c;
         // a grid that leaves most of the 148 SMs idle is split into narrower row tiles
         if (ctas >= 100 || g.bn_cplx <= 32) break;
         g.bn_cplx = round_up16(g.bn_cplx / 2);
@@ -698,14 +578,15 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         cuuint64_t dims[4] = {(cuuint64_t)q, (cuuint64_t)p, (cuuint64_t)taps * 2, 2};
         cuuint64_t str[3] = {(cuuint64_t)taps * 2 * q * 2, (cuuint64_t)q * 2, (cuuint64_t)a_real_elems * 2};
         cuuint32_t box[4] = {kKBlock, (cuuint32_t)g.bn_real, a_parts, 1};
-        if ((rc = encode(&ma_r, L->a_bf16, 4, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&ma_r, const_cast<__nv_bfloat16*>(a_op), 4, dims, str, box)) != CIRC_OK) return rc;
     }
     {
         const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
-        cuuint64_t dims[4] = {(cuuint64_t)2 * q, (cuuint64_t)2 * p, (cuuint64_t)taps * 2, (cuuint64_t)nc};
-        cuuint64_t str[3] = {(cuuint64_t)taps * 2 * 2 * q * 2, (cuuint64_t)2 * q * 2, (cuuint64_t)4 * a_real_elems * 2};
+        // embedded: 2p rows per problem; twin: p rows of (Wr, Wi) pairs
+        cuuint64_t dims[4] = {(cuuint64_t)2 * q, (cuuint64_t)rows_c, (cuuint64_t)taps * 2, (cuuint64_t)nc};
+        cuuint64_t str[3] = {(cuuint64_t)taps * 2 * 2 * q * 2, (cuuint64_t)2 * q * 2, (cuuint64_t)(twin ? 2 : 4) * a_real_elems * 2};
         cuuint32_t box[4] = {kKBlock, (cuuint32_t)g.bn_cplx, a_parts, 1};
-        if ((rc = encode(&ma_c, L->a_bf16 + 2 * a_real_elems, 4, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&ma_c, const_cast<__nv_bfloat16*>(a_op) + 2 * a_real_elems, 4, dims, str, box)) != CIRC_OK) return rc;
     }
     // X: [problem][v][h][w][part][Kq]
     const size_t cols_in = (size_t)g.V * g.H * g.W;
@@ -721,9 +602,10 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     }
     {
         const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
-        cuuint64_t dims[5] = {(cuuint64_t)2 * q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, (cuuint64_t)nc};
-        cuuint64_t str[4] = {(cuuint64_t)nsplit * 2 * q * 2, (cuuint64_t)g.W * nsplit * 2 * q * 2,
-                             (cuuint64_t)g.H * g.W * nsplit * 2 * q * 2, (cuuint64_t)2 * x_real_elems * 2};
+        const cuuint64_t wc = (cuuint64_t)(twin ? 2 * g.W : g.W);      // twin: (Zr, -Zi) columns, then (Zi, Zr) columns
+        cuuint64_t dims[5] = {(cuuint64_t)2 * q, wc, (cuuint64_t)g.H, (cuuint64_t)g.V, (cuuint64_t)nc};
+        cuuint64_t str[4] = {(cuuint64_t)nsplit * 2 * q * 2, wc * nsplit * 2 * q * 2,
+                             (cuuint64_t)g.H * wc * nsplit * 2 * q * 2, (cuuint64_t)(twin ? 4 : 2) * x_real_elems * 2};
         cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, (cuuint32_t)(g.th + halo), 1, 1};
         __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb) + 2 * x_real_elems;
         if ((rc = encode(&mxh_c, base, 5, dims, str, box)) != CIRC_OK) return rc;
@@ -754,8 +636,10 @@ static int launch_tc_one_kind(bool real, const __nv_bfloat16* xt, int x_rows, co
     g.th = 1;
     g.xrows = g.tw;
     g.xalloc = kTileCols;
-    g.tiles_w = (x_rows + g.tw - 1) / g.tw;
+    g.tiles_w = g.tiles_w_c = (x_rows + g.tw - 1) / g.tw;
     g.tiles_h = 1;
+    g.twin = 0;
+    g.Wo_c = x_rows;
     g.cols_out = x_rows;
     int bn = round_up16(a_rows) > 256 ? 256 : round_up16(a_rows);
     const int nt = (a_rows + bn - 1) / bn;

@@ -22,8 +22,12 @@ def _forward(h, case):
     return y.cpu().numpy().astype(np.float64)
 
 
-def test_tensor_contraction_wait_runs_out_and_the_handle_recovers():
-    case = synth.fc_case("timeout_tc", 512, 512, 64, 300, w_var=1.0 / 512, x_dist="uniform")
+@pytest.mark.parametrize("shape", ["large_batch", "row_streaming"])
+def test_tensor_contraction_wait_runs_out_and_the_handle_recovers(shape):
+    if shape == "large_batch":
+        case = synth.fc_case("timeout_tc", 512, 512, 64, 300, w_var=1.0 / 512, x_dist="uniform")
+    else:
+        case = synth.fc_case("timeout_rows", 128 * 64, 512, 64, 20, w_var=1.0 / 512, x_dist="uniform")
     h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
     try:
         circ.circ_set_variant(h, circ.CIRC_VARIANT_TENSOR)
@@ -36,6 +40,8 @@ def test_tensor_contraction_wait_runs_out_and_the_handle_recovers():
         circ.circ_debug_inject(h, circ.CIRC_INJECT_NONE)
         got = _forward(h, case)
         circ.circ_device_status(h)
+        rows_kernel = circ.circ_debug_last_kernels(h)[1] in (circ.CIRC_KERNEL_S2_ROWS, circ.CIRC_KERNEL_S2_ROWS_TWIN)
+        assert rows_kernel == (shape == "row_streaming")
         assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
     finally:
         circ.circ_destroy(h)
@@ -69,7 +75,7 @@ def test_injected_allocation_failures_give_alloc_errors():
         with pytest.raises(circ.CircError) as e:
             circ.circ_fc_create(case.m, case.n, case.k, case.w)
         assert e.value.code == circ.CIRC_ERR_ALLOC
-        circ.circ_debug_fail_alloc_after(3)                 # one of the stored forms
+        circ.circ_debug_fail_alloc_after(2)                 # the packed spectra
         with pytest.raises(circ.CircError) as e:
             circ.circ_fc_create(case.m, case.n, case.k, case.w)
         assert e.value.code == circ.CIRC_ERR_ALLOC
@@ -84,6 +90,11 @@ def test_injected_allocation_failures_give_alloc_errors():
         with pytest.raises(circ.CircError) as e:
             circ.circ_fc_forward(h, x, y, case.batch, torch.cuda.current_stream())
         assert e.value.code == circ.CIRC_ERR_ALLOC and circ.circ_workspace_bytes(h) == 0
+        circ.circ_debug_fail_alloc_after(2)                 # the stored form of the staged path (built on first use)
+        weights = circ.circ_weight_bytes(h)
+        with pytest.raises(circ.CircError) as e:
+            circ.circ_fc_forward(h, x, y, case.batch, torch.cuda.current_stream())
+        assert e.value.code == circ.CIRC_ERR_ALLOC and circ.circ_weight_bytes(h) == weights
         circ.circ_debug_fail_alloc_after(0)
         assert scale_rel_err(_forward(h, case), oracle_fc(case)) <= TOL_F32
     finally:

@@ -45,6 +45,109 @@ def test_fc_tensor_bf16(k, p, q, batch):
     assert scale_rel_err(got, oracle_fc(case)) <= TOL_BF16
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("k,p,q,batch,conv", [(4, 256, 64, 64, 0), (16, 64, 16, 30, 0), (64, 32, 8, 15, 1), (256, 16, 8, 7, 0),
+                                              (8, 2048, 24, 100, 0), (32, 48, 8, 1, 1), (16, 448, 16, 200, 0)])
+def test_fc_tensor_twin_columns(k, p, q, batch, conv, bf16):
+    # many row blocks, few columns: every complex weight is stored once and multiplies two column groups of X,
+    # (Zr, -Zi) for the real parts of the result and (Zi, Zr) for the imaginary parts
+    case = synth.fc_case(f"twin_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
+                         bias_var=0.01, relu=(batch % 2 == 1), bf16_io=bf16)
+    kernels = []
+    got, used = run_fc(case, T, convention=conv, kernels=kernels)
+    assert used == T and kernels[1] in (circ.CIRC_KERNEL_S2_TENSOR_TWIN, circ.CIRC_KERNEL_S2_ROWS_TWIN), kernels
+    assert not np.isnan(got).any()
+    assert scale_rel_err(got, oracle_fc(case, conv)) <= (TOL_BF16 if bf16 else TOL_F32)
+
+
+def test_twin_and_embedded_forms_agree_and_store_half_the_weights():
+    import torch
+    case = synth.fc_case("twin_vs_embed", 64 * 64, 16 * 64, 64, 24, w_var=1.0 / 1024, x_dist="uniform")
+    outs, sizes = [], []
+    for allow in (1, 0):
+        h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
+        try:
+            base = circ.circ_weight_bytes(h)
+            assert base == 4 * case.m * case.n // case.k                  # the packed spectra and nothing else
+            circ.circ_set_variant(h, T)
+            circ.circ_debug_set_contraction(h, allow, 0)
+            x = torch.from_numpy(case.x).cuda()
+            y = torch.empty(case.batch, case.m, device="cuda")
+            circ.circ_fc_forward(h, x, y, case.batch)
+            torch.cuda.synchronize()
+            want = circ.CIRC_KERNEL_S2_TENSOR_TWIN if allow else circ.CIRC_KERNEL_S2_TENSOR
+            assert circ.circ_debug_last_kernels(h)[1] == want
+            outs.append(y.cpu().numpy().astype(np.float64))
+            sizes.append(circ.circ_weight_bytes(h) - base)
+        finally:
+            circ.circ_destroy(h)
+    assert scale_rel_err(outs[0], outs[1]) <= 1e-5
+    assert scale_rel_err(outs[0], oracle_fc(case)) <= TOL_F32
+    assert sizes[0] < 0.6 * sizes[1]                                       # one copy of every complex value against two
+
+
+ROWS_SHAPES = [(64, 128, 8, 9), (16, 512, 16, 64), (256, 32, 8, 30), (4, 2048, 64, 100), (64, 256, 8, 64), (16, 520, 24, 128),
+               (32, 300, 8, 1), (8, 1100, 40, 17)]
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("k,p,q,batch", ROWS_SHAPES)
+def test_fc_tensor_row_streaming(k, p, q, batch, bf16):
+    # many row blocks, at most 256 columns: weight rows on the 128-row side of the MMA, all columns in one tile;
+    # ragged last row tile, ragged contraction tail, odd batches, with and without twin columns
+    case = synth.fc_case(f"rows_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
+                         bias_var=0.01, relu=(batch % 2 == 0), bf16_io=bf16)
+    ref = oracle_fc(case)
+    import torch
+    from gpu_helpers import to_device
+    for allow_twin in (1, 0):
+        h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
+        try:
+            circ.circ_set_bias(h, case.bias)
+            circ.circ_set_activation(h, int(case.relu))
+            code = circ.CIRC_BF16 if bf16 else circ.CIRC_F32
+            circ.circ_set_io_dtype(h, code, code)
+            circ.circ_set_variant(h, T)
+            circ.circ_debug_set_contraction(h, allow_twin, 1)
+            x = to_device(case.x, bf16)
+            y = torch.full((batch, case.m), float("nan"), device="cuda", dtype=torch.bfloat16 if bf16 else torch.float32)
+            circ.circ_fc_forward(h, x, y, batch)
+            torch.cuda.synchronize()
+            circ.circ_device_status(h)
+            kern = circ.circ_debug_last_kernels(h)[1]
+            assert kern in (circ.CIRC_KERNEL_S2_ROWS, circ.CIRC_KERNEL_S2_ROWS_TWIN), kern
+            if not allow_twin:
+                assert kern == circ.CIRC_KERNEL_S2_ROWS
+            got = y.float().cpu().numpy().astype(np.float64)
+            assert not np.isnan(got).any()
+            assert scale_rel_err(got, ref) <= (TOL_BF16 if bf16 else TOL_F32)
+        finally:
+            circ.circ_destroy(h)
+
+
+def test_stored_forms_are_built_on_first_use():
+    import torch
+    case = synth.fc_case("lazy_forms", 4096, 4096, 4, 1, w_var=1.0 / 4096, x_dist="uniform")
+    h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
+    try:
+        alg = 4 * case.m * case.n // case.k
+        x = torch.from_numpy(case.x).cuda()
+        y = torch.empty(1, case.m, device="cuda")
+        circ.circ_fc_forward(h, x, y, 1)                                   # the one-launch kernel reads the packed spectra
+        torch.cuda.synchronize()
+        assert circ.circ_last_variant(h) == circ.CIRC_VARIANT_FUSED
+        assert circ.circ_weight_bytes(h) + circ.circ_workspace_bytes(h) <= 1.1 * alg
+        assert scale_rel_err(y.cpu().numpy().astype(np.float64), oracle_fc(case)) <= TOL_F32
+        xb = torch.from_numpy(np.tile(case.x, (40, 1))).cuda()
+        yb = torch.empty(40, case.m, device="cuda")
+        circ.circ_fc_forward(h, xb, yb, 40)                                # the tensor path builds its own form now
+        torch.cuda.synchronize()
+        assert circ.circ_weight_bytes(h) > alg
+        assert torch.allclose(yb[0], y[0], rtol=0, atol=1e-4 * float(y.abs().max()))
+    finally:
+        circ.circ_destroy(h)
+
+
 def test_config2_b256_uses_tensor_cores():
     case = synth.config2(256)
     got, used = run_fc(case)
