@@ -192,7 +192,7 @@ static size_t x_operand_floats(const Layer* L, const Extent& e) {
 // Copies of Y: the row-streaming contraction writes one per piece of its contraction range.
 static size_t y_copies(const Layer* L, const Extent& e) {
     const ContractionPlan pl = plan_contraction(L, e);
-    return pl.rows ? (size_t)rows_pieces(L, pl.twin).cplx : 1;
+    return pl.rows ? (size_t)rows_pieces(L, e, pl.twin).cplx : 1;
 }
 
 static size_t workspace_need(const Layer* L, const Extent& e) {
@@ -315,7 +315,7 @@ int stage_contract(Layer* L, const float* xop, float* yop, const Extent& e, cuda
 
 int stage_output(Layer* L, const float* yop, void* y, const Extent& e, cudaStream_t stream, bool tensor) {
     const ContractionPlan pl = tensor ? plan_contraction(L, e) : ContractionPlan{false, false};
-    return launch_output_ifft(L, yop, y, e, stream, false, pl.twin, pl.rows ? rows_pieces(L, pl.twin) : RowsPieces{0, 0});
+    return launch_output_ifft(L, yop, y, e, stream, false, pl.twin, pl.rows ? rows_pieces(L, e, pl.twin) : RowsPieces{0, 0});
 }
 
 static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStream_t stream, bool tensor) {

@@ -231,7 +231,7 @@ int launch_contract_rows(const Layer* L, const __nv_bfloat16* xb, float* yop, co
 struct RowsPieces {
     int real, cplx;
 };
-RowsPieces rows_pieces(const Layer* L, bool twin);
+RowsPieces rows_pieces(const Layer* L, const Extent& e, bool twin);
 // Loads the fixed scratch array of the allocation-free entry point and caches its address (circ_noalloc.cu).
 int noalloc_warm();
 // Rounds w_stream into w_stream_bf16 (which must be allocated).

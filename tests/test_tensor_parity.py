@@ -46,7 +46,7 @@ def test_fc_tensor_bf16(k, p, q, batch):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
-@pytest.mark.parametrize("k,p,q,batch,conv", [(4, 256, 64, 64, 0), (16, 64, 16, 30, 0), (64, 32, 8, 15, 1), (256, 16, 8, 7, 0),
+@pytest.mark.parametrize("k,p,q,batch,conv", [(4, 256, 64, 64, 0), (16, 64, 16, 30, 0), (64, 32, 8, 15, 1), (128, 16, 8, 7, 0),
                                               (8, 2048, 24, 100, 0), (32, 48, 8, 1, 1), (16, 448, 16, 200, 0)])
 def test_fc_tensor_twin_columns(k, p, q, batch, conv, bf16):
     # many row blocks, few columns: every complex weight is stored once and multiplies two column groups of X,
