@@ -97,6 +97,10 @@ CIRC_API int circ_debug_set_fused_split(circ_handle h, int slices);
  * weight stored once, X twice); allow_rows = 0: never the row-streaming kernel.  1 / 1 (default): the planner decides. */
 CIRC_API int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows);
 
+/* circ_debug_set_transforms -- allow_bulk_input = 0: the input transforms of this handle never take the kernel that
+ * stages its tiles by bulk copies (the load-based kernel serves every size); 1 (default): the planner decides. */
+CIRC_API int circ_debug_set_transforms(circ_handle h, int allow_bulk_input);
+
 /* circ_debug_fail_alloc_after -- the n-th device allocation the library makes from now on fails as if the
  * device were out of memory (n = 1: the next one); n <= 0 cancels.  Exercises the CIRC_ERR_ALLOC paths. */
 CIRC_API int circ_debug_fail_alloc_after(long n);

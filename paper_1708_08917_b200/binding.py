@@ -67,6 +67,7 @@ SIGNATURES = {
     "circ_debug_fail_alloc_after": (_ci, [_cl]),
     "circ_debug_set_fused_split": (_ci, [_vp, _ci]),
     "circ_debug_set_contraction": (_ci, [_vp, _ci, _ci]),
+    "circ_debug_set_transforms": (_ci, [_vp, _ci]),
     "circ_last_error": (ctypes.c_char_p, []),
     "circ_last_code": (_ci, []),
 }
@@ -320,6 +321,10 @@ def circ_debug_set_fused_split(h: int, slices: int) -> None:
 
 def circ_debug_set_contraction(h: int, allow_twin: int, allow_rows: int) -> None:
     _check(load().circ_debug_set_contraction(h, int(allow_twin), int(allow_rows)))
+
+
+def circ_debug_set_transforms(h: int, allow_bulk_input: int) -> None:
+    _check(load().circ_debug_set_transforms(h, int(allow_bulk_input)))
 
 
 def circ_debug_fail_alloc_after(n: int) -> None:

@@ -101,6 +101,7 @@ struct Layer {
     size_t x_stage_bytes, y_stage_bytes;
     mutable int last_kernels[3];  // which S1 / S2 / S3 kernel served the most recent staged forward (KERNEL_* ids below)
     int inject;           // test-only fault injection (circ_debug.h): 0 = none
+    int no_bulk_input;    // 1: never use the bulk-staged input transforms (circ_debug_set_transforms)
     int no_rows_kernel;   // 1: never use the row-streaming tensor-core contraction (circ_debug_set_contraction)
     int no_twin;          // 1: never use the twin-column form of the tensor contraction (circ_debug_set_twin)
     int fused_split;      // column slices of the one-launch kernel forced by circ_debug_set_fused_split (0 = planner's choice)
@@ -241,6 +242,10 @@ int launch_round_stream(Layer* L, cudaStream_t stream);
 // 1: bfloat16 [problem][col][hi | lo][Kq] (split of float32 values); 2: bfloat16 [problem][col][Kq].
 // `twin` (xmode 1 / 2, fully-connected): complex problems get two column groups, (Zr, -Zi) and (Zi, Zr).
 int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream, bool twin = false);
+
+// S1 for large forwards (circ_input_bulk.cu): tiles staged by bulk copies, one exchange through shared memory.
+bool input_fft_bulk_supported(const Layer* L, const void* x, long total);
+int launch_input_fft_bulk(const Layer* L, const void* x, void* xop, int xmode, bool twin, const Extent& ext, cudaStream_t stream);
 
 // S2 / C2 on the float32 FMA pipes: Y = A . X per problem.
 int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream);

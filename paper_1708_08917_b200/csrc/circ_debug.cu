@@ -154,6 +154,16 @@ int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows) {
     return CIRC_OK;
 }
 
+int circ_debug_set_transforms(circ_handle h, int allow_bulk_input) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || (allow_bulk_input != 0 && allow_bulk_input != 1)) {
+        set_error(CIRC_ERR_ARG, "bad handle or flag %d", allow_bulk_input);
+        return CIRC_ERR_ARG;
+    }
+    L->no_bulk_input = !allow_bulk_input;
+    return CIRC_OK;
+}
+
 int circ_debug_fail_alloc_after(long n) {
     fail_alloc_after(n);
     return CIRC_OK;

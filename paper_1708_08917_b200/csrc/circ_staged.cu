@@ -57,18 +57,6 @@ __device__ __forceinline__ void split_at(Split s, int d, int rows, int& c, int& 
     }
 }
 
-__device__ __forceinline__ uint32_t bf16_pair(float lo, float hi) {
-    const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<const uint32_t*>(&t);
-}
-// Split two float32 values into bfloat16 high parts (returned, packed) and low parts (`lo_pair`):
-// v = hi + lo up to 2^-17 relative, which is what the three-pass tensor-core product needs.
-__device__ __forceinline__ uint32_t bf16_split_pair(float a, float b, uint32_t& lo_pair) {
-    const uint32_t hi = bf16_pair(a, b);
-    lo_pair = bf16_pair(a - __uint_as_float(hi << 16), b - __uint_as_float(hi & 0xffff0000u));
-    return hi;
-}
-
 // Operand Y -> tile (the first half of S3): fills zs[bin][transform] for the CTA's TT transforms.
 // TWIN: Y of a complex problem holds the real parts of all 2 Bho columns, then the imaginary parts (p rows each),
 // instead of 2p interleaved rows.
@@ -777,6 +765,8 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
         return CIRC_ERR_UNSUPPORTED;
     }
     const bool small = latency_bound(total, L->geo.k);
+    // large forwards of power-of-two blocks from 16 to 256: tiles staged by bulk copies, exchange through shared memory
+    if (!small && !L->no_bulk_input && input_fft_bulk_supported(L, x, total)) return launch_input_fft_bulk(L, x, xop, xmode, twin, ext, stream);
     auto go = [&](auto kc) -> int {
         constexpr int K = decltype(kc)::value;
         auto with_shape = [&](auto ec) {
