@@ -323,8 +323,9 @@ def sets_needed(per_set_bytes: int, max_sets: int) -> int:
     return int(min(max_sets, max(2, -(-2 * L2_BYTES // max(per_set_bytes, 1)) + 1)))
 
 
-def own_bytes(wl: Workload, variant: int, circ) -> dict:
-    """Bytes each kernel of the path reads and writes itself (its operands), per forward."""
+def own_bytes(wl: Workload, variant: int, circ, s2_kernel: int = 0) -> dict:
+    """Bytes each kernel of the path reads and writes itself (its operands), per forward; `s2_kernel` is the
+    CIRC_KERNEL_* id of the contraction that ran (it fixes the stored form of the weights and the layout of X)."""
     c = wl.case
     if wl.kind == "stack":
         return {}
@@ -341,13 +342,17 @@ def own_bytes(wl: Workload, variant: int, circ) -> dict:
     if variant == circ.CIRC_VARIANT_FUSED:
         return {"fused_fc": wl.alg_bytes}
     tensor = variant == circ.CIRC_VARIANT_TENSOR
+    twin = s2_kernel in (circ.CIRC_KERNEL_S2_TENSOR_TWIN, circ.CIRC_KERNEL_S2_ROWS_TWIN)
     xhat = cols_in * n * (2 if (tensor and c.bf16_io) else 4)          # float32, split bfloat16 (hi + lo), or bfloat16
+    if twin:
+        xhat = int(xhat * (2.0 - 2.0 / k))                              # the complex problems' columns twice
     yhat = cols_out * m * 4
-    spectra = taps * m * n // k                                         # complex-pair count x 2 = real values of the half spectra
+    spectra = taps * m * n // k                                         # real values of the half spectra
     if tensor:
-        a_b = spectra * 2 * (2 if c.bf16_io else 4)                     # embedded [Wr -Wi; Wi Wr]: twice the values; hi (+ lo) bfloat16
+        part_bytes = 2 if c.bf16_io else 4                              # hi (+ lo) bfloat16
+        a_b = spectra * part_bytes if twin else int(spectra * (2.0 - 2.0 / k)) * part_bytes   # embedded [Wr -Wi; Wi Wr]: complex values twice
     else:
-        a_b = spectra * 2 * 4
+        a_b = int(spectra * (2.0 - 2.0 / k)) * 4
     return {"input_fft": x_b + xhat, "contraction": xhat + yhat + a_b, "output_ifft": yhat + y_b}
 
 
@@ -665,7 +670,8 @@ def run_ours(args) -> int:
         for st_i in used_stages:
             rep_ms, _, _ = timer.time_steps(job, ksteps, cold=True, min_s=0.25, min_reps=10, max_s=1.5, stage=st_i, times=1 + R)
             stage_us[STAGES[st_i]] = max(0.0, 1e3 * (rep_ms - base_ms) / (R * ksteps))
-    ob = own_bytes(wl, variant, circ)
+    s2_kernel = circ.circ_debug_last_kernels(job.first_handle())[1] if wl.kind != "stack" else 0
+    ob = own_bytes(wl, variant, circ, s2_kernel)
     kernels = {}
     for kname, us_k in stage_us.items():
         ent = {"us": us_k, "own_bytes": ob.get(kname), "l2_warm": bool(ob.get(kname, 0) < L2_BYTES)}
@@ -690,7 +696,7 @@ def run_ours(args) -> int:
                 "algorithmic_bytes_per_step": wl.alg_bytes, "contraction_flops_per_step": wl.contraction_flops,
                 "hbm_frac_of_measured": wl.alg_bytes / (ms_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
                 "hbm_frac_of_nominal_8000": wl.alg_bytes / (ms_step * 1e-3) / 1e9 / 8000.0,
-                "kernel": dom, "kernels": kernels,
+                "kernel": dom, "kernels": kernels, "kernel_ids": (circ.circ_debug_last_kernels(job.first_handle()) if wl.kind != "stack" else None),
                 "kernel_frac": (kernels.get(dom, {}).get("frac_of_tensor") if rf["bound"] == "tensor" and dom == "contraction"
                                 else kernels.get(dom, {}).get("frac_of_hbm")),
                 "kernel_note": "per-kernel durations are differences between graphs with that kernel launched 4x and 1x per forward: "

@@ -28,7 +28,7 @@ enum {
 enum {
     CIRC_KERNEL_NONE = 0,
     CIRC_KERNEL_S1_LOADS = 1,   /* input transforms fed by per-thread vector loads */
-    CIRC_KERNEL_S1_BULK = 2,    /* input transforms fed by bulk asynchronous copies into shared memory */
+    CIRC_KERNEL_S1_BULK = 2,    /* input transforms fed by TMA copies into shared memory */
     CIRC_KERNEL_S2_FMA = 10,    /* contraction on the float32 FMA pipes */
     CIRC_KERNEL_S2_TENSOR = 11, /* contraction on the tensor cores, weights in the embedded real form [Wr -Wi; Wi Wr] */
     CIRC_KERNEL_S2_TENSOR_TWIN = 12, /* contraction on the tensor cores, every complex weight stored once (twin column groups of X) */
@@ -36,6 +36,7 @@ enum {
     CIRC_KERNEL_S2_ROWS_TWIN = 14, /* row-streaming tensor-core contraction with twin columns */
     CIRC_KERNEL_S3_LOADS = 20,  /* inverse transforms fed by per-thread loads */
     CIRC_KERNEL_S3_BULK = 21,   /* inverse transforms fed by bulk asynchronous copies */
+    CIRC_KERNEL_S3_TMA = 22,    /* inverse transforms with one exchange through shared memory, output written by TMA */
     CIRC_KERNEL_S4_FUSED = 30   /* the one-launch small-batch kernel */
 };
 
@@ -97,9 +98,10 @@ CIRC_API int circ_debug_set_fused_split(circ_handle h, int slices);
  * weight stored once, X twice); allow_rows = 0: never the row-streaming kernel.  1 / 1 (default): the planner decides. */
 CIRC_API int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows);
 
-/* circ_debug_set_transforms -- allow_bulk_input = 0: the input transforms of this handle never take the kernel that
- * stages its tiles by bulk copies (the load-based kernel serves every size); 1 (default): the planner decides. */
-CIRC_API int circ_debug_set_transforms(circ_handle h, int allow_bulk_input);
+/* circ_debug_set_transforms -- allow_tma_input = 0: the input transforms of this handle never take the kernel that
+ * stages its tiles by TMA (the load-based kernel serves every size); allow_tma_output = 0: likewise for the inverse
+ * transforms that write their tiles by TMA.  1 / 1 (default): the planner decides. */
+CIRC_API int circ_debug_set_transforms(circ_handle h, int allow_tma_input, int allow_tma_output);
 
 /* circ_debug_fail_alloc_after -- the n-th device allocation the library makes from now on fails as if the
  * device were out of memory (n = 1: the next one); n <= 0 cancels.  Exercises the CIRC_ERR_ALLOC paths. */

@@ -24,6 +24,7 @@ CIRC_STAGE_INPUT_FFT, CIRC_STAGE_CONTRACTION, CIRC_STAGE_OUTPUT_IFFT, CIRC_STAGE
 CIRC_KERNEL_NONE, CIRC_KERNEL_S1_LOADS, CIRC_KERNEL_S1_BULK = 0, 1, 2
 CIRC_KERNEL_S2_TENSOR_TWIN, CIRC_KERNEL_S2_ROWS, CIRC_KERNEL_S2_ROWS_TWIN = 12, 13, 14
 CIRC_KERNEL_S2_FMA, CIRC_KERNEL_S2_TENSOR, CIRC_KERNEL_S3_LOADS, CIRC_KERNEL_S3_BULK, CIRC_KERNEL_S4_FUSED = 10, 11, 20, 21, 30
+CIRC_KERNEL_S3_TMA = 22
 CIRC_INJECT_NONE, CIRC_INJECT_TENSOR_NO_COPY, CIRC_INJECT_BULK_NO_COPY = 0, 1, 2
 
 # name -> (restype, argtypes); mirrors include/circ.h one to one
@@ -67,7 +68,7 @@ SIGNATURES = {
     "circ_debug_fail_alloc_after": (_ci, [_cl]),
     "circ_debug_set_fused_split": (_ci, [_vp, _ci]),
     "circ_debug_set_contraction": (_ci, [_vp, _ci, _ci]),
-    "circ_debug_set_transforms": (_ci, [_vp, _ci]),
+    "circ_debug_set_transforms": (_ci, [_vp, _ci, _ci]),
     "circ_last_error": (ctypes.c_char_p, []),
     "circ_last_code": (_ci, []),
 }
@@ -323,8 +324,8 @@ def circ_debug_set_contraction(h: int, allow_twin: int, allow_rows: int) -> None
     _check(load().circ_debug_set_contraction(h, int(allow_twin), int(allow_rows)))
 
 
-def circ_debug_set_transforms(h: int, allow_bulk_input: int) -> None:
-    _check(load().circ_debug_set_transforms(h, int(allow_bulk_input)))
+def circ_debug_set_transforms(h: int, allow_tma_input: int, allow_tma_output: int = 1) -> None:
+    _check(load().circ_debug_set_transforms(h, int(allow_tma_input), int(allow_tma_output)))
 
 
 def circ_debug_fail_alloc_after(n: int) -> None:

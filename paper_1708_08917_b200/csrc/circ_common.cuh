@@ -101,11 +101,17 @@ struct Layer {
     size_t x_stage_bytes, y_stage_bytes;
     mutable int last_kernels[3];  // which S1 / S2 / S3 kernel served the most recent staged forward (KERNEL_* ids below)
     int inject;           // test-only fault injection (circ_debug.h): 0 = none
-    int no_bulk_input;    // 1: never use the bulk-staged input transforms (circ_debug_set_transforms)
+    int no_bulk_input;    // 1: never use the TMA-staged input transforms (circ_debug_set_transforms)
+    int no_tma_output;    // 1: never use the TMA-written inverse transforms (circ_debug_set_transforms)
     int no_rows_kernel;   // 1: never use the row-streaming tensor-core contraction (circ_debug_set_contraction)
     int no_twin;          // 1: never use the twin-column form of the tensor contraction (circ_debug_set_twin)
     int fused_split;      // column slices of the one-launch kernel forced by circ_debug_set_fused_split (0 = planner's choice)
     Layer* transposed;  // the n x m layer W^T (built on first use by the backward pass), or nullptr
+};
+
+// Copies of Y that the row-streaming contraction writes for a real / a complex problem ({0, 0}: Y is a single array).
+struct RowsPieces {
+    int real, cplx;
 };
 
 // Kernel ids recorded in Layer::last_kernels (read back through circ_debug_last_kernels).
@@ -120,6 +126,7 @@ enum {
     KERNEL_S2_ROWS_TWIN = 14, // the same with twin columns
     KERNEL_S3_LOADS = 20,     // inverse transforms, per-thread loads
     KERNEL_S3_BULK = 21,      // inverse transforms, tiles staged by bulk asynchronous copies
+    KERNEL_S3_TMA = 22,       // inverse transforms, one exchange through shared memory, output tile written by TMA
     KERNEL_S4_FUSED = 30      // the one-launch kernel: last_kernels = {this id, column slices, row blocks per thread block}
 };
 
@@ -229,9 +236,6 @@ inline bool use_twin(const Layer* L, const Extent& e) { return plan_contraction(
 int launch_contract_rows(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin);
 // Copies of Y that the row-streaming contraction writes for a real / a complex problem; the inverse-transform kernel
 // adds them up.  {0, 0}: Y is a single array.
-struct RowsPieces {
-    int real, cplx;
-};
 RowsPieces rows_pieces(const Layer* L, const Extent& e, bool twin);
 // Loads the fixed scratch array of the allocation-free entry point and caches its address (circ_noalloc.cu).
 int noalloc_warm();
@@ -246,6 +250,10 @@ int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const 
 // S1 for large forwards (circ_input_bulk.cu): tiles staged by bulk copies, one exchange through shared memory.
 bool input_fft_bulk_supported(const Layer* L, const void* x, long total);
 int launch_input_fft_bulk(const Layer* L, const void* x, void* xop, int xmode, bool twin, const Extent& ext, cudaStream_t stream);
+
+// S3 for large forwards (circ_output_bulk.cu): one exchange through shared memory, output tiles written by TMA.
+bool output_ifft_tma_supported(const Layer* L, const void* y, const Extent& ext);
+int launch_output_ifft_tma(const Layer* L, const float* yop, void* y, const Extent& ext, cudaStream_t stream);
 
 // S2 / C2 on the float32 FMA pipes: Y = A . X per problem.
 int launch_contract_fma(const Layer* L, const float* xop, float* yop, const Extent& ext, cudaStream_t stream);

@@ -10,7 +10,7 @@ static_assert((int)CIRC_KERNEL_S1_LOADS == (int)KERNEL_S1_LOADS && (int)CIRC_KER
                   (int)CIRC_KERNEL_S2_TENSOR_TWIN == (int)KERNEL_S2_TENSOR_TWIN && (int)CIRC_KERNEL_S2_ROWS == (int)KERNEL_S2_ROWS &&
                   (int)CIRC_KERNEL_S2_ROWS_TWIN == (int)KERNEL_S2_ROWS_TWIN &&
                   (int)CIRC_KERNEL_S3_LOADS == (int)KERNEL_S3_LOADS && (int)CIRC_KERNEL_S3_BULK == (int)KERNEL_S3_BULK &&
-                  (int)CIRC_KERNEL_S4_FUSED == (int)KERNEL_S4_FUSED,
+                  (int)CIRC_KERNEL_S4_FUSED == (int)KERNEL_S4_FUSED && (int)CIRC_KERNEL_S3_TMA == (int)KERNEL_S3_TMA,
               "public and internal kernel ids must agree");
 static_assert((int)CIRC_INJECT_TENSOR_NO_COPY == (int)INJECT_TENSOR_NO_COPY && (int)CIRC_INJECT_BULK_NO_COPY == (int)INJECT_BULK_NO_COPY,
               "public and internal injection kinds must agree");
@@ -154,13 +154,14 @@ int circ_debug_set_contraction(circ_handle h, int allow_twin, int allow_rows) {
     return CIRC_OK;
 }
 
-int circ_debug_set_transforms(circ_handle h, int allow_bulk_input) {
+int circ_debug_set_transforms(circ_handle h, int allow_tma_input, int allow_tma_output) {
     Layer* L = reinterpret_cast<Layer*>(h);
-    if (!L || (allow_bulk_input != 0 && allow_bulk_input != 1)) {
-        set_error(CIRC_ERR_ARG, "bad handle or flag %d", allow_bulk_input);
+    if (!L || (allow_tma_input != 0 && allow_tma_input != 1) || (allow_tma_output != 0 && allow_tma_output != 1)) {
+        set_error(CIRC_ERR_ARG, "bad handle or flags %d, %d", allow_tma_input, allow_tma_output);
         return CIRC_ERR_ARG;
     }
-    L->no_bulk_input = !allow_bulk_input;
+    L->no_bulk_input = !allow_tma_input;
+    L->no_tma_output = !allow_tma_output;
     return CIRC_OK;
 }
 

@@ -111,6 +111,14 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     return d;
 }
 
+// Bounded wait without an abort flag: false when the phase never completes.
+__device__ __forceinline__ bool mbar_wait_plain(uint64_t* bar, uint32_t parity, uint32_t limit = kSpinLimit) {
+    for (uint32_t it = 0; it < limit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (it > 64) __nanosleep(64);
+    }
+    return false;
+}
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -133,7 +141,8 @@ inline EncodeTiledFn tensor_map_encoder() {
 }
 
 inline int encode_tensor_map(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
-                  const cuuint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16) {
+                  const cuuint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                  CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = tensor_map_encoder();
     if (!fn) {
         set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
@@ -141,7 +150,7 @@ inline int encode_tensor_map(CUtensorMap* map, void* base, int rank, const cuuin
     }
     cuuint32_t ones[5] = {1, 1, 1, 1, 1};
     const CUresult r = fn(map, dtype, (cuuint32_t)rank, base, dims, strides_bytes, box, ones,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);

@@ -23,7 +23,7 @@ def _run(case, allow_bulk, variant=circ.CIRC_VARIANT_AUTO):
         code = circ.CIRC_BF16 if case.bf16_io else circ.CIRC_F32
         circ.circ_set_io_dtype(h, code, code)
         circ.circ_set_variant(h, variant)
-        circ.circ_debug_set_transforms(h, allow_bulk)
+        circ.circ_debug_set_transforms(h, allow_bulk, 1)
         x = to_device(case.x, case.bf16_io)
         y = torch.full((case.batch, case.m), float("nan"), device="cuda", dtype=torch.bfloat16 if case.bf16_io else torch.float32)
         circ.circ_fc_forward(h, x, y, case.batch)
