@@ -70,8 +70,9 @@ template <int K, typename TOUT>
 __global__ void __launch_bounds__(OutBulk<K, TOUT>::NT)
 output_ifft_tma_kernel(const __grid_constant__ CUtensorMap map_yc, const __grid_constant__ CUtensorMap map_yr,
                        const __grid_constant__ CUtensorMap map_y, const float* __restrict__ bias, int relu, int p, int Bho, int ntiles,
-                       int* status, int pdl_late) {
+                       int* status, int pdl_late, int no_copy) {
     using S = OutBulk<K, TOUT>;
+    const uint32_t spin_limit = no_copy ? (1u << 12) : kSpinLimit;   // no_copy: fault injection (tests only)
     constexpr int L2 = S::L2, R1 = S::R1, E2 = S::E2, TT = S::TT, NC = S::NC;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* in0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
@@ -115,6 +116,7 @@ output_ifft_tma_kernel(const __grid_constant__ CUtensorMap map_yc, const __grid_
         tile_origin(tile, c0, i0);
         unsigned char* dst = in0 + (size_t)b * S::IN;
         mbar_expect_tx(&full[b], (uint32_t)S::IN_RAW);
+        if (no_copy) return;                             // the bytes were announced, nothing is in flight: the wait runs out
         tma_load_4d(dst, &map_yc, &full[b], 2 * i0, c0, 0, 0);
         tma_load_4d(dst + S::IN_C, &map_yc, &full[b], 2 * i0, Bho + c0, 0, 0);
         tma_load_4d(dst + 2 * S::IN_C, &map_yr, &full[b], i0, c0, 0, 0);
@@ -132,7 +134,7 @@ output_ifft_tma_kernel(const __grid_constant__ CUtensorMap map_yc, const __grid_
         unsigned char* out = out0 + (size_t)(S::NOUT == 2 ? b : 0) * S::OUT;
         int c0, i0;
         tile_origin(tile, c0, i0);
-        ok = mbar_wait_plain(&full[b], (uint32_t)(it >> 1) & 1u);
+        ok = mbar_wait_plain(&full[b], (uint32_t)(it >> 1) & 1u, spin_limit);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         // ---- this thread's bins: Y[f2 + L2 f1] of transform `lane`, then pass A ----------------------------------
@@ -217,8 +219,10 @@ output_ifft_tma_kernel(const __grid_constant__ CUtensorMap map_yc, const __grid_
     if (!ok) {
         // a wait gave up: report it, and give the copies in flight a bounded wait to land before the memory goes away
         if (tid == 0) atomicExch(status, 1);
-        mbar_wait_plain(&full[it & 1], (uint32_t)(it >> 1) & 1u);
-        mbar_wait_plain(&full[(it + 1) & 1], (uint32_t)((it + 1) >> 1) & 1u);
+        if (!no_copy) {
+            mbar_wait_plain(&full[it & 1], (uint32_t)(it >> 1) & 1u, 1u << 16);
+            mbar_wait_plain(&full[(it + 1) & 1], (uint32_t)((it + 1) >> 1) & 1u, 1u << 16);
+        }
     }
 }
 
@@ -280,7 +284,8 @@ static int launch_one(const Layer* L, const float* yop, void* y, const Extent& e
     const long resident = (long)sms * per_sm;
     const unsigned blocks = (unsigned)(ntiles < resident ? ntiles : resident);
     launch_kernel(dependent_launches(), kernel, dim3(blocks), dim3(S::NT), S::SMEM, stream, map_yc, map_yr, map_y,
-                  static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bho, (int)ntiles, L->dev_status, (int)(dependent_launches() == PDL_LATE));
+                  static_cast<const float*>(L->bias_dev), L->relu, p, ext.Bho, (int)ntiles, L->dev_status, (int)(dependent_launches() == PDL_LATE),
+                  (int)(L->inject == INJECT_BULK_NO_COPY));
     return CIRC_OK;
 }
 

@@ -47,21 +47,23 @@ def test_tensor_contraction_wait_runs_out_and_the_handle_recovers(shape):
         circ.circ_destroy(h)
 
 
-def test_bulk_fed_inverse_transform_wait_runs_out_and_the_handle_recovers():
-    # 3000 pairs x 16 row blocks = 48000 transforms: large enough for the bulk-fed kernel
-    case = synth.fc_case("timeout_bulk", 16 * 64, 8 * 64, 64, 6000, w_var=1.0 / 512, x_dist="normal")
+@pytest.mark.parametrize("batch", [6000, 6002])
+def test_bulk_fed_inverse_transform_wait_runs_out_and_the_handle_recovers(batch):
+    # 3000 pairs x 16 row blocks = 48000 transforms: large enough for the kernels that stage their tiles by asynchronous
+    # copies (whole tiles of two pairs: the TMA kernel; 3001 pairs: the bulk-copy kernel)
+    case = synth.fc_case("timeout_bulk", 16 * 64, 8 * 64, 64, batch, w_var=1.0 / 512, x_dist="normal")
     h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
     try:
         circ.circ_debug_inject(h, circ.CIRC_INJECT_BULK_NO_COPY)
         _forward(h, case)
-        assert circ.circ_debug_last_kernels(h)[2] == circ.CIRC_KERNEL_S3_BULK
+        assert circ.circ_debug_last_kernels(h)[2] in (circ.CIRC_KERNEL_S3_BULK, circ.CIRC_KERNEL_S3_TMA)
         with pytest.raises(circ.CircError) as e:
             circ.circ_device_status(h)
         assert e.value.code == circ.CIRC_ERR_DEVICE_TIMEOUT
         circ.circ_debug_inject(h, circ.CIRC_INJECT_NONE)
         got = _forward(h, case)
         circ.circ_device_status(h)
-        rows = [0, 1, 2999, 3000, 5999]
+        rows = [0, 1, 2999, 3000, batch - 1]
         ref = oracle.fc(case.w, case.x[rows])
         assert scale_rel_err(got[rows], ref) <= TOL_F32
     finally:
