@@ -101,8 +101,11 @@ def workload(name: str) -> Workload:
 
     def fc(case, desc, w16=False):
         s = 2 if case.bf16_io else 4
-        alg = (2 if w16 else 4) * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
         p, q = case.m // case.k, case.n // case.k
+        # bytes per stored spectrum value: with bfloat16 activations the tensor-core path (batch > 8, q a multiple of 8)
+        # multiplies by, and therefore stores, bfloat16 spectra; every other path reads float32 ones (or _w16's bfloat16)
+        s_w = 2 if (w16 or (case.bf16_io and case.batch > 8 and q % 8 == 0)) else 4
+        alg = s_w * case.m * case.n // case.k + s * case.batch * (case.n + case.m) + (4 * case.m if case.bias is not None else 0)
         return Workload(name, desc, "fc", case, case.batch, alg, 2.0 * case.m * case.n * case.batch, s, s,
                         float(p) * q * case.batch * (4 * case.k - 4), fft_flops(case.m, case.n, case.k, case.batch), w16)
 
@@ -140,7 +143,7 @@ def workload(name: str) -> Workload:
     if name == "cfg4":
         c = synth.config4()
         pix = c.N * c.H * c.W
-        alg = 4 * c.r * c.r * c.c_out * c.c_in // c.k + 2 * pix * (c.c_in + c.c_out)
+        alg = 2 * c.r * c.r * c.c_out * c.c_in // c.k + 2 * pix * (c.c_in + c.c_out)     # bfloat16 spectra, bfloat16 pixels
         return Workload(name, "CONV 3x3 pad 1, 256->256 ch, 28x28, batch 32, k=16, bf16 activations", "conv", c, c.N, alg,
                         2.0 * pix * c.r * c.r * c.c_in * c.c_out, 2, 2,
                         float(c.r * c.r) * (c.c_out // c.k) * (c.c_in // c.k) * pix * (4 * c.k - 4),

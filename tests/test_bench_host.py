@@ -24,9 +24,13 @@ def test_workload_accounting():
     assert w.dense_flops == 2.0 * 4096 * 4096 * 256 and w.samples == 256
     c4 = bench.workload("cfg4")
     assert c4.kind == "conv" and c4.samples == 32
-    assert c4.alg_bytes == 4 * 9 * 256 * 256 // 16 + 2 * 32 * 28 * 28 * 512
+    assert c4.alg_bytes == 2 * 9 * 256 * 256 // 16 + 2 * 32 * 28 * 28 * 512      # bfloat16 spectra and pixels
     s = bench.workload("sweep_n1024_k16_b64_bf16")
     assert s.case.bf16_io and s.sx == 2 and s.case.w.shape == (64, 64, 16)
+    # bfloat16 activations on the tensor path: the stored spectra are bfloat16 too; the one-launch kernel reads float32 ones
+    assert s.alg_bytes == 2 * 1024 * 1024 // 16 + 2 * 64 * 2048
+    assert bench.workload("sweep_n1024_k16_b1_bf16").alg_bytes == 4 * 1024 * 1024 // 16 + 2 * 1 * 2048
+    assert bench.workload("sweep_n1024_k256_b64_bf16").alg_bytes == 4 * 1024 * 1024 // 256 + 2 * 64 * 2048   # q = 4: FMA path
     l2 = bench.workload("cfg3_l2")
     assert (l2.case.m, l2.case.n, l2.case.k, l2.case.batch) == (1024, 4096, 128, 128) and l2.case.x.shape == (128, 4096)
     with pytest.raises(SystemExit):
