@@ -57,6 +57,18 @@ TABLE_ROWS = (["cfg1", "cfg2_b1", "cfg2_b16", "cfg2_b256", "cfg3_stack", "cfg4"]
 # when the source has changed since, the figure is withheld (reported as null).  These are builder-run
 # captures (profiles/), not counters read during this run: `traffic_source` in the JSON line says so.
 NCU_TRAFFIC: dict = {
+    ("sweep_n16384_k4_b1024", "contraction"): {"bytes_per_launch": 591302144 + 58379520,
+                                               "source_sha256": "532dd6636825660d699b29a99ea6b13901970957b3ada4df54019b00538078ac"},
+    ("sweep_n16384_k4_b1", "fused_fc"): {"bytes_per_launch": 268548096 + 3760384,
+                                         "source_sha256": "b9ba9386726b06f2e3c224c12e7a946d67c050f28211b6514922226939366a3c"},
+    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6300672,
+                                   "source_sha256": "532dd6636825660d699b29a99ea6b13901970957b3ada4df54019b00538078ac"},
+    ("cfg2_b256", "input_fft"): {"bytes_per_launch": 4212480,
+                                 "source_sha256": "2c9d8d956e6004b7049ae076da55f24fc7f1013caf4f6a5a8cd8e9c1a80e9d02"},
+    ("cfg2_b256", "output_ifft"): {"bytes_per_launch": 4241664,
+                                   "source_sha256": "2c9d8d956e6004b7049ae076da55f24fc7f1013caf4f6a5a8cd8e9c1a80e9d02"},
+    ("cfg4", "contraction"): {"bytes_per_launch": 13059584,
+                              "source_sha256": "532dd6636825660d699b29a99ea6b13901970957b3ada4df54019b00538078ac"},
 }
 
 
@@ -704,7 +716,9 @@ def run_ours(args) -> int:
                                 else kernels.get(dom, {}).get("frac_of_hbm")),
                 "kernel_note": "per-kernel durations are differences between graphs with that kernel launched 4x and 1x per forward: "
                                "repeat launches re-read the same buffers, so they are L2-warm where l2_warm is true",
-                "traffic": traffic, "traffic_source": "ncu capture summarised under profiles/ (not read in this run)" if traffic else None}
+                "traffic": traffic,
+                "traffic_source": ("ncu capture of this kernel and workload summarised under profiles/ (dram__bytes_read.sum + "
+                                   "dram__bytes_write.sum per launch; not read in this run)") if traffic else None}
 
     # ---- end to end through the host-pointer entry point: pinned host x -> device -> forward -> pinned host y ----
     # Every step does its own two copies; consecutive steps go to different streams (and different handles, each
