@@ -397,11 +397,16 @@ class Job:
                                f"{self.sets * self.per_set / 1e6:.0f} MB of algorithmic bytes "
                                f"({'>' if self.sets * self.per_set >= 2 * L2_BYTES else 'less than'} 2 x L2); L2 flushed between repeats")
         self.handles, self.xs, self.ys, self.stacks, self.stack_layers = [], [], [], [], []
-        x0 = None
+        x0 = torch.from_numpy(c.x).cuda().to(self.tdt)
+        self.create_ms = None      # set 0: create + reserve, i.e. copy of the defining vectors, spectra (S0), stored form, workspace
         for s in range(self.sets):
+            if s == 0:
+                torch.cuda.synchronize()
+                t_create = time.perf_counter()
+            elif s == 1:
+                torch.cuda.synchronize()
+                self.create_ms = 1e3 * (time.perf_counter() - t_create)
             # every set and every rank gets its own batch: the drawn batch, rolled by (rank, set) rows and columns
-            if x0 is None:
-                x0 = torch.from_numpy(c.x).cuda().to(self.tdt)
             xs = x0 if (s == 0 and rank == 0) else torch.roll(x0, shifts=(s + 7 * rank, 3 * s + rank), dims=(0, x0.dim() - 1)).contiguous()
             self.xs.append(xs)
             self.ys.append(torch.empty(self.y_shape, device="cuda", dtype=self.tdt))
@@ -435,6 +440,8 @@ class Job:
                 circ.circ_set_variant(h, variant)
             self.handles.append(h)
         torch.cuda.synchronize()
+        if self.create_ms is None:
+            self.create_ms = 1e3 * (time.perf_counter() - t_create)
 
     def first_handle(self):
         return self.stack_layers[0][0] if self.wl.kind == "stack" else self.handles[0]
@@ -619,7 +626,7 @@ def run_row(name: str, timer: Timer, peaks: dict, floors: dict, args, circ, torc
                "us_warm": 1e3 * warm_ms / 8, "samples_per_s": wl.samples / (us * 1e-6),
                "dense_equiv_tflops": wl.dense_flops / (us * 1e-6) / 1e12, "bound": rf["bound"], "frac": rf["frac"],
                "alg_mb": wl.alg_bytes / 1e6, "repeats": reps, "sets": job.sets,
-               "latency_bound": wl.alg_bytes < 32e6,
+               "latency_bound": wl.alg_bytes < 32e6, "create_ms": job.create_ms,
                "launch_floors": us / floors["launch_floor_us"]}
         return row
     finally:
@@ -797,7 +804,7 @@ def run_ours(args) -> int:
             "config": {"workload": wl.name, "description": wl.desc, "samples_per_step_per_gpu": wl.samples, "variant": variant,
                        "path": {1: "fused", 2: "fma", 3: "tensor"}.get(variant, "?"),
                        "timing": f"median of {reps} repeats of exactly {args.steps} steps (one CUDA graph per repeat), cold",
-                       "l2": job.footprint_note, "us_per_step_cold": 1e3 * ms_step, "us_per_step_warm": warm_us,
+                       "l2": job.footprint_note, "create_ms": job.create_ms, "us_per_step_cold": 1e3 * ms_step, "us_per_step_warm": warm_us,
                        "dense_equiv_tflops": wl.dense_flops * world / (ms_step * 1e-3) / 1e12,
                        "floors": floors, "dense_context": dense, "table": table},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,

@@ -26,6 +26,11 @@
 #ifndef CIRC_H_
 #define CIRC_H_
 
+/*
+ * Environment: CIRC_LOG (any value, read once per process) makes the library print one line on stderr for every error,
+ * every created layer (shape, block size, bytes of spectra) and every forward (variant, kernels, columns, workspace and
+ * stored-form bytes).  Off by default; nothing else in the environment is read.
+ */
 #ifdef __cplusplus
 extern "C" {
 #endif

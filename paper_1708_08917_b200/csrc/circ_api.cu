@@ -16,13 +16,26 @@ static thread_local char g_err[512] = "";
 static thread_local int g_code = CIRC_OK;
 static std::atomic<long> g_launches{0};
 
+// CIRC_LOG in the environment (read once): one line on stderr per error, per created layer and per forward.
+bool log_enabled() {
+    static const bool on = getenv("CIRC_LOG") != nullptr;
+    return on;
+}
 void set_error(int code, const char* fmt, ...) {
     g_code = code;
     va_list ap;
     va_start(ap, fmt);
     vsnprintf(g_err, sizeof(g_err), fmt, ap);
     va_end(ap);
-    if (getenv("CIRC_LOG")) fprintf(stderr, "[circ] error %d: %s\n", code, g_err);
+    if (log_enabled()) fprintf(stderr, "[circ] error %d: %s\n", code, g_err);
+}
+void log_line(const char* fmt, ...) {
+    char buf[384];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    fprintf(stderr, "[circ] %s\n", buf);
 }
 void count_launches(long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -147,6 +160,9 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
         cudaFree(L->w_dev);
         L->w_dev = nullptr;
     }
+    if (log_enabled())
+        log_line("create %s m=%d n=%d k=%d (transform size %d) p=%d q=%d taps=%d spectra=%zu bytes", kind ? "conv" : "fc", m, n, L->geo.ku,
+                 L->geo.k, L->geo.p, L->geo.q, taps, (size_t)taps * L->geo.p * L->geo.q * L->geo.k * sizeof(float));
     return L;
 }
 
@@ -331,6 +347,10 @@ static int run_staged(Layer* L, const void* x, void* y, const Extent& e, cudaStr
     if ((rc = stage_contract(L, xop, yop, e, stream, tensor)) != CIRC_OK) return rc;
     if ((rc = stage_output(L, yop, y, e, stream, tensor)) != CIRC_OK) return rc;
     L->last_variant = tensor ? CIRC_VARIANT_TENSOR : CIRC_VARIANT_STAGED;
+    if (log_enabled())
+        log_line("forward %s variant=%s kernels=%d/%d/%d columns=%ld workspace=%zu bytes stored forms=%zu bytes", L->kind ? "conv" : "fc",
+                 tensor ? "tensor" : "staged", L->last_kernels[0], L->last_kernels[1], L->last_kernels[2],
+                 L->kind ? 2L * e.Nh * e.Ho * e.Wo : 2L * e.Bh, L->ws_bytes, (size_t)circ_weight_bytes(reinterpret_cast<circ_handle>(L)));
     return CIRC_OK;
 }
 
@@ -382,6 +402,9 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
         }
         rc = launch_fused_fc(L, x, y, batch, s);
         if (rc == CIRC_OK) L->last_variant = CIRC_VARIANT_FUSED;
+        if (rc == CIRC_OK && log_enabled())
+            log_line("forward fc variant=fused batch=%d column slices=%d row blocks per thread block=%d spectra=%zu bytes", batch,
+                     L->last_kernels[1], L->last_kernels[2], (size_t)L->geo.p * L->geo.q * L->geo.k * (L->w_dtype == CIRC_BF16 ? 2 : 4));
         return rc;
     }
     if (variant == CIRC_VARIANT_TENSOR && !tensor_supported(L)) {

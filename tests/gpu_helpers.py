@@ -18,6 +18,16 @@ def scale_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(got.astype(np.float64) - ref)) / denom)
 
 
+def floored_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """The secondary, element-wise figure: max_t |g_t - o_t| / max(|o_t|, 1e-3 rms(o)).  Reported, not a pass criterion:
+    it divides by each element's own magnitude (floored), so it is larger than E wherever small outputs carry the
+    absolute error of large sums."""
+    ref = ref.astype(np.float64)
+    floor = 1e-3 * float(np.sqrt(np.mean(ref * ref)))
+    den = np.maximum(np.abs(ref), floor if floor > 0.0 else 1.0)
+    return float(np.max(np.abs(got.astype(np.float64) - ref) / den))
+
+
 def to_device(a: np.ndarray, bf16: bool) -> torch.Tensor:
     t = torch.from_numpy(np.ascontiguousarray(a)).cuda()
     return t.to(torch.bfloat16) if bf16 else t
