@@ -129,31 +129,43 @@ contract_rows_kernel(const __grid_constant__ CUtensorMap map_a_real, const __gri
         if (lane == 0) {
             int s = 0, issued = 0;
             uint32_t par = 0;
-            bool wrapped = false, ok = true, waited = false;
+            bool wrapped = false, ok = true;
+            // The weights were written when the layer was made: their copies do not depend on the kernel before this
+            // one.  The first trip around the ring therefore announces its bytes and fetches its weight tiles before
+            // waiting for that kernel; the X tiles of those stages follow after the wait.
+            int ahead = 0;
+            if (!g.no_copy) {
+                for (int tile = blockIdx.x; tile < g.tiles && ahead < g.stages; tile += gridDim.x) {
+                    const RowsTile t = rows_decode(g, tile);
+                    const uint32_t tx_bytes = (uint32_t)g.nsplit * ((uint32_t)t.npad * 128 + a_bytes);
+                    for (int kb = t.kb0; kb < t.kb1 && ahead < g.stages; ++kb, ++ahead) {
+                        unsigned char* as = ring + (size_t)ahead * stage_bytes + (size_t)g.nsplit * x_bytes;
+                        mbar_expect_tx(&full_bar[ahead], tx_bytes);
+                        tma_load_4d(as, t.real ? &map_a_real : &map_a_cplx, &full_bar[ahead], kb * kRowsKBlock, t.row0, 0, t.prob_in_kind);
+                    }
+                }
+            }
+            pdl_wait();                              // X is written by the transform kernel before this one
+            int it = 0;
             for (int tile = blockIdx.x; tile < g.tiles && ok; tile += gridDim.x) {
                 const RowsTile t = rows_decode(g, tile);
                 const CUtensorMap* map_a = t.real ? &map_a_real : &map_a_cplx;
                 const CUtensorMap* map_xhi = t.real ? &map_xhi_real : &map_xhi_cplx;
                 const CUtensorMap* map_xlo = t.real ? &map_xlo_real : &map_xlo_cplx;
                 const uint32_t tx_bytes = (uint32_t)g.nsplit * ((uint32_t)t.npad * 128 + a_bytes);
-                for (int kb = t.kb0; kb < t.kb1; ++kb) {
+                for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     if (wrapped) ok = mbar_wait(&empty_bar[s], par ^ 1u, &abort_flag, g.spin_limit);
                     if (!ok) break;
                     unsigned char* xs = ring + (size_t)s * stage_bytes;
                     unsigned char* as = xs + (size_t)g.nsplit * x_bytes;
-                    mbar_expect_tx(&full_bar[s], tx_bytes);
+                    if (it >= ahead) mbar_expect_tx(&full_bar[s], tx_bytes);
                     if (g.no_copy) {                 // fault injection: nothing is in flight, the consumer's wait runs out
                         ok = false;
                         issued = 0;
                         break;
                     }
-                    // the weights were written when the layer was made: their copy does not wait for the kernel before
-                    // this one; [part][row][128 B]: hi parts first, then lo parts
-                    tma_load_4d(as, map_a, &full_bar[s], kb * kRowsKBlock, t.row0, 0, t.prob_in_kind);
-                    if (!waited) {
-                        pdl_wait();                  // X is written by the transform kernel before this one
-                        waited = true;
-                    }
+                    // [part][row][128 B]: hi parts first, then lo parts
+                    if (it >= ahead) tma_load_4d(as, map_a, &full_bar[s], kb * kRowsKBlock, t.row0, 0, t.prob_in_kind);
                     tma_load_4d(xs, map_xhi, &full_bar[s], kb * kRowsKBlock, 0, t.prob_in_kind, 0);
                     if (g.nsplit == 2) tma_load_4d(xs + x_bytes, map_xlo, &full_bar[s], kb * kRowsKBlock, 0, t.prob_in_kind, 0);
                     if (issued < g.stages) ++issued;
