@@ -36,7 +36,7 @@ enum {
     CIRC_KERNEL_S2_ROWS_TWIN = 14, /* row-streaming tensor-core contraction with twin columns */
     CIRC_KERNEL_S3_LOADS = 20,  /* inverse transforms fed by per-thread loads */
     CIRC_KERNEL_S3_BULK = 21,   /* inverse transforms fed by bulk asynchronous copies */
-    CIRC_KERNEL_S3_TMA = 22,    /* inverse transforms with one exchange through shared memory, output written by TMA */
+    CIRC_KERNEL_S3_TMA = 22,    /* inverse transforms with tiles loaded and written by TMA (one exchange through shared memory; short blocks: one thread per transform) */
     CIRC_KERNEL_S4_FUSED = 30   /* the one-launch small-batch kernel */
 };
 

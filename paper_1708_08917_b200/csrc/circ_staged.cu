@@ -845,7 +845,8 @@ int launch_output_ifft(const Layer* L, const float* yop, void* y, const Extent& 
         return CIRC_ERR_UNSUPPORTED;
     }
     const size_t copy_stride = (size_t)2 * ext.Bho * p * L->geo.k;     // all problems of Y
-    // large forwards of power-of-two blocks from 32 to 256: one exchange through shared memory, tiles written by TMA
+    // large forwards of power-of-two blocks: tiles loaded and written by TMA (32 .. 256: one exchange through shared memory;
+    // 4 .. 16: one thread per transform).  16384 x 16384, batch 1024, float32: k = 4: 28.7 -> 19.1 us, k = 16: 37 -> 19.1 us.
     if (!small && !correlation && !twin && pieces.real == 0 && !L->no_tma_output && output_ifft_tma_supported(L, y, ext))
         return launch_output_ifft_tma(L, yop, y, ext, stream);
     const bool bulk = !twin && pieces.real == 0 && !small && !embedded(L->geo) && L->geo.k >= 16 && L->geo.k <= 256 && (total & 1) == 0 && total >= 148L * 256 &&

@@ -47,11 +47,12 @@ def test_tensor_contraction_wait_runs_out_and_the_handle_recovers(shape):
         circ.circ_destroy(h)
 
 
-@pytest.mark.parametrize("batch", [6000, 6002])
-def test_bulk_fed_inverse_transform_wait_runs_out_and_the_handle_recovers(batch):
-    # 3000 pairs x 16 row blocks = 48000 transforms: large enough for the kernels that stage their tiles by asynchronous
-    # copies (whole tiles of two pairs: the TMA kernel; 3001 pairs: the bulk-copy kernel)
-    case = synth.fc_case("timeout_bulk", 16 * 64, 8 * 64, 64, batch, w_var=1.0 / 512, x_dist="normal")
+@pytest.mark.parametrize("m,n,k,batch", [(16 * 64, 8 * 64, 64, 6000), (16 * 64, 8 * 64, 64, 6002), (128 * 4, 8 * 4, 4, 600)])
+def test_bulk_fed_inverse_transform_wait_runs_out_and_the_handle_recovers(m, n, k, batch):
+    # large enough for the kernels that stage their tiles by asynchronous copies: k = 64, 3000 pairs x 16 row blocks (whole
+    # tiles of two pairs: the TMA kernel; 3001 pairs: the bulk-copy kernel); k = 4, 300 pairs x 128 row blocks (the TMA
+    # kernel for short blocks)
+    case = synth.fc_case(f"timeout_bulk_{k}", m, n, k, batch, w_var=1.0 / n, x_dist="normal")
     h = circ.circ_fc_create(case.m, case.n, case.k, case.w)
     try:
         circ.circ_debug_inject(h, circ.CIRC_INJECT_BULK_NO_COPY)
@@ -63,7 +64,8 @@ def test_bulk_fed_inverse_transform_wait_runs_out_and_the_handle_recovers(batch)
         circ.circ_debug_inject(h, circ.CIRC_INJECT_NONE)
         got = _forward(h, case)
         circ.circ_device_status(h)
-        rows = [0, 1, 2999, 3000, batch - 1]
+        half = (batch + 1) // 2
+        rows = [0, 1, half - 1, half, batch - 1]
         ref = oracle.fc(case.w, case.x[rows])
         assert scale_rel_err(got[rows], ref) <= TOL_F32
     finally:

@@ -1,5 +1,6 @@
-"""GPU parity for the inverse-transform kernel that writes its tiles by TMA (large forwards, float32 k = 32 .. 256,
-bfloat16 k = 64 .. 256, p a multiple of 32 or a divisor of it with whole tiles): bias and ReLU, float32 and bfloat16
+"""GPU parity for the inverse-transform kernels that write their tiles by TMA (large forwards; float32 k = 32 .. 256,
+bfloat16 k = 64 .. 256, p a multiple of 32 or a divisor of it with whole tiles; short blocks, one thread per transform:
+float32 k = 4 .. 16, bfloat16 k = 8, 16, p a multiple of 128): bias and ReLU, float32 and bfloat16
 outputs, odd batches, Y that comes as several copies with real and imaginary parts apart (after the row-streaming
 contraction), and agreement with the load-based kernels."""
 import numpy as np
@@ -65,6 +66,31 @@ def test_tma_written_inverse_transforms(k, p, q, batch, bf16):
         old, kernels_old = _run(case, 0)
         assert kernels_old[2] != circ.CIRC_KERNEL_S3_TMA
         assert scale_rel_err(got, old) <= (2e-2 if bf16 else 2e-5)     # the same transform, another order of operations
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("k,p,q,batch", [
+    (4, 128, 8, 600),      # one complex problem; one tile per pair
+    (4, 256, 16, 301),     # two tiles per pair, odd batch
+    (8, 128, 8, 400),
+    (16, 384, 8, 255),     # three tiles per pair, seven complex problems, odd batch
+    (16, 128, 16, 2000),   # more tiles than resident thread blocks: the double buffers are reused many times
+    (8, 192, 8, 500),      # p not a multiple of 128 -> the other kernels
+])
+def test_tma_written_inverse_transforms_of_short_blocks(k, p, q, batch, bf16):
+    case = synth.fc_case(f"outtma_small_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
+                         bias_var=0.01, relu=True, bf16_io=bf16)
+    got, kernels = _run(case, 1, circ.CIRC_VARIANT_TENSOR)
+    served = p % 128 == 0 and k >= (8 if bf16 else 4)
+    assert (kernels[2] == circ.CIRC_KERNEL_S3_TMA) == served, kernels
+    assert not np.isnan(got).any()
+    rows = _rows(batch)
+    ref = oracle.fc(case.w, case.x[rows], bias=case.bias, relu=case.relu)
+    assert scale_rel_err(got[rows], ref) <= (TOL_BF16 if bf16 else TOL_F32)
+    if served:
+        old, kernels_old = _run(case, 0, circ.CIRC_VARIANT_TENSOR)
+        assert kernels_old[2] != circ.CIRC_KERNEL_S3_TMA
+        assert scale_rel_err(got, old) <= (2e-2 if bf16 else 2e-5)
 
 
 @pytest.mark.parametrize("bf16", [False, True])
