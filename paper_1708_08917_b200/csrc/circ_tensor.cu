@@ -73,8 +73,11 @@ struct TileCoord {
 __device__ __forceinline__ TileCoord decode_tile(const TcArgs& g, long tile) {
     TileCoord t;
     unsigned cta = (unsigned)tile;
-    t.real = cta < (unsigned)g.ctas_real;
-    if (!t.real) cta -= (unsigned)g.ctas_real;
+    // complex tiles (twice the contraction length) come first, so that a grid with more tiles than thread blocks
+    // ends on the short ones
+    const unsigned ctas_cplx = (unsigned)g.tiles - (unsigned)g.ctas_real;
+    t.real = cta >= ctas_cplx;
+    if (t.real) cta -= ctas_cplx;
     const unsigned tiles_w = (unsigned)(t.real ? g.tiles_w : g.tiles_w_c);
     const unsigned sp_tiles = (unsigned)(g.V * g.tiles_h) * tiles_w;
     const unsigned nt = (unsigned)(t.real ? g.nt_real : g.nt_cplx);
@@ -564,7 +567,11 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         g.ctas_real = 2 * g.nt_real * sp_tiles;
         ctas = (long)g.ctas_real + (long)(k / 2 - 1) * g.nt_cplx * sp_tiles_c;
         // a grid that leaves most of the 148 SMs idle is split into narrower row tiles
-        if (ctas >= 100 || g.bn_cplx <= 32) break;
+        // ... and so is a grid of fewer than 200 long float32 tiles (16 K blocks or more): with at most one tile per thread
+        // block the longest tile sets the time; half-height tiles take 0.67 of it and most thread blocks then take a short
+        // real tile on top (4096 x 4096, k = 4, batch 1024: 57.4 -> 49.4 us; short tiles, where latency rules, lose by it)
+        const bool long_tiles = nsplit == 2 && (2 * q + kKBlock - 1) / kKBlock >= 16 && g.bn_cplx > 128;
+        if (ctas >= (long_tiles ? 200 : 100) || g.bn_cplx <= 32) break;
         g.bn_cplx = round_up16(g.bn_cplx / 2);
         if (g.bn_real > 32) g.bn_real = round_up16(g.bn_real / 2);
     }
