@@ -168,6 +168,21 @@ def conv_pixels(w, x, pad: int, pixels, bias=None, relu: bool = False, conventio
     return y
 
 
+POOL_MAX, POOL_AVG, POOL_L2 = 0, 1, 2
+
+
+def pool(x, window: int, stride: int, mode: int = POOL_MAX) -> np.ndarray:
+    """Pooling layer (Sec. 2.1): ``x[N][H][W][C]`` -> ``y[N][Ho][Wo][C]``, whole windows only, no padding."""
+    x = _d(x)
+    N, H, W, C = x.shape
+    assert 1 <= window <= min(H, W) and stride >= 1 and mode in (POOL_MAX, POOL_AVG, POOL_L2)
+    Ho, Wo = (H - window) // stride + 1, (W - window) // stride + 1
+    y = np.empty((N, Ho, Wo, C), dtype=np.float64)
+    _load().circ_oracle_pool(ctypes.c_int(mode), ctypes.c_int(window), ctypes.c_int(stride), ctypes.c_int(N), ctypes.c_int(H),
+                             ctypes.c_int(W), ctypes.c_int(C), _ptr(x), _ptr(y))
+    return y
+
+
 def dft(re, im=None, sign: int = -1):
     """Naive O(k^2) DFT (``sign=-1`` forward, ``+1`` inverse, both unnormalised) -> (re, im)."""
     re = _d(re)

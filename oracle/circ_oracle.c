@@ -11,6 +11,7 @@
  *          with W cut into p x q circulant k x k blocks  (Eq. 3, Sec. 3.1)
  *   CONV : Y(x,y,p) = sum_{i,j,c} F(i,j,c,p) X(x+i-1, y+j-1, c)   (Eq. 6)
  *          with the channel pair (c,p) of F block-circulant at every tap (Sec. 3.2, Eq. 7)
+ *   POOL : max / mean / L2 norm over window x window pixels, per channel   (Sec. 2.1)
  *
  * Every circulant block is expanded element by element from its defining
  * vector; all arithmetic is float64; there is no FFT anywhere in the layer
@@ -287,6 +288,38 @@ ORACLE_API void circ_oracle_conv_backward_weight(int c_out, int c_in, int r, int
                     }
             }
         }
+}
+
+/*
+ * Pooling layer (Sec. 2.1: subsampling of the extracted features by a max, average or L2-norm over a window; Sec. 4.2:
+ * the peripheral computing block): x[N][H][W][C] -> y[N][Ho][Wo][C], Ho = (H - window) / stride + 1 (whole windows
+ * only, no padding), y(n, i, j, c) = op over a, b in [0, window) of x(n, stride i + a, stride j + b, c).
+ * mode 0: maximum, 1: arithmetic mean, 2: L2 norm (square root of the sum of squares).
+ */
+ORACLE_API void circ_oracle_pool(int mode, int window, int stride, int N, int H, int W, int C, const double* x, double* y) {
+    const int Ho = (H - window) / stride + 1, Wo = (W - window) / stride + 1;
+#ifdef _OPENMP
+#pragma omp parallel for collapse(2) schedule(static)
+#endif
+    for (int n = 0; n < N; ++n)
+        for (int i = 0; i < Ho; ++i)
+            for (int j = 0; j < Wo; ++j)
+                for (int c = 0; c < C; ++c) {
+                    double acc = mode == 0 ? -INFINITY : 0.0;
+                    for (int a = 0; a < window; ++a)
+                        for (int b = 0; b < window; ++b) {
+                            const double v = x[(((size_t)n * H + (size_t)(stride * i + a)) * W + (size_t)(stride * j + b)) * C + c];
+                            if (mode == 0)
+                                acc = v > acc ? v : acc;
+                            else if (mode == 1)
+                                acc += v;
+                            else
+                                acc += v * v;
+                        }
+                    if (mode == 1) acc /= (double)(window * window);
+                    if (mode == 2) acc = sqrt(acc);
+                    y[(((size_t)n * Ho + i) * Wo + j) * C + c] = acc;
+                }
 }
 
 /*

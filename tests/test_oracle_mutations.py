@@ -152,3 +152,52 @@ def test_unmutated_copy_passes_backward_pins(tmp_path):
 @pytest.mark.parametrize("name", sorted(BACKWARD_MUTATIONS))
 def test_planted_backward_mistake_is_caught(tmp_path, name):
     assert not _backward_pins_hold(_build_backward(tmp_path, name)), f"pins did not notice mutation {name}"
+
+
+# ---- the pooling function: mistakes planted there must break its hand cases ------------------------------------------
+POOL_MUTATIONS = {
+    "pool_min_instead_of_max": ("acc = v > acc ? v : acc;", "acc = v < acc ? v : acc;"),
+    "pool_max_starts_at_zero": ("double acc = mode == 0 ? -INFINITY : 0.0;", "double acc = 0.0;"),
+    "pool_stride_ignored_on_rows": ("(size_t)(stride * i + a)) * W", "(size_t)(i + a)) * W"),
+    "pool_rows_and_columns_swapped": ("(size_t)(stride * i + a)) * W + (size_t)(stride * j + b)", "(size_t)(stride * j + b)) * W + (size_t)(stride * i + a)"),
+    "pool_mean_divides_by_window": ("acc /= (double)(window * window);", "acc /= (double)window;"),
+    "pool_window_one_short": ("for (int b = 0; b < window; ++b) {\n                            const double v", "for (int b = 0; b < window - 1; ++b) {\n                            const double v"),
+    "pool_l2_without_root": ("if (mode == 2) acc = sqrt(acc);", "if (mode == 2) acc = acc;"),
+    "pool_channels_mixed": ("* C + c];\n                            if (mode == 0)", "* C + (C - 1 - c)];\n                            if (mode == 0)"),
+}
+
+
+def _pool_pins_hold(lib) -> bool:
+    golden = Path(__file__).resolve().parent / "golden" / "pool_cases.txt"
+    ok = True
+    for line in golden.read_text().splitlines():
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, shape, xs, ys = [part.split() for part in line.split("|")]
+        mode, window, stride = (int(v) for v in head)
+        H, W, C = (int(v) for v in shape)
+        x = np.array(xs, dtype=np.float64)
+        want = np.array(ys, dtype=np.float64)
+        y = np.full(want.shape, np.nan)
+        lib.circ_oracle_pool(mode, window, stride, 1, H, W, C, x.ctypes.data_as(_dp), y.ctypes.data_as(_dp))
+        ok &= bool(np.allclose(y, want, rtol=0, atol=1e-12))
+    return bool(ok)
+
+
+def test_unmutated_copy_passes_the_pool_pins(tmp_path):
+    (tmp_path / "plain.c").write_text(SRC.read_text())
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(tmp_path / "plain.so"), str(tmp_path / "plain.c"), "-lm"], check=True)
+    assert _pool_pins_hold(ctypes.CDLL(str(tmp_path / "plain.so")))
+
+
+@pytest.mark.parametrize("name", sorted(POOL_MUTATIONS))
+def test_planted_pool_mistake_is_caught(tmp_path, name):
+    old, new = POOL_MUTATIONS[name]
+    text = SRC.read_text()
+    assert text.count(old) == 1, f"mutation anchor for {name} must be unique"
+    out = tmp_path / f"{name}.c"
+    out.write_text(text.replace(old, new, 1))
+    lib = tmp_path / f"{name}.so"
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(lib), str(out), "-lm"], check=True)
+    assert not _pool_pins_hold(ctypes.CDLL(str(lib))), f"pins did not notice mutation {name}"

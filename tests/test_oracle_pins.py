@@ -8,6 +8,7 @@ Sec. 3.1).  None of these tests touches the CUDA library.
 """
 import numpy as np
 import pytest
+import torch
 import scipy.linalg
 
 import oracle
@@ -371,3 +372,57 @@ def test_conv_backward_weight_one_tap_reduces_to_fc_backward():
     for conv in (0, 1):
         _, gw_fc = oracle.fc_backward(w, x.reshape(-1, q * k), g.reshape(-1, p * k), convention=conv)
         np.testing.assert_allclose(oracle.conv_backward_weight(x, g, 1, 0, k, convention=conv)[0, 0], gw_fc, atol=1e-11)
+
+
+# ---- pooling layer (Sec. 2.1, Sec. 4.2) -------------------------------------------------------------------------------
+def _pool_cases(golden_dir):
+    cases = []
+    for line in (golden_dir / "pool_cases.txt").read_text().splitlines():
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        head, shape, xs, ys = [part.split() for part in line.split("|")]
+        mode, window, stride = (int(v) for v in head)
+        H, W, C = (int(v) for v in shape)
+        cases.append((mode, window, stride, np.array(xs, dtype=np.float64).reshape(1, H, W, C), np.array(ys, dtype=np.float64)))
+    return cases
+
+
+def test_pool_hand_cases(golden_dir):
+    cases = _pool_cases(golden_dir)
+    assert len(cases) >= 12
+    for mode, window, stride, x, want in cases:
+        got = oracle.pool(x, window, stride, mode)
+        assert got.shape[1] == (x.shape[1] - window) // stride + 1 and got.shape[2] == (x.shape[2] - window) // stride + 1
+        np.testing.assert_allclose(got.reshape(-1), want, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("N,H,W,C,window,stride", [(2, 13, 13, 5, 3, 2), (1, 28, 28, 3, 2, 2), (3, 9, 11, 4, 3, 1), (1, 7, 5, 2, 5, 3),
+                                                   (2, 6, 6, 1, 1, 1), (1, 8, 8, 2, 2, 3)])
+def test_pool_against_torch_float64(N, H, W, C, window, stride):
+    rng = np.random.default_rng(N * 1000 + H * 10 + window)
+    x = rng.standard_normal((N, H, W, C))
+    t = torch.from_numpy(x).permute(0, 3, 1, 2)                      # the library routine takes [N][C][H][W]
+    want_max = torch.nn.functional.max_pool2d(t, window, stride).permute(0, 2, 3, 1).numpy()
+    want_avg = torch.nn.functional.avg_pool2d(t, window, stride).permute(0, 2, 3, 1).numpy()
+    want_l2 = torch.nn.functional.lp_pool2d(t, 2.0, window, stride).permute(0, 2, 3, 1).numpy()
+    assert np.array_equal(oracle.pool(x, window, stride, oracle.POOL_MAX), want_max)      # a maximum is exact
+    np.testing.assert_allclose(oracle.pool(x, window, stride, oracle.POOL_AVG), want_avg, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(oracle.pool(x, window, stride, oracle.POOL_L2), want_l2, rtol=1e-12, atol=1e-13)
+
+
+def test_pool_invariants():
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 10, 9, 3))
+    for mode in (oracle.POOL_MAX, oracle.POOL_AVG):
+        assert np.array_equal(oracle.pool(x, 1, 1, mode), x)                       # a 1 x 1 window is the identity
+    np.testing.assert_allclose(oracle.pool(x, 1, 1, oracle.POOL_L2), np.abs(x), rtol=1e-15)
+    assert np.array_equal(oracle.pool(x, 1, 2, oracle.POOL_MAX), x[:, ::2, ::2, :])   # stride alone subsamples
+    mx, av, l2 = (oracle.pool(x, 3, 2, m) for m in (oracle.POOL_MAX, oracle.POOL_AVG, oracle.POOL_L2))
+    assert (mx >= av).all() and (l2 >= np.abs(av) * 3 - 1e-12).all()                  # max >= mean; ||v||_2 >= sqrt(n) |mean|, n = 9
+    c = np.full((1, 6, 6, 2), -2.5)
+    assert (oracle.pool(c, 2, 2, oracle.POOL_MAX) == -2.5).all() and (oracle.pool(c, 2, 2, oracle.POOL_AVG) == -2.5).all()
+    assert np.allclose(oracle.pool(c, 2, 2, oracle.POOL_L2), 5.0)
+    # transposing the image transposes the result (rows and columns are treated alike)
+    xt = np.ascontiguousarray(x.transpose(0, 2, 1, 3))
+    assert np.array_equal(oracle.pool(xt, 3, 2, oracle.POOL_MAX), oracle.pool(x, 3, 2, oracle.POOL_MAX).transpose(0, 2, 1, 3))
