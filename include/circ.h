@@ -300,6 +300,25 @@ CIRC_API int circ_device_status(circ_handle h);
 CIRC_API const char* circ_last_error(void);
 CIRC_API int circ_last_code(void);
 
+/* Pooling operations of circ_pool_forward. */
+enum { CIRC_POOL_MAX = 0, CIRC_POOL_AVG = 1, CIRC_POOL_L2 = 2 };
+
+/*
+ * circ_pool_forward -- the pooling layer (Sec. 2.1: a subsampling of the extracted features by a max, average or
+ * L2-norm calculation; Sec. 4.2: one of the operations of the peripheral computing block).  No handle: the layer has
+ * no parameters.
+ *   x : DEVICE pointer, [N][H][W][C] contiguous (the layout of circ_conv_forward's output), float32 or bfloat16 (dtype)
+ *   y : DEVICE pointer, [N][Ho][Wo][C], same element type, Ho = (H - window) / stride + 1, Wo likewise: whole windows
+ *       only, no padding; y(n, i, j, c) = op over a, b in [0, window) of x(n, stride i + a, stride j + b, c)
+ *   mode : CIRC_POOL_MAX, CIRC_POOL_AVG (arithmetic mean) or CIRC_POOL_L2 (square root of the sum of squares)
+ *   dtype : CIRC_F32 or CIRC_BF16 (arithmetic in float32; bfloat16 results rounded to nearest even)
+ *   stream : a cudaStream_t passed as void*; the call only enqueues one kernel and allocates nothing
+ * Both buffers stay the caller's.  Errors: CIRC_ERR_ARG (NULL or misaligned pointer, unknown mode or dtype),
+ * CIRC_ERR_SHAPE (a dimension < 1, window > H or W or 64, stride < 1), CIRC_ERR_CUDA.
+ */
+CIRC_API int circ_pool_forward(const void* x, void* y, int N, int H, int W, int C, int window, int stride, int mode, int dtype,
+                               void* stream);
+
 #ifdef __cplusplus
 }
 #endif

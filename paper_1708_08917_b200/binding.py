@@ -18,6 +18,7 @@ LIB_PATH = _HERE / "libcirc.so"
 CIRC_OK = 0
 CIRC_ERR_ARG, CIRC_ERR_SHAPE, CIRC_ERR_ALLOC, CIRC_ERR_CUDA, CIRC_ERR_DEVICE_TIMEOUT, CIRC_ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6
 CIRC_F32, CIRC_BF16 = 0, 1
+CIRC_POOL_MAX, CIRC_POOL_AVG, CIRC_POOL_L2 = 0, 1, 2
 CIRC_VARIANT_AUTO, CIRC_VARIANT_FUSED, CIRC_VARIANT_STAGED, CIRC_VARIANT_TENSOR = 0, 1, 2, 3
 # include/circ_debug.h
 CIRC_STAGE_INPUT_FFT, CIRC_STAGE_CONTRACTION, CIRC_STAGE_OUTPUT_IFFT, CIRC_STAGE_FUSED = 0, 1, 2, 3
@@ -69,6 +70,7 @@ SIGNATURES = {
     "circ_debug_set_fused_split": (_ci, [_vp, _ci]),
     "circ_debug_set_contraction": (_ci, [_vp, _ci, _ci]),
     "circ_debug_set_transforms": (_ci, [_vp, _ci, _ci]),
+    "circ_pool_forward": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp]),
     "circ_last_error": (ctypes.c_char_p, []),
     "circ_last_code": (_ci, []),
 }
@@ -164,6 +166,11 @@ def circ_fc_forward(h: int, x, y, batch: int, stream=None) -> None:
 def circ_conv_forward(h: int, x, y, N: int, H: int, W: int, stream=None) -> None:
     """Enqueue the channel-last convolution ``x[N][H][W][C] -> y[N][Ho][Wo][P]``."""
     _check(load().circ_conv_forward(h, _ptr(x), _ptr(y), N, H, W, _stream(stream)))
+
+
+def circ_pool_forward(x, y, N: int, H: int, W: int, C: int, window: int, stride: int, mode: int, dtype: int, stream=None) -> None:
+    """Enqueue the pooling layer ``x[N][H][W][C] -> y[N][Ho][Wo][C]`` (whole windows, no padding)."""
+    _check(load().circ_pool_forward(_ptr(x), _ptr(y), N, H, W, C, window, stride, mode, dtype, _stream(stream)))
 
 
 def circ_fc_forward_host(h: int, x_host, y_host, batch: int, stream=None) -> None:

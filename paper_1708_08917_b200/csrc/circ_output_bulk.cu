@@ -73,7 +73,7 @@ output_ifft_tma_kernel(const __grid_constant__ CUtensorMap map_yc, const __grid_
                        int* status, int pdl_late, int no_copy) {
     using S = OutBulk<K, TOUT>;
     const uint32_t spin_limit = no_copy ? (1u << 12) : kSpinLimit;   // no_copy: fault injection (tests only)
-    constexpr int L2 = S::L2, R1 = S::R1, E2 = S::E2, TT = S::TT, NC = S::NC;
+    constexpr int L2 = S::L2, R1 = S::R1, E2 = S::E2, TT = S::TT;
     extern __shared__ unsigned char smem_dyn[];
     unsigned char* in0 = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     unsigned char* out0 = in0 + 2 * S::IN;
