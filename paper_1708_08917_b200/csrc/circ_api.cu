@@ -179,7 +179,7 @@ int ensure_forms(Layer* L, unsigned forms, cudaStream_t stream) {
     __nv_bfloat16 *a_bf16 = nullptr, *a_twin = nullptr;
     bool ok = true;
     if (need_f32) ok = ok && dev_alloc(&a_f32, L->a_elems * sizeof(float)) == cudaSuccess;
-    if (need_bf16) ok = ok && dev_alloc(&a_bf16, 2 * L->a_elems * sizeof(__nv_bfloat16) + 256) == cudaSuccess;
+    if (need_bf16) ok = ok && dev_alloc(&a_bf16, bf16_form_elems(L) * sizeof(__nv_bfloat16) + 256) == cudaSuccess;
     if (need_twin) ok = ok && dev_alloc(&a_twin, twin_elems(L) * sizeof(__nv_bfloat16) + 256) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
@@ -201,7 +201,7 @@ int ensure_forms(Layer* L, unsigned forms, cudaStream_t stream) {
 }
 
 static size_t x_operand_floats(const Layer* L, const Extent& e) {
-    const size_t xin = (size_t)2 * e.Bh * L->geo.q * L->geo.k;   // all problems of X
+    const size_t xin = (size_t)2 * e.Bh * padded_q(L->geo.q) * L->geo.k;   // all problems of X (bfloat16 runs may be padded)
     return (use_twin(L, e) ? 2 * xin : xin);                     // twin columns: the complex problems twice
 }
 
@@ -408,7 +408,7 @@ int circ_fc_forward(circ_handle h, const void* x, void* y, int batch, void* stre
         return rc;
     }
     if (variant == CIRC_VARIANT_TENSOR && !tensor_supported(L)) {
-        set_error(CIRC_ERR_UNSUPPORTED, "the tensor-core contraction needs q = n/k to be a multiple of 8 (q=%d)", L->geo.q);
+        set_error(CIRC_ERR_UNSUPPORTED, "the tensor-core contraction needs q = n/k to be a multiple of 4 (q=%d)", L->geo.q);
         return CIRC_ERR_UNSUPPORTED;
     }
     return run_staged(L, x, y, fc_extent(batch), s, variant == CIRC_VARIANT_TENSOR);
@@ -656,7 +656,7 @@ long circ_weight_bytes(circ_handle h) {
     if (L->w_stream) b += blocks * L->geo.k * sizeof(float);
     if (L->w_stream_bf16) b += blocks * L->geo.k * sizeof(__nv_bfloat16);
     if (L->a_f32) b += L->a_elems * sizeof(float);
-    if (L->a_bf16) b += 2 * L->a_elems * sizeof(__nv_bfloat16) + 256;
+    if (L->a_bf16) b += bf16_form_elems(L) * sizeof(__nv_bfloat16) + 256;
     if (L->a_twin) b += twin_elems(L) * sizeof(__nv_bfloat16) + 256;
     if (L->transposed) b += (size_t)circ_weight_bytes(reinterpret_cast<circ_handle>(L->transposed));
     return (long)b;

@@ -224,7 +224,12 @@ int launch_defining_vectors(const Layer* L, float* w_out, cudaStream_t stream);
 // Stored operand layouts, built on first use.  `forms` is a mask of FORM_*; fails with CIRC_ERR_UNSUPPORTED when a
 // form is missing while `stream` is being captured (building allocates).
 enum { FORM_A_F32 = 1, FORM_A_BF16 = 2, FORM_A_TWIN = 4 };
-inline size_t twin_elems(const Layer* L) { return L->a_elems + (size_t)2 * L->geo.taps * L->geo.p * L->geo.q; }   // bfloat16 values of a_twin
+// The bfloat16 operands of the tensor-core contractions (X, a_bf16, a_twin) keep their contraction runs a multiple of 8
+// entries long (16 bytes: what a TMA stride and the hi | lo part offset need): a layer with q = 4, 12, 20 ... column blocks
+// stores them with 4 zero entries (8 for the (Re, Im) runs of complex problems) at the end of every run.
+__host__ __device__ inline int padded_q(int q) { return (q + 7) & ~7; }
+inline size_t bf16_form_elems(const Layer* L) { return 2 * L->a_elems / L->geo.q * padded_q(L->geo.q); }   // bfloat16 values of a_bf16 (hi and lo)
+inline size_t twin_elems(const Layer* L) { return (L->a_elems + (size_t)2 * L->geo.taps * L->geo.p * L->geo.q) / L->geo.q * padded_q(L->geo.q); }   // bfloat16 values of a_twin
 int ensure_forms(Layer* L, unsigned forms, cudaStream_t stream);
 // How the tensor-core contraction of a forward runs (circ_tensor_rows.cu): `twin`: weights stored once, X twice;
 // `rows`: the row-streaming kernel instead of the large-batch one.

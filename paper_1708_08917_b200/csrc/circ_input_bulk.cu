@@ -320,7 +320,7 @@ static int launch_k(const Layer* L, const void* x, void* xop, int xmode, bool tw
 bool input_fft_bulk_supported(const Layer* L, const void* x, long total) {
     const int k = L->geo.k, q = L->geo.q;
     const int kmin = L->x_dtype == CIRC_BF16 ? 64 : 32;
-    return !embedded(L->geo) && k >= kmin && k <= 256 && (q % 32 == 0 || 32 % q == 0) && total >= 148L * 64 &&
+    return !embedded(L->geo) && k >= kmin && k <= 256 && (q % 32 == 0 || (32 % q == 0 && q % 8 == 0)) && total >= 148L * 64 &&
            (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && L->dev_status != nullptr && tensor_map_encoder() != nullptr;
 }
 

@@ -89,8 +89,10 @@ __global__ void spectrum_forms_kernel(const float* __restrict__ w_stream, float*
                 a_f32[r1 + 2 * j + 1] = fre;
             }
         }
-        // split bfloat16 operands: [problem][row][hi|lo][tap][Kq]
-        const size_t rsz = (size_t)p * taps * 2 * q;  // one real problem, hi and lo
+        // split bfloat16 operands: [problem][row][hi|lo][tap][Kq], runs padded to a multiple of 8 entries (the buffers
+        // were zeroed first when that adds entries)
+        const int qs = padded_q(q);
+        const size_t rsz = (size_t)p * taps * 2 * qs;  // one real problem, hi and lo
         auto put = [&](__nv_bfloat16* a, size_t b0, size_t row, int kq, int kk, float val) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(val);
             const __nv_bfloat16 lo = __float2bfloat16_rn(val - __bfloat162float(hi));
@@ -101,21 +103,21 @@ __global__ void spectrum_forms_kernel(const float* __restrict__ w_stream, float*
         if (a_bf16) {
             const size_t b0 = problem_offset(prob, rsz, 4 * rsz);
             if (problem_is_real(prob)) {
-                put(a_bf16, b0, i, q, j, fre);
+                put(a_bf16, b0, i, qs, j, fre);
             } else {
-                put(a_bf16, b0, (size_t)2 * i, 2 * q, 2 * j, fre);
-                put(a_bf16, b0, (size_t)2 * i, 2 * q, 2 * j + 1, -fim);
-                put(a_bf16, b0, (size_t)2 * i + 1, 2 * q, 2 * j, fim);
-                put(a_bf16, b0, (size_t)2 * i + 1, 2 * q, 2 * j + 1, fre);
+                put(a_bf16, b0, (size_t)2 * i, 2 * qs, 2 * j, fre);
+                put(a_bf16, b0, (size_t)2 * i, 2 * qs, 2 * j + 1, -fim);
+                put(a_bf16, b0, (size_t)2 * i + 1, 2 * qs, 2 * j, fim);
+                put(a_bf16, b0, (size_t)2 * i + 1, 2 * qs, 2 * j + 1, fre);
             }
         }
         if (a_twin) {
             const size_t b0 = problem_offset(prob, rsz, 2 * rsz);
             if (problem_is_real(prob)) {
-                put(a_twin, b0, i, q, j, fre);
+                put(a_twin, b0, i, qs, j, fre);
             } else {
-                put(a_twin, b0, i, 2 * q, 2 * j, fre);
-                put(a_twin, b0, i, 2 * q, 2 * j + 1, fim);
+                put(a_twin, b0, i, 2 * qs, 2 * j, fre);
+                put(a_twin, b0, i, 2 * qs, 2 * j + 1, fim);
             }
         }
     }
@@ -183,6 +185,10 @@ int launch_precompute(Layer* L, cudaStream_t stream) {
 int launch_spectrum_forms(Layer* L, float* a_f32, __nv_bfloat16* a_bf16, __nv_bfloat16* a_twin, cudaStream_t stream) {
     const Geometry& g = L->geo;
     if (a_f32 || a_bf16 || a_twin) {
+        if (padded_q(g.q) != g.q) {     // the padding entries of the bfloat16 runs are zeros
+            if (a_bf16) CIRC_CUDA_TRY(cudaMemsetAsync(a_bf16, 0, bf16_form_elems(L) * sizeof(__nv_bfloat16), stream), CIRC_ERR_CUDA);
+            if (a_twin) CIRC_CUDA_TRY(cudaMemsetAsync(a_twin, 0, twin_elems(L) * sizeof(__nv_bfloat16), stream), CIRC_ERR_CUDA);
+        }
         const long total = (long)g.taps * g.p * g.q * (g.k / 2 + 1);
         spectrum_forms_kernel<<<grid_for((size_t)total, 256), 256, 0, stream>>>(L->w_stream, a_f32, a_bf16, a_twin, g, total);
         count_launches(1);

@@ -30,7 +30,7 @@ static int variant_for(const Layer* L, int batch) {
 
 // the per-layer workspace of the ordinary forward: all problems of X and of Y (the slack covers the alignment gap)
 static size_t stack_workspace(const Layer* L, const Extent& e) {
-    return ((size_t)2 * e.Bh * L->geo.q * L->geo.k + (size_t)2 * e.Bho * L->geo.p * L->geo.k) * sizeof(float) + 512;
+    return ((size_t)2 * e.Bh * padded_q(L->geo.q) * L->geo.k + (size_t)2 * e.Bho * L->geo.p * L->geo.k) * sizeof(float) + 512;
 }
 
 static int grow_activations(Stack* S, size_t need) {
@@ -150,7 +150,7 @@ int circ_stack_forward(circ_stack_handle s, const void* x, void* y, int batch, v
             return CIRC_ERR_UNSUPPORTED;
         }
         if (variant[l] == CIRC_VARIANT_TENSOR && !tensor_supported(L)) {
-            set_error(CIRC_ERR_UNSUPPORTED, "layer %d: the tensor-core contraction needs q %% 8 == 0", l);
+            set_error(CIRC_ERR_UNSUPPORTED, "layer %d: the tensor-core contraction needs q %% 4 == 0", l);
             return CIRC_ERR_UNSUPPORTED;
         }
     }
@@ -189,7 +189,7 @@ int circ_stack_forward(circ_stack_handle s, const void* x, void* y, int batch, v
         if ((rc = ensure_workspace(L, stack_workspace(L, e))) != CIRC_OK) return rc;
         if ((rc = ensure_forms(L, tensor ? FORM_A_BF16 : FORM_A_F32, st)) != CIRC_OK) return rc;   // stacks use the embedded weights
         float* xop = static_cast<float*>(L->ws);
-        float* yop = xop + (((size_t)2 * e.Bh * L->geo.q * L->geo.k + 63) & ~(size_t)63);
+        float* yop = xop + (((size_t)2 * e.Bh * padded_q(L->geo.q) * L->geo.k + 63) & ~(size_t)63);   // (bfloat16 runs may be padded)
         if (!operand_ready) {
             const int xmode = !tensor ? 0 : (L->x_dtype == CIRC_BF16 ? 2 : 1);
             if ((rc = launch_input_fft(L, in, xop, xmode, e, st)) != CIRC_OK) return rc;

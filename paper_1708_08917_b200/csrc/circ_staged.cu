@@ -202,35 +202,49 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
     } else {
         // vector scatter: one work item = (bin, 4 consecutive transforms) = 16 bytes of (Re, Im) bfloat16
         // pairs per part; consecutive lanes = consecutive groups = consecutive memory.
+        // (q is a multiple of 4; runs are padded_q(q) entries long and the group that ends a run also zeroes its padding)
         __nv_bfloat16* xb = static_cast<__nv_bfloat16*>(xop);
         constexpr int GROUPS = TT / 4;
+        const int qs = padded_q(q);
+        const size_t real_sz = cols * qs * NPART, cplx_sz = (TWIN ? 4 : 2) * real_sz;
+        const uint2 zero2 = make_uint2(0u, 0u);
+        const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
         for (int item = threadIdx.x; item < GROUPS * K; item += kThreads) {
             const int grp = item % GROUPS, f = item / GROUPS;
             const long T0 = (long)blockIdx.x * TT + grp * 4;
-            if (T0 >= total) continue;                 // total is a multiple of 8 (q % 8 == 0)
+            if (T0 >= total) continue;                 // total is a multiple of 4
             int c, j;
             split_at<TT>(sp, grp * 4, q, c, j);
+            const bool pad = qs != q && j + 4 == q;    // this group ends its column's run
             const float4 za = *reinterpret_cast<const float4*>(&zs[f][grp * 4]);
             const float4 zb = *reinterpret_cast<const float4*>(&zs[f][grp * 4 + 2]);
             if (f == 0 || f == K / 2) {
                 __nv_bfloat16* xg = xb + problem_offset(f == 0 ? 0 : 1, real_sz, cplx_sz);
-                __nv_bfloat16* d0 = xg + (size_t)c * (NPART * q) + j;
-                __nv_bfloat16* d1 = xg + ((size_t)Bh + c) * (NPART * q) + j;
+                __nv_bfloat16* d0 = xg + (size_t)c * (NPART * qs) + j;
+                __nv_bfloat16* d1 = xg + ((size_t)Bh + c) * (NPART * qs) + j;
                 uint32_t l0, l1, l2, l3;
                 const uint32_t h0 = bf16_split_pair(za.x, za.z, l0), h1 = bf16_split_pair(zb.x, zb.z, l1);
                 const uint32_t h2 = bf16_split_pair(za.y, za.w, l2), h3 = bf16_split_pair(zb.y, zb.w, l3);
                 *reinterpret_cast<uint2*>(d0) = make_uint2(h0, h1);
                 *reinterpret_cast<uint2*>(d1) = make_uint2(h2, h3);
                 if constexpr (XMODE == 1) {
-                    *reinterpret_cast<uint2*>(d0 + q) = make_uint2(l0, l1);
-                    *reinterpret_cast<uint2*>(d1 + q) = make_uint2(l2, l3);
+                    *reinterpret_cast<uint2*>(d0 + qs) = make_uint2(l0, l1);
+                    *reinterpret_cast<uint2*>(d1 + qs) = make_uint2(l2, l3);
+                }
+                if (pad) {
+                    *reinterpret_cast<uint2*>(d0 + 4) = zero2;
+                    *reinterpret_cast<uint2*>(d1 + 4) = zero2;
+                    if constexpr (XMODE == 1) {
+                        *reinterpret_cast<uint2*>(d0 + qs + 4) = zero2;
+                        *reinterpret_cast<uint2*>(d1 + qs + 4) = zero2;
+                    }
                 }
             } else {
                 const bool mirror = f > K / 2;
                 const int g = mirror ? K - f : f;
                 const float sgn = mirror ? -1.f : 1.f;
                 __nv_bfloat16* d = xb + problem_offset(g + 1, real_sz, cplx_sz) +
-                                   ((size_t)(mirror ? Bh : 0) + c) * (NPART * 2 * q) + 2 * j;
+                                   ((size_t)(mirror ? Bh : 0) + c) * (NPART * 2 * qs) + 2 * j;
                 const float i0 = sgn * za.y, i1 = sgn * za.w, i2 = sgn * zb.y, i3 = sgn * zb.w;
                 uint32_t l0, l1, l2, l3;
                 const uint32_t h0 = bf16_split_pair(za.x, i0, l0), h1 = bf16_split_pair(za.z, i1, l1);
@@ -239,16 +253,20 @@ __device__ __forceinline__ void scatter_operand(const float2 (*zs)[Tile<K, EMAX>
                     // a word holds (re | im << 16): negating im flips its sign bit, swapping re and im swaps the halves
                     constexpr uint32_t S = 0x80000000u;
                     auto swp = [](uint32_t v) { return __byte_perm(v, 0u, 0x1032); };
-                    __nv_bfloat16* d2 = d + cols * (size_t)(NPART * 2 * q);
+                    __nv_bfloat16* d2 = d + cols * (size_t)(NPART * 2 * qs);
                     *reinterpret_cast<uint4*>(d) = make_uint4(h0 ^ S, h1 ^ S, h2 ^ S, h3 ^ S);
                     *reinterpret_cast<uint4*>(d2) = make_uint4(swp(h0), swp(h1), swp(h2), swp(h3));
                     if constexpr (XMODE == 1) {
-                        *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0 ^ S, l1 ^ S, l2 ^ S, l3 ^ S);
-                        *reinterpret_cast<uint4*>(d2 + 2 * q) = make_uint4(swp(l0), swp(l1), swp(l2), swp(l3));
+                        *reinterpret_cast<uint4*>(d + 2 * qs) = make_uint4(l0 ^ S, l1 ^ S, l2 ^ S, l3 ^ S);
+                        *reinterpret_cast<uint4*>(d2 + 2 * qs) = make_uint4(swp(l0), swp(l1), swp(l2), swp(l3));
                     }
                 } else {
                     *reinterpret_cast<uint4*>(d) = make_uint4(h0, h1, h2, h3);
-                    if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * q) = make_uint4(l0, l1, l2, l3);
+                    if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * qs) = make_uint4(l0, l1, l2, l3);
+                    if (pad) {                         // (twin columns are only used when there is no padding)
+                        *reinterpret_cast<uint4*>(d + 8) = zero4;
+                        if constexpr (XMODE == 1) *reinterpret_cast<uint4*>(d + 2 * qs + 8) = zero4;
+                    }
                 }
             }
         }
@@ -756,8 +774,8 @@ static bool latency_bound(long transforms, int k) {
 int launch_input_fft(const Layer* L, const void* x, void* xop, int xmode, const Extent& ext, cudaStream_t stream, bool twin) {
     const int q = L->geo.q, n = L->n;
     const long total = (long)ext.Bh * q;
-    if (xmode != 0 && (q % 8) != 0) {
-        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need q %% 8 == 0 (q=%d)", q);
+    if (xmode != 0 && (q % 4) != 0) {
+        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need q %% 4 == 0 (q=%d)", q);
         return CIRC_ERR_UNSUPPORTED;
     }
     if (twin && (xmode == 0 || embedded(L->geo))) {
@@ -925,8 +943,8 @@ int launch_relay(const Layer* L, const float* yop, void* xop_next, int xmode, co
         set_error(CIRC_ERR_ARG, "relay operand mode %d", xmode);
         return CIRC_ERR_ARG;
     }
-    if (xmode == 1 && (p % 8) != 0) {
-        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need p %% 8 == 0 (p=%d)", p);
+    if (xmode == 1 && (p % 4) != 0) {
+        set_error(CIRC_ERR_UNSUPPORTED, "bfloat16 operands need p %% 4 == 0 (p=%d)", p);
         return CIRC_ERR_UNSUPPORTED;
     }
     const bool small = latency_bound(total, L->geo.k);

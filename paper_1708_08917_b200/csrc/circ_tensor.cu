@@ -441,7 +441,8 @@ static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims
 
 static int round_up16(int v) { return (v + 15) & ~15; }
 
-bool tensor_supported(const Layer* L) { return (L->geo.q % 8) == 0 && encode_fn() != nullptr; }
+// q a multiple of 4: the input transforms hand over four column blocks at a time; the operands' runs are padded to 8
+bool tensor_supported(const Layer* L) { return (L->geo.q % 4) == 0 && encode_fn() != nullptr; }
 
 // Ring depth, CTAs per SM and grid for a planned launch; maps = {A real, A complex, X hi real, X lo real, X hi complex, X lo complex}.
 static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int taps, int kq_max, long ctas, cudaStream_t stream) {
@@ -505,7 +506,7 @@ static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int ta
 
 int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin) {
     const Geometry& geo = L->geo;
-    const int p = geo.p, q = geo.q, k = geo.k, taps = geo.taps;
+    const int p = geo.p, q = padded_q(geo.q), k = geo.k, taps = geo.taps;   // q: the (padded) run length of the operands
     TcArgs g;
     g.yop = yop;
     g.status = L->dev_status;

@@ -300,7 +300,7 @@ ContractionPlan plan_contraction(const Layer* L, const Extent& e) {
     ContractionPlan pl = {false, false};
     if (L->kind != 0) return pl;
     const long cols = 2L * e.Bh;
-    const bool twin_ok = !L->no_twin && !embedded(L->geo) && L->geo.p >= 16 && (long)L->geo.p >= 2 * cols;
+    const bool twin_ok = !L->no_twin && !embedded(L->geo) && L->geo.p >= 16 && (long)L->geo.p >= 2 * cols && L->geo.q % 8 == 0;
     const bool rows_ok = !L->no_rows_kernel;
     if (rows_ok && twin_ok && 2 * cols <= 256 && rows_tiles(L, true) >= 64) return ContractionPlan{true, true};
     if (rows_ok && cols <= 256 && rows_tiles(L, false) >= 64) return ContractionPlan{false, true};
@@ -353,7 +353,7 @@ RowsPieces rows_pieces(const Layer* L, const Extent& e, bool twin) {
 }
 
 int launch_contract_rows(const Layer* L, const __nv_bfloat16* xb, float* yop, const Extent& ext, int nsplit, cudaStream_t stream, bool twin) {
-    const int p = L->geo.p, q = L->geo.q, k = L->geo.k;
+    const int p = L->geo.p, q = padded_q(L->geo.q), k = L->geo.k;   // q: the (padded) run length of the operands
     const __nv_bfloat16* a_op = twin ? L->a_twin : L->a_bf16;
     if (!a_op || L->kind != 0) {
         set_error(CIRC_ERR_ARG, "the stored form of the spectra for this contraction has not been built, or not a fully-connected layer");

@@ -28,13 +28,13 @@ def _check(case, tol, want_s3):
     (64, 16, 8, 6002),     # 48016 transforms: even, last tile of 32 half full
     (16, 40, 8, 4000),     # one lane per transform
     (256, 6, 8, 15000),    # 16 lanes per transform, 45000 transforms
-    (128, 5, 3, 20000),    # q % 8 != 0: the fp32 FMA contraction feeds the same kernel
+    (128, 5, 3, 20000),    # q % 4 != 0: the fp32 FMA contraction feeds the same kernel
 ])
 def test_bulk_tiles_float32(k, p, q, batch):
     case = synth.fc_case(f"bulk_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
                          bias_var=0.01, relu=True)
     used = _check(case, TOL_F32, circ.CIRC_KERNEL_S3_BULK)
-    assert used == (circ.CIRC_VARIANT_TENSOR if q % 8 == 0 else circ.CIRC_VARIANT_STAGED)
+    assert used == (circ.CIRC_VARIANT_TENSOR if q % 4 == 0 else circ.CIRC_VARIANT_STAGED)
 
 
 def test_bulk_tiles_bfloat16():

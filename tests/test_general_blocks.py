@@ -21,7 +21,7 @@ def test_fc_any_block_size(k, p, q, batch):
     case = synth.fc_case(f"gen_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
                          bias_var=0.01, relu=(batch % 2 == 0))
     got, used = run_fc(case)
-    assert used == (circ.CIRC_VARIANT_TENSOR if q % 8 == 0 else circ.CIRC_VARIANT_STAGED)
+    assert used == (circ.CIRC_VARIANT_TENSOR if q % 4 == 0 else circ.CIRC_VARIANT_STAGED)
     assert not np.isnan(got).any()
     assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
 

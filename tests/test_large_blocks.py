@@ -16,11 +16,11 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("k", [512, 1024])
 @pytest.mark.parametrize("p,q,batch", [(1, 1, 1), (2, 3, 2), (3, 2, 5), (5, 4, 17), (2, 8, 40), (3, 16, 33), (9, 8, 130)])
 def test_fc_large_blocks(k, p, q, batch):
-    # q % 8 == 0 runs the tensor-core contraction, other q the fp32 FMA one; odd batches leave a half-filled pair
+    # q % 4 == 0 runs the tensor-core contraction (runs padded to 8 entries), other q the fp32 FMA one; odd batches leave a half-filled pair
     case = synth.fc_case(f"large_{k}_{p}_{q}_{batch}", p * k, q * k, k, batch, w_var=1.0 / (q * k), x_dist="normal",
                          bias_var=0.01, relu=(batch % 2 == 0))
     got, used = run_fc(case)
-    assert used == (circ.CIRC_VARIANT_TENSOR if q % 8 == 0 else circ.CIRC_VARIANT_STAGED)
+    assert used == (circ.CIRC_VARIANT_TENSOR if q % 4 == 0 else circ.CIRC_VARIANT_STAGED)
     assert not np.isnan(got).any()
     assert scale_rel_err(got, oracle_fc(case)) <= TOL_F32
 
