@@ -107,14 +107,24 @@ def fc_backward(w, x, g, convention: int = 0, want_gx: bool = True, want_gw: boo
     return gx, gw
 
 
-def conv(w, x, pad: int, bias=None, relu: bool = False, convention: int = 0) -> np.ndarray:
-    """Eq. 6 with zero padding: ``w[r][r][p][q][k]``, ``x[N][H][W][C]`` -> ``y[N][Ho][Wo][P]``."""
+def conv(w, x, pad: int, bias=None, relu: bool = False, convention: int = 0, stride: int = 1) -> np.ndarray:
+    """Eq. 6 with zero padding: ``w[r][r][p][q][k]``, ``x[N][H][W][C]`` -> ``y[N][Ho][Wo][P]``; ``stride`` > 1 keeps
+    every stride-th output position of it in both directions."""
     w = _d(w)
     x = _d(x)
     r, r2, p, q, k = w.shape
     assert r == r2
     N, H, W, C = x.shape
     assert C == q * k
+    if stride != 1:
+        assert stride >= 1
+        Ho, Wo = (H + 2 * pad - r) // stride + 1, (W + 2 * pad - r) // stride + 1
+        b = None if bias is None else _d(bias)
+        y = np.empty((N, Ho, Wo, p * k), dtype=np.float64)
+        _load().circ_oracle_conv_strided(ctypes.c_int(p * k), ctypes.c_int(C), ctypes.c_int(r), ctypes.c_int(pad), ctypes.c_int(stride),
+                                         ctypes.c_int(k), ctypes.c_int(convention), _ptr(w), _ptr(x), _ptr(b),
+                                         ctypes.c_int(int(relu)), ctypes.c_int(N), ctypes.c_int(H), ctypes.c_int(W), _ptr(y))
+        return y
     Ho, Wo = H + 2 * pad - r + 1, W + 2 * pad - r + 1
     b = None if bias is None else _d(bias)
     y = np.empty((N, Ho, Wo, p * k), dtype=np.float64)

@@ -147,6 +147,22 @@ ORACLE_API void circ_oracle_conv(int c_out, int c_in, int r, int pad, int k, int
 }
 
 /*
+ * Strided CONV layer: Eq. 6 evaluated at every `stride`-th output position in both directions (the subsampling
+ * convolution of the networks the paper evaluates; Eq. 6 itself is the stride-1 case):
+ *   y(n, i, j, :) = [Eq. 6 output](n, stride i, stride j, :),   Ho = (H + 2 pad - r) / stride + 1, Wo likewise.
+ */
+ORACLE_API void circ_oracle_conv_strided(int c_out, int c_in, int r, int pad, int stride, int k, int convention, const double* w,
+                                         const double* x, const double* bias, int relu, int N, int H, int W, double* y) {
+    const int Ho = (H + 2 * pad - r) / stride + 1, Wo = (W + 2 * pad - r) / stride + 1;
+#pragma omp parallel for collapse(3) schedule(static)
+    for (int nn = 0; nn < N; ++nn)
+        for (int ho = 0; ho < Ho; ++ho)
+            for (int wo = 0; wo < Wo; ++wo)
+                conv_pixel(c_out, c_in, r, pad, k, convention, w, x, bias, relu, H, W, nn, stride * ho, stride * wo,
+                           y + (((size_t)nn * Ho + ho) * Wo + wo) * c_out);
+}
+
+/*
  * The same definition evaluated only at the listed output pixels (for checks at
  * sizes where the whole tensor would take too long): pix[3*t..3*t+2] = (n, ho, wo),
  * y_out[t][c_out].

@@ -201,3 +201,45 @@ def test_planted_pool_mistake_is_caught(tmp_path, name):
     lib = tmp_path / f"{name}.so"
     subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(lib), str(out), "-lm"], check=True)
     assert not _pool_pins_hold(ctypes.CDLL(str(lib))), f"pins did not notice mutation {name}"
+
+
+# ---- the strided convolution: mistakes planted there must break its hand case -----------------------------------------
+STRIDE_MUTATIONS = {
+    "stride_ignored_on_columns": ("nn, stride * ho, stride * wo,", "nn, stride * ho, wo,"),
+    "stride_rows_and_columns_swapped": ("nn, stride * ho, stride * wo,", "nn, stride * wo, stride * ho,"),
+    "stride_extent_without_division": ("const int Ho = (H + 2 * pad - r) / stride + 1, Wo = (W + 2 * pad - r) / stride + 1;\n#pragma omp parallel for collapse(3) schedule(static)\n    for (int nn = 0; nn < N; ++nn)\n        for (int ho = 0; ho < Ho; ++ho)\n            for (int wo = 0; wo < Wo; ++wo)\n                conv_pixel(c_out, c_in, r, pad, k, convention, w, x, bias, relu, H, W, nn, stride * ho",
+                                       "const int Ho = (H + 2 * pad - r) / stride + 1, Wo = (W + 2 * pad - r) / stride + 1;\n#pragma omp parallel for collapse(3) schedule(static)\n    for (int nn = 0; nn < N; ++nn)\n        for (int ho = 0; ho < Ho; ++ho)\n            for (int wo = 0; wo < Wo; ++wo)\n                conv_pixel(c_out, c_in, r, pad, k, convention, w, x, bias, relu, H, W, nn, stride * ho + 1"),
+}
+
+
+def _stride_pins_hold(lib) -> bool:
+    ok = True
+    x = np.arange(12, dtype=np.float64)
+    w = np.full(1, 2.0)
+    y = np.full(4, np.nan)
+    lib.circ_oracle_conv_strided(1, 1, 1, 0, 2, 1, 0, w.ctypes.data_as(_dp), x.ctypes.data_as(_dp), None, 0, 1, 3, 4, y.ctypes.data_as(_dp))
+    ok &= bool(np.array_equal(y, [0.0, 4.0, 16.0, 20.0]))
+    x = np.arange(16, dtype=np.float64)
+    w = np.ones(4)
+    y = np.full(4, np.nan)
+    lib.circ_oracle_conv_strided(1, 1, 2, 0, 2, 1, 0, w.ctypes.data_as(_dp), x.ctypes.data_as(_dp), None, 0, 1, 4, 4, y.ctypes.data_as(_dp))
+    ok &= bool(np.array_equal(y, [10.0, 18.0, 42.0, 50.0]))
+    return bool(ok)
+
+
+def test_unmutated_copy_passes_the_stride_pins(tmp_path):
+    (tmp_path / "plain.c").write_text(SRC.read_text())
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(tmp_path / "plain.so"), str(tmp_path / "plain.c"), "-lm"], check=True)
+    assert _stride_pins_hold(ctypes.CDLL(str(tmp_path / "plain.so")))
+
+
+@pytest.mark.parametrize("name", sorted(STRIDE_MUTATIONS))
+def test_planted_stride_mistake_is_caught(tmp_path, name):
+    old, new = STRIDE_MUTATIONS[name]
+    text = SRC.read_text()
+    assert text.count(old) == 1, f"mutation anchor for {name} must be unique"
+    out = tmp_path / f"{name}.c"
+    out.write_text(text.replace(old, new, 1))
+    lib = tmp_path / f"{name}.so"
+    subprocess.run(["gcc", "-O1", "-shared", "-fPIC", "-o", str(lib), str(out), "-lm"], check=True)
+    assert not _stride_pins_hold(ctypes.CDLL(str(lib))), f"pins did not notice mutation {name}"

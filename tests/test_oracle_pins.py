@@ -426,3 +426,35 @@ def test_pool_invariants():
     # transposing the image transposes the result (rows and columns are treated alike)
     xt = np.ascontiguousarray(x.transpose(0, 2, 1, 3))
     assert np.array_equal(oracle.pool(xt, 3, 2, oracle.POOL_MAX), oracle.pool(x, 3, 2, oracle.POOL_MAX).transpose(0, 2, 1, 3))
+
+
+# ---- strided convolution: Eq. 6 kept at every stride-th output position -------------------------------------------------
+@pytest.mark.parametrize("r,pad,stride,p,q,k,N,H,W", [(3, 1, 2, 2, 2, 4, 2, 9, 8), (3, 0, 2, 1, 2, 4, 1, 7, 7), (5, 2, 3, 1, 1, 3, 1, 11, 10),
+                                                      (1, 0, 2, 2, 1, 2, 2, 5, 4), (3, 1, 4, 1, 1, 2, 1, 13, 6), (2, 0, 2, 1, 1, 4, 1, 5, 8)])
+def test_strided_conv_against_torch_float64(r, pad, stride, p, q, k, N, H, W):
+    w = RNG.standard_normal((r, r, p, q, k))
+    x = RNG.standard_normal((N, H, W, q * k))
+    bias = RNG.standard_normal(p * k)
+    for conv in (0, 1):
+        F = _dense_filters(w, k, conv)
+        ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2), torch.from_numpy(F), bias=torch.from_numpy(bias),
+                                         padding=pad, stride=stride).permute(0, 2, 3, 1).numpy()
+        got = oracle.conv(w, x, pad, bias=bias, convention=conv, stride=stride)
+        assert got.shape == ref.shape == (N, (H + 2 * pad - r) // stride + 1, (W + 2 * pad - r) // stride + 1, p * k)
+        np.testing.assert_allclose(got, ref, atol=1e-11)
+        # and it is the stride-1 result of Eq. 6 kept at every stride-th position, rows and columns alike
+        full = oracle.conv(w, x, pad, bias=bias, convention=conv)
+        assert np.array_equal(got, full[:, ::stride, ::stride, :][:, :got.shape[1], :got.shape[2], :])
+
+
+def test_strided_conv_hand_case():
+    # one channel (k = 1 makes the block a scalar), 1 x 1 filter of weight 2, stride 2 on a 3 x 4 image: picks and doubles
+    # pixels (0,0), (0,2), (2,0), (2,2); a row index mistaken for a column index would pick others
+    x = np.arange(12, dtype=np.float64).reshape(1, 3, 4, 1)
+    w = np.full((1, 1, 1, 1, 1), 2.0)
+    got = oracle.conv(w, x, 0, stride=2)
+    assert got.shape == (1, 2, 2, 1) and np.array_equal(got.reshape(-1), [0.0, 4.0, 16.0, 20.0])
+    # 2 x 2 filter of ones, stride 2, no padding: sums of the four 2 x 2 corners of a 4 x 4 image
+    x = np.arange(16, dtype=np.float64).reshape(1, 4, 4, 1)
+    got = oracle.conv(np.ones((2, 2, 1, 1, 1)), x, 0, stride=2)
+    assert np.array_equal(got.reshape(-1), [10.0, 18.0, 42.0, 50.0])
