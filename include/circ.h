@@ -300,6 +300,18 @@ CIRC_API int circ_device_status(circ_handle h);
 CIRC_API const char* circ_last_error(void);
 CIRC_API int circ_last_code(void);
 
+/*
+ * circ_conv_set_stride -- strided convolution: every stride-th output position of Eq. 6 is kept in both directions,
+ * y(n, i, j, :) = [Eq. 6](n, stride i, stride j, :), Ho = (H + 2 pad - r) / stride + 1, Wo likewise (the subsampling
+ * convolution of the networks the paper evaluates; Eq. 6 itself is stride 1, the default).  Only the positions that are
+ * kept are computed: the input tile of the tensor-core contraction is fetched as one sub-tile per phase (row, column offset
+ * modulo the stride) by strided TMA boxes, and a filter tap reads a shifted view of its phase's sub-tile.
+ *   stride : 1 .. 4.  Strides above 1 need the tensor-core contraction (c_in / k a multiple of 4; circ_conv_forward
+ *            returns CIRC_ERR_UNSUPPORTED otherwise) and are not served by the backward calls.
+ * Errors: CIRC_ERR_ARG (not a convolution handle), CIRC_ERR_SHAPE (stride out of range).
+ */
+CIRC_API int circ_conv_set_stride(circ_handle h, int stride);
+
 /* Pooling operations of circ_pool_forward. */
 enum { CIRC_POOL_MAX = 0, CIRC_POOL_AVG = 1, CIRC_POOL_L2 = 2 };
 

@@ -70,6 +70,7 @@ SIGNATURES = {
     "circ_debug_set_fused_split": (_ci, [_vp, _ci]),
     "circ_debug_set_contraction": (_ci, [_vp, _ci, _ci]),
     "circ_debug_set_transforms": (_ci, [_vp, _ci, _ci]),
+    "circ_conv_set_stride": (_ci, [_vp, _ci]),
     "circ_pool_forward": (_ci, [_vp, _vp, _ci, _ci, _ci, _ci, _ci, _ci, _ci, _ci, _vp]),
     "circ_last_error": (ctypes.c_char_p, []),
     "circ_last_code": (_ci, []),
@@ -166,6 +167,10 @@ def circ_fc_forward(h: int, x, y, batch: int, stream=None) -> None:
 def circ_conv_forward(h: int, x, y, N: int, H: int, W: int, stream=None) -> None:
     """Enqueue the channel-last convolution ``x[N][H][W][C] -> y[N][Ho][Wo][P]``."""
     _check(load().circ_conv_forward(h, _ptr(x), _ptr(y), N, H, W, _stream(stream)))
+
+
+def circ_conv_set_stride(h: int, stride: int) -> None:
+    _check(load().circ_conv_set_stride(h, int(stride)))
 
 
 def circ_pool_forward(x, y, N: int, H: int, W: int, C: int, window: int, stride: int, mode: int, dtype: int, stream=None) -> None:

@@ -126,7 +126,7 @@ Layer* make_layer(int kind, int m, int n, int k, int taps, int r, int pad, const
     L->kind = kind;
     L->m = m;
     L->n = n;
-    L->geo = Geometry{m / k, n / k, kt, taps, r, pad, k};
+    L->geo = Geometry{m / k, n / k, kt, taps, r, pad, k, 1};
     L->x_dtype = L->y_dtype = (kind == 1 ? CIRC_BF16 : CIRC_F32);
     L->variant = CIRC_VARIANT_AUTO;
     if (cudaGetDevice(&L->device) != cudaSuccess) {
@@ -245,8 +245,8 @@ Extent conv_extent(const Layer* L, int N, int H, int W) {
     Extent e;
     e.H = H;
     e.W = W;
-    e.Ho = H + 2 * L->geo.pad - L->geo.r + 1;
-    e.Wo = W + 2 * L->geo.pad - L->geo.r + 1;
+    e.Ho = (H + 2 * L->geo.pad - L->geo.r) / L->geo.stride + 1;
+    e.Wo = (W + 2 * L->geo.pad - L->geo.r) / L->geo.stride + 1;
     e.Nh = (N + 1) / 2;
     e.B = N * H * W;
     e.Bh = e.Nh * H * W;
@@ -435,6 +435,10 @@ int circ_conv_forward(circ_handle h, const void* x, void* y, int N, int H, int W
         return CIRC_ERR_UNSUPPORTED;
     }
     const bool tensor = L->variant == CIRC_VARIANT_TENSOR || (L->variant == CIRC_VARIANT_AUTO && tensor_supported(L));
+    if (L->geo.stride > 1 && !tensor) {
+        set_error(CIRC_ERR_UNSUPPORTED, "a strided convolution runs on the tensor-core contraction only (needs c_in / k to be a multiple of 4)");
+        return CIRC_ERR_UNSUPPORTED;
+    }
     return run_staged(L, x, y, conv_extent(L, N, H, W), static_cast<cudaStream_t>(stream), tensor);
 }
 
@@ -488,7 +492,7 @@ int circ_conv_forward_host(circ_handle h, const void* x_host, void* y_host, int 
         set_error(CIRC_ERR_ARG, "bad handle, NULL host pointer or empty image");
         return CIRC_ERR_ARG;
     }
-    const int Ho = H + 2 * L->geo.pad - L->geo.r + 1, Wo = W + 2 * L->geo.pad - L->geo.r + 1;
+    const int Ho = (H + 2 * L->geo.pad - L->geo.r) / L->geo.stride + 1, Wo = (W + 2 * L->geo.pad - L->geo.r) / L->geo.stride + 1;
     if (Ho < 1 || Wo < 1) {
         set_error(CIRC_ERR_SHAPE, "image smaller than the filter");
         return CIRC_ERR_SHAPE;
@@ -540,6 +544,20 @@ int circ_set_activation(circ_handle h, int relu) {
         return CIRC_ERR_ARG;
     }
     L->relu = relu;
+    return CIRC_OK;
+}
+
+int circ_conv_set_stride(circ_handle h, int stride) {
+    Layer* L = reinterpret_cast<Layer*>(h);
+    if (!L || L->kind != 1) {
+        set_error(CIRC_ERR_ARG, "circ_conv_set_stride needs a convolution handle");
+        return CIRC_ERR_ARG;
+    }
+    if (stride < 1 || stride > 4) {
+        set_error(CIRC_ERR_SHAPE, "stride=%d must be in [1, 4]", stride);
+        return CIRC_ERR_SHAPE;
+    }
+    L->geo.stride = stride;
     return CIRC_OK;
 }
 

@@ -652,6 +652,10 @@ int circ_conv_backward_input(circ_handle h, const void* grad_y, void* grad_x, in
         set_error(CIRC_ERR_ARG, "circ_conv_backward_input needs a convolution handle");
         return CIRC_ERR_ARG;
     }
+    if (reinterpret_cast<Layer*>(h)->geo.stride != 1) {
+        set_error(CIRC_ERR_UNSUPPORTED, "the backward passes serve stride 1 only");
+        return CIRC_ERR_UNSUPPORTED;
+    }
     const int Ho = H + 2 * L->geo.pad - L->geo.r + 1, Wo = W + 2 * L->geo.pad - L->geo.r + 1;
     if (N < 1 || H < 1 || W < 1 || Ho < 1 || Wo < 1) {
         set_error(CIRC_ERR_SHAPE, "bad image extent N=%d H=%d W=%d for r=%d pad=%d", N, H, W, L->geo.r, L->geo.pad);
@@ -670,6 +674,10 @@ int circ_conv_backward_weight(circ_handle h, const void* x, const void* grad_y, 
     if (!L || L->kind != 1) {
         set_error(CIRC_ERR_ARG, "circ_conv_backward_weight needs a convolution handle");
         return CIRC_ERR_ARG;
+    }
+    if (reinterpret_cast<Layer*>(h)->geo.stride != 1) {
+        set_error(CIRC_ERR_UNSUPPORTED, "the backward passes serve stride 1 only");
+        return CIRC_ERR_UNSUPPORTED;
     }
     if (!x || !grad_y || !grad_w || (reinterpret_cast<uintptr_t>(x) & 15u) || (reinterpret_cast<uintptr_t>(grad_y) & 15u) ||
         (reinterpret_cast<uintptr_t>(grad_w) & 15u)) {

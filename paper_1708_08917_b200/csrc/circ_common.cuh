@@ -43,6 +43,7 @@ struct Geometry {
                       // vectors folded back, y[t] = c[t] + c[t + ku], and the linear convolution is a circular one of
                       // any length k >= 2 ku - 1.  S0 and S1 zero-pad w_ij and x_j to k, S3 folds; everything in
                       // between works on k-point spectra and does not know.
+    int stride;       // CONV: every stride-th output position of Eq. 6 is kept (1 unless circ_conv_set_stride)
 };
 __host__ __device__ inline bool embedded(const Geometry& g) { return g.ku != g.k; }
 

@@ -140,16 +140,17 @@ inline EncodeTiledFn tensor_map_encoder() {
     return fn;
 }
 
+// elem_strides (optional): traversal stride per dimension; a box extent of N x stride then brings N elements.
 inline int encode_tensor_map(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes,
                   const cuuint32_t* box, CUtensorMapDataType dtype = CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
-                  CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
+                  CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B, const cuuint32_t* elem_strides = nullptr) {
     EncodeTiledFn fn = tensor_map_encoder();
     if (!fn) {
         set_error(CIRC_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
         return CIRC_ERR_CUDA;
     }
     cuuint32_t ones[5] = {1, 1, 1, 1, 1};
-    const CUresult r = fn(map, dtype, (cuuint32_t)rank, base, dims, strides_bytes, box, ones,
+    const CUresult r = fn(map, dtype, (cuuint32_t)rank, base, dims, strides_bytes, box, elem_strides ? elem_strides : ones,
                           CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {

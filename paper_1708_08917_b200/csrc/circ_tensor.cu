@@ -42,7 +42,8 @@ struct TcArgs {
     int tw, th;              // output pixels per tile (tw wide, th high)
     int pitch;               // input tile row pitch in pixels: tw + r - 1 (halo included)
     int xrows;               // pixels of the input tile that the TMA box brings: pitch * (th + r - 1)
-    int xalloc;              // pixels reserved per stage for the input tile (covers every tap's 128-row view)
+    int xalloc;              // pixels reserved per sub-tile of the input tile (whole swizzle groups)
+    int xtail;               // pixels reserved behind the last sub-tile of a part, so that every tap's 128-row view stays inside the stage
     int tiles_w, tiles_h;    // tiles per image (real problems)
     int twin;                // complex problems in twin-column form: p rows, columns [real parts | imaginary parts]
     int Wo_c, tiles_w_c;     // output columns and column tiles of a complex problem (twice the real ones when twin)
@@ -56,6 +57,11 @@ struct TcArgs {
     uint32_t spin_limit;     // polls before a wait gives up (kSpinLimit; a few thousand under fault injection)
     int pdl_late;            // issue the dependent-launch trigger after the CTA's last tile instead of first thing
     int no_copy;             // fault injection (tests only): the producer announces its bytes but issues no copy
+    int stride;              // strided convolution: output pixel (i, j) reads input pixels (stride i + di - pad, stride j + dj - pad)
+    int sp, nph;             // phases per direction min(stride, r) and in all (sp * sp): the input tile comes as one
+                             // sub-tile per phase (a, b) = (row, column) offset modulo the stride, each fetched by a
+                             // strided TMA box; tap (di, dj) reads sub-tile (di % stride, dj % stride) shifted by
+                             // (di / stride, dj / stride).  stride 1: one sub-tile, the tile with its halo.
 };
 
 // Instruction descriptor: bf16 x bf16 -> f32, both operands K-major, M = 128, N = bn.
@@ -158,7 +164,8 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
     // stage ring, 1024-byte aligned (the swizzle pattern repeats every 1024 bytes); every stage has room
     // for the input tile and for all taps' weight tiles of the widest row tile
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const uint32_t x_bytes = (uint32_t)g.xalloc * 128;                                    // one part (hi or lo) of the input tile
+    const uint32_t xph_bytes = (uint32_t)g.xalloc * 128;                                  // one sub-tile (phase) of one part of the input tile
+    const uint32_t x_bytes = (uint32_t)g.nph * xph_bytes + (uint32_t)g.xtail * 128;       // one part (hi or lo) of the input tile
     const uint32_t stage_bytes = (uint32_t)g.nsplit * (x_bytes + (uint32_t)g.taps * (uint32_t)bn_max * 128);
     unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~(uintptr_t)1023);
     uint32_t acc_cols = 32;                      // columns of one accumulator
@@ -206,7 +213,7 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                 const CUtensorMap* map_xhi = t.real ? &map_xhi_real : &map_xhi_cplx;
                 const CUtensorMap* map_xlo = t.real ? &map_xlo_real : &map_xlo_cplx;
                 const uint32_t a_bytes = (uint32_t)t.bn * 128;           // one tap's weight tile
-                const uint32_t tx_bytes = (uint32_t)g.nsplit * ((uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes);
+                const uint32_t tx_bytes = (uint32_t)g.nsplit * ((uint32_t)g.nph * (uint32_t)g.xrows * 128 + (uint32_t)g.taps * a_bytes);
                 const int kblocks = (t.Kq + kKBlock - 1) / kKBlock;
                 // one iteration = one K block: input tile (hi [, lo]) and all taps' weight tiles (hi [, lo])
                 {
@@ -223,10 +230,13 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                         }
                         // input tile with its halo: starts pad pixels before the output tile (negative and
                         // out-of-image coordinates read the zero fill)
-                        tma_load_5d(xs, map_xhi, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v, t.prob_in_kind);
-                        if (g.nsplit == 2)
-                            tma_load_5d(xs + x_bytes, map_xlo, &full_bar[s], kb * kKBlock, t.wo0 - g.pad, t.ho0 - g.pad, t.v,
-                                        t.prob_in_kind);
+                        for (int ph = 0; ph < g.nph; ++ph) {
+                            const int pa = ph / g.sp, pb = ph - pa * g.sp;
+                            const int w0 = g.stride * t.wo0 - g.pad + pb, h0 = g.stride * t.ho0 - g.pad + pa;
+                            tma_load_5d(xs + ph * xph_bytes, map_xhi, &full_bar[s], kb * kKBlock, w0, h0, t.v, t.prob_in_kind);
+                            if (g.nsplit == 2)
+                                tma_load_5d(xs + x_bytes + ph * xph_bytes, map_xlo, &full_bar[s], kb * kKBlock, w0, h0, t.v, t.prob_in_kind);
+                        }
                         // one box brings every tap's weight tile, hi parts first, then lo parts: [part][row][128 B]
                         tma_load_4d(as, map_a, &full_bar[s], kb * kKBlock, t.row0, 0, t.prob_in_kind);
                         if (issued < g.stages) ++issued;
@@ -308,7 +318,22 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
                             for (int prod = 0; prod < g.npass; ++prod) {          // hi*hi, hi*lo(A), lo(X)*hi
                                 const uint64_t dx = prod == 2 ? dx_lo : dx_hi;
                                 const uint64_t da = prod == 1 ? da_lo : da_hi;
-                                if (g.r == 3) {
+                                if (g.stride > 1) {
+                                    // tap (di, dj) reads the sub-tile of phase (di % stride, dj % stride), shifted by the quotients
+                                    uint64_t db = da;
+                                    for (int di = 0; di < g.r; ++di) {
+                                        const int pa = di % g.stride, qa = di / g.stride;
+                                        for (int dj = 0; dj < g.r; ++dj, db += tap_step) {
+                                            const int pb = dj % g.stride, qb = dj / g.stride;
+                                            const uint64_t dxx = dx + (uint64_t)(pa * g.sp + pb) * (uint64_t)(xph_bytes >> 4) +
+                                                                 (uint64_t)qa * row_step + (uint64_t)(qb * 8);
+                                            tc_mma_bf16(d_tmem, dxx, db, idesc, accumulate);
+                                            for (int k4 = 1; k4 < ksteps; ++k4)
+                                                tc_mma_bf16(d_tmem, dxx + (uint64_t)(k4 * 2), db + (uint64_t)(k4 * 2), idesc, 1u);
+                                            accumulate = 1u;
+                                        }
+                                    }
+                                } else if (g.r == 3) {
                                     issue_taps_k<3>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
                                 } else if (g.r == 1) {
                                     issue_taps_k<1>(ksteps, d_tmem, dx, da, row_step, tap_step, idesc, accumulate);
@@ -435,8 +460,10 @@ contract_tc_kernel(const __grid_constant__ CUtensorMap map_a_real, const __grid_
 
 // ---- host side ---------------------------------------------------------------------------------
 static EncodeTiledFn encode_fn() { return tensor_map_encoder(); }
-static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes, const cuuint32_t* box) {
-    return encode_tensor_map(map, base, rank, dims, strides_bytes, box);
+static int encode(CUtensorMap* map, void* base, int rank, const cuuint64_t* dims, const cuuint64_t* strides_bytes, const cuuint32_t* box,
+                  const cuuint32_t* elem_strides = nullptr) {
+    return encode_tensor_map(map, base, rank, dims, strides_bytes, box, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B,
+                             elem_strides);
 }
 
 static int round_up16(int v) { return (v + 15) & ~15; }
@@ -447,7 +474,7 @@ bool tensor_supported(const Layer* L) { return (L->geo.q % 4) == 0 && encode_fn(
 // Ring depth, CTAs per SM and grid for a planned launch; maps = {A real, A complex, X hi real, X lo real, X hi complex, X lo complex}.
 static int launch_planned(TcArgs& g, const CUtensorMap* maps, int nsplit, int taps, int kq_max, long ctas, cudaStream_t stream) {
     const int bn_max = g.bn_real > g.bn_cplx ? g.bn_real : g.bn_cplx;
-    const size_t stage_bytes = (size_t)nsplit * ((size_t)g.xalloc * 128 + (size_t)taps * bn_max * 128);
+    const size_t stage_bytes = (size_t)nsplit * (((size_t)g.nph * g.xalloc + g.xtail) * 128 + (size_t)taps * bn_max * 128);
     if (stage_bytes + 1024 > 199 * 1024) {
         set_error(CIRC_ERR_UNSUPPORTED, "filter taps x row tile do not fit one shared-memory stage (%zu bytes)", stage_bytes);
         return CIRC_ERR_UNSUPPORTED;
@@ -531,16 +558,29 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     }
     g.twin = twin ? 1 : 0;
     g.Wo_c = twin ? 2 * g.Wo : g.Wo;
-    const int halo = geo.r - 1;
-    g.tw = g.Wo_c < kTileCols - halo ? g.Wo_c : kTileCols - halo;   // the wider problem kind sets the tile
-    g.pitch = g.tw + halo;
-    g.th = (kTileCols - g.tw) / g.pitch + 1;          // (th - 1) * pitch + tw <= 128 MMA rows
-    if (g.th > g.Ho) g.th = g.Ho;
-    g.xrows = g.pitch * (g.th + halo);
-    {
+    // strided convolution: tiles live in output-pixel space; each phase's sub-tile has (r - 1) / stride halo pixels
+    g.stride = L->kind == 1 ? geo.stride : 1;
+    g.sp = g.stride < geo.r ? g.stride : geo.r;
+    g.nph = g.sp * g.sp;
+    const int halo = (geo.r - 1) / g.stride;
+    int tw_cap = kTileCols - halo;
+    if (256 / g.stride - halo < tw_cap) tw_cap = 256 / g.stride - halo;   // a strided box spans pitch x stride pixels, at most 256
+    for (;;) {
+        g.tw = g.Wo_c < tw_cap ? g.Wo_c : tw_cap;   // the wider problem kind sets the tile
+        g.pitch = g.tw + halo;
+        g.th = (kTileCols - g.tw) / g.pitch + 1;          // (th - 1) * pitch + tw <= 128 MMA rows
+        if (g.th > g.Ho) g.th = g.Ho;
+        g.xrows = g.pitch * (g.th + halo);
+        // a tap's view starts up to halo rows and halo pixels into its sub-tile and spans 128 pixel slots: views that
+        // run past their sub-tile read the next one (or the tail) into output slots that are never stored
         const int reach = halo * g.pitch + halo + kTileCols;   // last row any tap's 128-row view touches, plus one
-        const int need = g.xrows > reach ? g.xrows : reach;
-        g.xalloc = (need + 7) & ~7;                            // whole 1024-byte swizzle groups
+        g.xalloc = (g.xrows + 7) & ~7;                         // whole 1024-byte swizzle groups
+        g.xtail = reach > g.xalloc ? ((reach - g.xalloc + 7) & ~7) : 0;
+        // several sub-tiles (a strided convolution) of a wide, flat tile can outgrow a stage: narrower tiles are
+        // taller, and the halo rows weigh less
+        const long x_b = (long)nsplit * ((long)g.nph * g.xalloc + g.xtail) * 128;
+        if (g.nph == 1 || x_b + (long)nsplit * taps * 16 * 128 <= 160 * 1024 || tw_cap <= 8) break;
+        tw_cap /= 2;
     }
     g.tiles_w = (g.Wo + g.tw - 1) / g.tw;
     g.tiles_w_c = (g.Wo_c + g.tw - 1) / g.tw;
@@ -551,7 +591,7 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
     {
         // all taps' weight tiles of one K block share a stage with the input tile: narrow the row
         // tile until a stage fits half of the shared memory (two stages), or all of it at worst
-        const long x_b = (long)nsplit * g.xalloc * 128;
+        const long x_b = (long)nsplit * ((long)g.nph * g.xalloc + g.xtail) * 128;
         long room = 96 * 1024 - x_b;
         if (room < (long)nsplit * taps * 16 * 128) room = 198 * 1024 - x_b;
         int cap = (int)(room / ((long)nsplit * taps * 128)) & ~15;
@@ -596,17 +636,19 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         cuuint32_t box[4] = {kKBlock, (cuuint32_t)g.bn_cplx, a_parts, 1};
         if ((rc = encode(&ma_c, const_cast<__nv_bfloat16*>(a_op) + 2 * a_real_elems, 4, dims, str, box)) != CIRC_OK) return rc;
     }
-    // X: [problem][v][h][w][part][Kq]
+    // X: [problem][v][h][w][part][Kq]; a strided convolution fetches every stride-th pixel of a phase (a box extent of
+    // N x stride brings N pixels)
+    const cuuint32_t xstr[5] = {1, (cuuint32_t)g.stride, (cuuint32_t)g.stride, 1, 1};
     const size_t cols_in = (size_t)g.V * g.H * g.W;
     const size_t x_real_elems = cols_in * nsplit * q;
     {
         cuuint64_t dims[5] = {(cuuint64_t)q, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.V, 2};
         cuuint64_t str[4] = {(cuuint64_t)nsplit * q * 2, (cuuint64_t)g.W * nsplit * q * 2,
                              (cuuint64_t)g.H * g.W * nsplit * q * 2, (cuuint64_t)x_real_elems * 2};
-        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, (cuuint32_t)(g.th + halo), 1, 1};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)(g.pitch * g.stride), (cuuint32_t)((g.th + halo) * g.stride), 1, 1};
         __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb);
-        if ((rc = encode(&mxh_r, base, 5, dims, str, box)) != CIRC_OK) return rc;
-        if ((rc = encode(&mxl_r, base + (nsplit == 2 ? q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxh_r, base, 5, dims, str, box, xstr)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxl_r, base + (nsplit == 2 ? q : 0), 5, dims, str, box, xstr)) != CIRC_OK) return rc;
     }
     {
         const int nc = k / 2 - 1 > 0 ? k / 2 - 1 : 1;
@@ -614,10 +656,10 @@ int launch_contract_tc(const Layer* L, const __nv_bfloat16* xb, float* yop, cons
         cuuint64_t dims[5] = {(cuuint64_t)2 * q, wc, (cuuint64_t)g.H, (cuuint64_t)g.V, (cuuint64_t)nc};
         cuuint64_t str[4] = {(cuuint64_t)nsplit * 2 * q * 2, wc * nsplit * 2 * q * 2,
                              (cuuint64_t)g.H * wc * nsplit * 2 * q * 2, (cuuint64_t)(twin ? 4 : 2) * x_real_elems * 2};
-        cuuint32_t box[5] = {kKBlock, (cuuint32_t)g.pitch, (cuuint32_t)(g.th + halo), 1, 1};
+        cuuint32_t box[5] = {kKBlock, (cuuint32_t)(g.pitch * g.stride), (cuuint32_t)((g.th + halo) * g.stride), 1, 1};
         __nv_bfloat16* base = const_cast<__nv_bfloat16*>(xb) + 2 * x_real_elems;
-        if ((rc = encode(&mxh_c, base, 5, dims, str, box)) != CIRC_OK) return rc;
-        if ((rc = encode(&mxl_c, base + (nsplit == 2 ? 2 * q : 0), 5, dims, str, box)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxh_c, base, 5, dims, str, box, xstr)) != CIRC_OK) return rc;
+        if ((rc = encode(&mxl_c, base + (nsplit == 2 ? 2 * q : 0), 5, dims, str, box, xstr)) != CIRC_OK) return rc;
     }
 
     const CUtensorMap maps[6] = {ma_r, ma_c, mxh_r, mxl_r, mxh_c, mxl_c};
@@ -638,12 +680,16 @@ static int launch_tc_one_kind(bool real, const __nv_bfloat16* xt, int x_rows, co
     g.npass = 3;
     g.spin_limit = kSpinLimit;
     g.no_copy = 0;
+    g.stride = 1;
+    g.sp = 1;
+    g.nph = 1;
     g.W = g.Wo = x_rows; g.H = g.Ho = 1; g.V = 1;
     g.tw = x_rows < kTileCols ? x_rows : kTileCols;
     g.pitch = g.tw;
     g.th = 1;
     g.xrows = g.tw;
     g.xalloc = kTileCols;
+    g.xtail = 0;
     g.tiles_w = g.tiles_w_c = (x_rows + g.tw - 1) / g.tw;
     g.tiles_h = 1;
     g.twin = 0;
