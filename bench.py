@@ -57,13 +57,13 @@ TABLE_ROWS = (["cfg1", "cfg2_b1", "cfg2_b16", "cfg2_b256", "cfg3_stack", "cfg4"]
 # when the source has changed since, the figure is withheld (reported as null).  These are builder-run
 # captures (profiles/), not counters read during this run: `traffic_source` in the JSON line says so.
 NCU_TRAFFIC: dict = {
-    ("sweep_n16384_k4_b1024", "contraction"): {"bytes_per_launch": 562115072 + 53097728, "source_sha256": "d8aae5e3d350cb95cce7c98b3d431c023a5b0e756240bfa5fdc94a4febe642d8"},
-    ("sweep_n16384_k4_b1", "fused_fc"): {"bytes_per_launch": 268547584 + 3823872, "source_sha256": "b9ba9386726b06f2e3c224c12e7a946d67c050f28211b6514922226939366a3c"},
-    ("sweep_n16384_k64_b1024", "contraction"): {"bytes_per_launch": 100209152 + 26082304, "source_sha256": "d8aae5e3d350cb95cce7c98b3d431c023a5b0e756240bfa5fdc94a4febe642d8"},
-    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6300928, "source_sha256": "d8aae5e3d350cb95cce7c98b3d431c023a5b0e756240bfa5fdc94a4febe642d8"},
+    ("sweep_n16384_k4_b1024", "contraction"): {"bytes_per_launch": 616559616, "source_sha256": "92cec56a36476480a1ded93e200f58eb5fed3f5a33f90191daf70a4c15f8f513"},
+    ("sweep_n16384_k4_b1", "fused_fc"): {"bytes_per_launch": 272659200, "source_sha256": "b9ba9386726b06f2e3c224c12e7a946d67c050f28211b6514922226939366a3c"},
+    ("sweep_n16384_k64_b1024", "contraction"): {"bytes_per_launch": 126377984, "source_sha256": "92cec56a36476480a1ded93e200f58eb5fed3f5a33f90191daf70a4c15f8f513"},
+    ("cfg4", "contraction"): {"bytes_per_launch": 13097984, "source_sha256": "92cec56a36476480a1ded93e200f58eb5fed3f5a33f90191daf70a4c15f8f513"},
     ("cfg2_b256", "input_fft"): {"bytes_per_launch": 4212736, "source_sha256": "92670eeeee80adeed252110b54bdb9fa814258a2354f4f6a324b74a2cc8c680a"},
-    ("cfg2_b256", "output_ifft"): {"bytes_per_launch": 4239616, "source_sha256": "92670eeeee80adeed252110b54bdb9fa814258a2354f4f6a324b74a2cc8c680a"},
-    ("cfg4", "contraction"): {"bytes_per_launch": 13059072, "source_sha256": "d8aae5e3d350cb95cce7c98b3d431c023a5b0e756240bfa5fdc94a4febe642d8"},
+    ("cfg2_b256", "contraction"): {"bytes_per_launch": 6309888, "source_sha256": "92cec56a36476480a1ded93e200f58eb5fed3f5a33f90191daf70a4c15f8f513"},
+    ("cfg2_b256", "output_ifft"): {"bytes_per_launch": 4235776, "source_sha256": "92670eeeee80adeed252110b54bdb9fa814258a2354f4f6a324b74a2cc8c680a"},
 }
 
 
